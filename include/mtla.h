@@ -1,0 +1,155 @@
+/*
+ * mtla.h: C ABI of the B200 (sm_100a) Multi-head Temporal Latent Attention library.
+ *
+ * One handle is one MTLA attention layer (Section 4 of the paper) together with the
+ * compressed temporal-latent cache of a batch of sequences that advance in lock-step.
+ * Notation follows the paper: d (model dim), n_h heads of d_h, latent rank r, decoupled
+ * RoPE dim d_h^R (written d_R here), temporal stride s, hyper-network width d_w.
+ *
+ * Conventions for every call
+ *   - Returns MTLA_OK (0) or a negative mtla_status.  Argument errors are detected before
+ *     anything is enqueued and leave the handle unchanged.
+ *   - "device" pointers are CUDA device addresses, 16-byte aligned; "host" pointers are
+ *     ordinary host addresses.  `stream` is a cudaStream_t passed as void* (NULL = the
+ *     legacy default stream).  Calls enqueue work on `stream` and return; the caller
+ *     synchronises.  Calls on one handle must be issued in order on one stream.
+ *   - Ownership: the caller owns x, y, the weight buffers (may be freed once mtla_create
+ *     has completed on its stream) and the arena (must outlive the handle and must not be
+ *     touched while the handle lives).  The library owns only the host-side handle.
+ *     Nothing here calls cudaMalloc: all device memory is carved from the arena.
+ *   - Element type of x, y, weights and cache is config.dtype (fp32 or bf16); reductions
+ *     are fp32.  Matrices are row-major.
+ */
+#ifndef MTLA_H_
+#define MTLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mtla_handle mtla_handle;
+
+typedef enum {
+  MTLA_OK = 0,
+  MTLA_ERR_INVALID_ARG = -1,      /* null pointer, misaligned pointer, non-positive size */
+  MTLA_ERR_UNSUPPORTED_SHAPE = -2,/* dims outside what the kernels are built for (see mtla_create) */
+  MTLA_ERR_ARENA_TOO_SMALL = -3,
+  MTLA_ERR_CAPACITY = -4,         /* token count would exceed max_tokens / max_prefill_tokens */
+  MTLA_ERR_BATCH_MISMATCH = -5,   /* B differs from the batch the cache currently holds */
+  MTLA_ERR_CUDA = -6,             /* a CUDA runtime call or launch failed */
+  MTLA_ERR_STATE = -7,            /* call not valid in the handle's current state */
+  MTLA_ERR_DEVICE_TIMEOUT = -8    /* a bounded device-side wait gave up (reported by mtla_check) */
+} mtla_status;
+
+enum { MTLA_DTYPE_FP32 = 0, MTLA_DTYPE_BF16 = 1 };
+
+/* Layer dimensions (paper's Section 4 and 4.3) and capacities. */
+typedef struct {
+  int32_t d_model;            /* d */
+  int32_t n_heads;            /* n_h, 1..32 */
+  int32_t head_dim;           /* d_h, 64 or 128 */
+  int32_t latent_rank;        /* r, multiple of 64, <= 512 */
+  int32_t rope_dim;           /* d_R, even, multiple of 32, <= 64 */
+  int32_t stride;             /* s >= 1; s = 1 is plain multi-head latent attention (w = 1) */
+  int32_t hyper_dim;          /* d_w <= 256; 0 selects r/4 (Appendix: 256 -> 64) */
+  int32_t max_batch;          /* capacity in sequences */
+  int32_t max_tokens;         /* capacity in tokens per sequence: ceil(max_tokens/s) slots */
+  int32_t max_prefill_tokens; /* largest T of one mtla_prefill call; 0 = no prefill workspace */
+  int32_t dtype;              /* MTLA_DTYPE_* */
+  float ln_eps;               /* 0 selects 1e-5 */
+  float rope_theta;           /* 0 selects 10000 */
+} mtla_config;
+
+/* Device pointers to the parameters, row-major [in][out], element type config.dtype.
+ * They are repacked into the arena by mtla_create and not referenced afterwards.
+ * Bias pointers may be NULL (treated as zero). */
+typedef struct {
+  const void* w_q;       /* [d][n_h*d_h]      Eq. 7 */
+  const void* w_qr;      /* [d][n_h*d_R]      RoPE queries, Section 4.3 */
+  const void* w_r;       /* [d][r]            Eq. 8 */
+  const void* w_kr;      /* [d][d_R]          shared RoPE key, Section 4.3 */
+  const void* ln_gamma;  /* [r]               LayerNorm after Eq. 8 */
+  const void* ln_beta;   /* [r] */
+  const void* w_k;       /* [r][n_h*d_h]      Eq. 9 */
+  const void* w_v;       /* [r][n_h*d_h]      Eq. 10 */
+  const void* w_o;       /* [n_h*d_h][d]      Eq. 11 */
+  const void* hyp_c_w;   /* [r][d_w]          Eq. 13, Linear(c_i) */
+  const void* hyp_c_b;   /* [d_w] or NULL */
+  const void* hyp_pe_w;  /* [r][d_w]          Eq. 13, Linear(pe_j) */
+  const void* hyp_pe_b;  /* [d_w] or NULL */
+} mtla_weights;
+
+/* Device bytes mtla_create needs for this configuration (weights, tables, cache, decode
+ * scratch and, if max_prefill_tokens > 0, the prefill workspace).  0 if cfg is invalid. */
+size_t mtla_arena_bytes(const mtla_config* cfg);
+
+/* Builds a layer (Section 4): validates cfg, repacks the weights into `arena` (device,
+ * 1024-byte aligned, >= mtla_arena_bytes(cfg)), builds the positional tables (sinusoidal
+ * pe_j pushed through Linear(pe_j) of Eq. 13; RoPE angles of Section 4.3) and starts with
+ * an empty cache.  The packing kernels run on `stream`.  *out receives the handle. */
+int mtla_create(const mtla_config* cfg, const mtla_weights* weights, void* arena,
+                size_t arena_bytes, void* stream, mtla_handle** out);
+
+/* Parallel prefill (Section 4.2 with the RoPE shortcut of Section 4.3): consumes T prompt
+ * tokens for each of B sequences, x device [B][T][d], and reproduces what T decode steps
+ * would have produced: y device [B][T][d] (may be NULL to skip the outputs), the
+ * ceil(T/s) cache slots, and the open slot if T is not a multiple of s.  The stride-aware
+ * causal mask is applied as a predicate, never materialised.  Requires an empty cache
+ * (tokens == 0), B <= max_batch, T <= min(max_prefill_tokens, max_tokens). */
+int mtla_prefill(mtla_handle* h, const void* x, int32_t B, int32_t T, void* y, void* stream);
+
+/* One incremental decoding step (Section 4.1, Eq. 13, Eq. 17) for every sequence:
+ * x device [B][d] is token number tokens+1; its latent is merged into slot
+ * ceil((tokens+1)/s) (a new slot opens when tokens mod s == 0), the slot's RoPE key is
+ * replaced by this token's, and y device [B][d] receives the attention output over all
+ * slots in the absorbed form.  B is the batch fixed by the preceding prefill / import, or
+ * by the first decode step on an empty cache. */
+int mtla_decode_step(mtla_handle* h, const void* x, int32_t B, void* y, void* stream);
+
+/* Same step with HOST buffers: copies x_host [B][d] to the device, runs the step and copies
+ * y back to y_host [B][d], all enqueued on `stream` (pinned host memory keeps it async). */
+int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y_host,
+                          void* stream);
+
+/* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3). */
+size_t mtla_cache_bytes(const mtla_handle* h);
+
+/* Releases the host-side handle.  The arena is the caller's. */
+int mtla_destroy(mtla_handle* h);
+
+/* ---- support calls (state inspection, cache checkpointing, diagnostics) ---- */
+
+/* Empties the cache (tokens = 0, batch unset).  Nothing is enqueued. */
+int mtla_reset(mtla_handle* h);
+
+/* Current position: tokens consumed per sequence, slots held (= ceil(tokens/s)), batch. */
+int mtla_position(const mtla_handle* h, int32_t* tokens, int32_t* slots, int32_t* batch);
+
+/* Copies the cache in use to dst (device), layout [B][slots][r + d_R], element type dtype;
+ * `bytes` must be >= mtla_cache_bytes(h). */
+int mtla_cache_export(mtla_handle* h, void* dst, size_t bytes, void* stream);
+
+/* Replaces the cache by src (device) [B][ceil(tokens/s)][r + d_R] and sets the position to
+ * `tokens`.  If tokens is not a multiple of s the last slot is open and its fp32
+ * accumulator is initialised from the stored value. */
+int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens, void* stream);
+
+/* Synchronises `stream` and reports a sticky device-side status (MTLA_ERR_DEVICE_TIMEOUT if
+ * a bounded wait inside a kernel gave up; MTLA_ERR_CUDA if the stream is in error). */
+int mtla_check(mtla_handle* h, void* stream);
+
+/* Number of kernels the library has launched on behalf of this handle since creation. */
+int64_t mtla_launch_count(const mtla_handle* h);
+
+/* Name of the decode-attention kernel variant the handle dispatches to ("fma" or "tcgen05"). */
+const char* mtla_attention_variant(const mtla_handle* h);
+
+const char* mtla_error_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTLA_H_ */

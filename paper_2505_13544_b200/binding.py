@@ -1,0 +1,249 @@
+"""ctypes binding over libmtla.so: argument marshalling only.
+
+Every function here has the name of the C call it wraps (see include/mtla.h) and passes
+torch tensors by data_ptr(); torch is used for device memory and streams, nothing else.
+There is no CPU fallback: if the library cannot be built or loaded the import of a symbol
+raises, and every non-zero status raises MTLAError.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+
+import torch
+
+from .build import LIB_PATH, build_library
+
+MTLA_DTYPE_FP32, MTLA_DTYPE_BF16 = 0, 1
+_DTYPES = {torch.float32: MTLA_DTYPE_FP32, torch.bfloat16: MTLA_DTYPE_BF16,
+           "fp32": MTLA_DTYPE_FP32, "bf16": MTLA_DTYPE_BF16}
+_TORCH_DTYPES = {MTLA_DTYPE_FP32: torch.float32, MTLA_DTYPE_BF16: torch.bfloat16}
+
+WEIGHT_NAMES = ("w_q", "w_qr", "w_r", "w_kr", "ln_gamma", "ln_beta", "w_k", "w_v", "w_o",
+                "hyp_c_w", "hyp_c_b", "hyp_pe_w", "hyp_pe_b")
+
+EXPORTED_SYMBOLS = (
+    "mtla_arena_bytes", "mtla_create", "mtla_prefill", "mtla_decode_step",
+    "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
+    "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
+    "mtla_attention_variant", "mtla_error_string")
+
+
+class MTLAError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {error_string(status)} ({status})")
+
+
+class mtla_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "d_model", "n_heads", "head_dim", "latent_rank", "rope_dim", "stride", "hyper_dim",
+        "max_batch", "max_tokens", "max_prefill_tokens", "dtype")] + [
+        ("ln_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
+
+
+class mtla_weights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads (building first if needed) the CUDA library; raises if that is impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    build_library()
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    cfg_p, w_p = ctypes.POINTER(mtla_config), ctypes.POINTER(mtla_weights)
+    sigs = {
+        "mtla_arena_bytes": (sz, [cfg_p]),
+        "mtla_create": (ctypes.c_int, [cfg_p, w_p, vp, sz, vp, ctypes.POINTER(vp)]),
+        "mtla_prefill": (ctypes.c_int, [vp, vp, i32, i32, vp, vp]),
+        "mtla_decode_step": (ctypes.c_int, [vp, vp, i32, vp, vp]),
+        "mtla_decode_step_host": (ctypes.c_int, [vp, vp, i32, vp, vp]),
+        "mtla_cache_bytes": (sz, [vp]),
+        "mtla_destroy": (ctypes.c_int, [vp]),
+        "mtla_reset": (ctypes.c_int, [vp]),
+        "mtla_position": (ctypes.c_int, [vp, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                         ctypes.POINTER(i32)]),
+        "mtla_cache_export": (ctypes.c_int, [vp, vp, sz, vp]),
+        "mtla_cache_import": (ctypes.c_int, [vp, vp, i32, i32, vp]),
+        "mtla_check": (ctypes.c_int, [vp, vp]),
+        "mtla_launch_count": (ctypes.c_int64, [vp]),
+        "mtla_attention_variant": (ctypes.c_char_p, [vp]),
+        "mtla_error_string": (ctypes.c_char_p, [ctypes.c_int]),
+    }
+    for name, (res, args) in sigs.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def error_string(status: int) -> str:
+    return load_library().mtla_error_string(status).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise MTLAError(status, where)
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+@dataclass
+class Handle:
+    """A live layer: the C handle plus the torch tensors that must outlive it."""
+    ptr: int
+    config: mtla_config
+    arena: torch.Tensor
+    dtype: torch.dtype
+    device: torch.device
+
+
+def make_config(*, d_model, n_heads, head_dim, latent_rank, rope_dim, stride, hyper_dim=0,
+                max_batch, max_tokens, max_prefill_tokens=0, dtype="bf16", ln_eps=0.0,
+                rope_theta=0.0) -> mtla_config:
+    return mtla_config(d_model, n_heads, head_dim, latent_rank, rope_dim, stride, hyper_dim,
+                       max_batch, max_tokens, max_prefill_tokens, _DTYPES[dtype], ln_eps,
+                       rope_theta)
+
+
+def mtla_arena_bytes(cfg: mtla_config) -> int:
+    return load_library().mtla_arena_bytes(ctypes.byref(cfg))
+
+
+def mtla_create(cfg: mtla_config, weights: dict, device="cuda:0", stream=None) -> Handle:
+    """weights: name -> CUDA tensor, row-major [in][out], dtype matching cfg.dtype."""
+    lib = load_library()
+    nbytes = lib.mtla_arena_bytes(ctypes.byref(cfg))
+    if nbytes == 0:
+        raise MTLAError(-2, "mtla_arena_bytes")
+    device = torch.device(device)
+    dtype = _TORCH_DTYPES[cfg.dtype]
+    with torch.cuda.device(device):
+        arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+        base = (arena.data_ptr() + 1023) // 1024 * 1024
+        w = mtla_weights()
+        keep = []
+        for name in WEIGHT_NAMES:
+            t = weights.get(name)
+            if t is None:
+                setattr(w, name, None)
+                continue
+            if t.dtype != dtype or not t.is_cuda:
+                raise TypeError(f"weight {name}: expected a {dtype} CUDA tensor")
+            t = t.contiguous()
+            keep.append(t)
+            setattr(w, name, t.data_ptr())
+        out = ctypes.c_void_p()
+        st = _stream_ptr(stream)
+        _check(lib.mtla_create(ctypes.byref(cfg), ctypes.byref(w), base, nbytes, st,
+                               ctypes.byref(out)), "mtla_create")
+        torch.cuda.current_stream().synchronize()   # packing done: weight tensors may be freed
+    return Handle(out.value, cfg, arena, dtype, device)
+
+
+def _expect(t: torch.Tensor, h: Handle, shape, name: str, cuda=True) -> None:
+    if t.dtype != h.dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise TypeError(f"{name}: expected contiguous {h.dtype} tensor of shape {tuple(shape)}")
+    if cuda != t.is_cuda:
+        raise TypeError(f"{name}: expected a {'CUDA' if cuda else 'host'} tensor")
+
+
+def mtla_prefill(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, want_output=True,
+                 stream=None):
+    """x [B][T][d] on the device; returns y [B][T][d] (or None when want_output is False)."""
+    b, t, d = x.shape
+    _expect(x, h, (b, t, h.config.d_model), "x")
+    if want_output and y is None:
+        y = torch.empty_like(x)
+    if y is not None:
+        _expect(y, h, x.shape, "y")
+    _check(load_library().mtla_prefill(h.ptr, x.data_ptr(), b, t,
+                                       y.data_ptr() if y is not None else None,
+                                       _stream_ptr(stream)), "mtla_prefill")
+    return y
+
+
+def mtla_decode_step(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, stream=None):
+    """x [B][d] on the device; returns y [B][d]."""
+    b = x.shape[0]
+    _expect(x, h, (b, h.config.d_model), "x")
+    if y is None:
+        y = torch.empty_like(x)
+    _expect(y, h, x.shape, "y")
+    _check(load_library().mtla_decode_step(h.ptr, x.data_ptr(), b, y.data_ptr(),
+                                           _stream_ptr(stream)), "mtla_decode_step")
+    return y
+
+
+def mtla_decode_step_host(h: Handle, x_host: torch.Tensor, y_host: torch.Tensor, stream=None):
+    """x_host, y_host [B][d] in (preferably pinned) host memory; copies are enqueued on the stream."""
+    b = x_host.shape[0]
+    _expect(x_host, h, (b, h.config.d_model), "x_host", cuda=False)
+    _expect(y_host, h, x_host.shape, "y_host", cuda=False)
+    _check(load_library().mtla_decode_step_host(h.ptr, x_host.data_ptr(), b, y_host.data_ptr(),
+                                                _stream_ptr(stream)), "mtla_decode_step_host")
+    return y_host
+
+
+def mtla_cache_bytes(h: Handle) -> int:
+    return load_library().mtla_cache_bytes(h.ptr)
+
+
+def mtla_destroy(h: Handle) -> None:
+    if h.ptr:
+        _check(load_library().mtla_destroy(h.ptr), "mtla_destroy")
+        h.ptr = 0
+
+
+def mtla_reset(h: Handle) -> None:
+    _check(load_library().mtla_reset(h.ptr), "mtla_reset")
+
+
+def mtla_position(h: Handle) -> tuple[int, int, int]:
+    """(tokens, slots, batch)."""
+    t, s, b = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _check(load_library().mtla_position(h.ptr, ctypes.byref(t), ctypes.byref(s),
+                                        ctypes.byref(b)), "mtla_position")
+    return t.value, s.value, b.value
+
+
+def mtla_cache_export(h: Handle, stream=None) -> torch.Tensor:
+    """The cache in use as a tensor [B][slots][r + d_R]."""
+    _, slots, batch = mtla_position(h)
+    width = h.config.latent_rank + h.config.rope_dim
+    out = torch.empty(batch, slots, width, dtype=h.dtype, device=h.device)
+    if out.numel():
+        _check(load_library().mtla_cache_export(h.ptr, out.data_ptr(),
+                                                out.numel() * out.element_size(),
+                                                _stream_ptr(stream)), "mtla_cache_export")
+    return out
+
+
+def mtla_cache_import(h: Handle, cache: torch.Tensor, tokens: int, stream=None) -> None:
+    """cache [B][ceil(tokens/s)][r + d_R] on the device."""
+    b = cache.shape[0]
+    slots = -(-tokens // h.config.stride)
+    _expect(cache, h, (b, slots, h.config.latent_rank + h.config.rope_dim), "cache")
+    _check(load_library().mtla_cache_import(h.ptr, cache.data_ptr(), b, tokens,
+                                            _stream_ptr(stream)), "mtla_cache_import")
+
+
+def mtla_check(h: Handle, stream=None) -> None:
+    _check(load_library().mtla_check(h.ptr, _stream_ptr(stream)), "mtla_check")
+
+
+def mtla_launch_count(h: Handle) -> int:
+    return load_library().mtla_launch_count(h.ptr)
+
+
+def mtla_attention_variant(h: Handle) -> str:
+    return load_library().mtla_attention_variant(h.ptr).decode()

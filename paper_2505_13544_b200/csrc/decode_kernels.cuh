@@ -1,0 +1,297 @@
+// Decode-step kernels that are not GEMMs: the fused LayerNorm / hyper-network gate / slot
+// update / RoPE kernel, the CUDA-core split-K attention over the compressed cache, and the
+// cross-split combine.
+#pragma once
+
+#include <math.h>
+
+#include "common.cuh"
+
+namespace mtla {
+
+// Column offsets of the fused input projection output row: [ q | q^R | c_raw | k^R ].
+struct ProjLayout {
+  int off_q, off_qr, off_c, off_kr, width;
+};
+
+struct PostArgs {
+  const float* p1;        // [B][proj.width] fused projection of this step's tokens (fp32)
+  ProjLayout proj;
+  const float* gamma;     // [r]
+  const float* beta;      // [r]
+  const float* hyp_c_w;   // [r][d_w] fp32
+  const float* hyp_c_b;   // [d_w]
+  const float* gate_pe;   // [d_w]: Linear(pe_j) of Eq. 13 for this step's slot number j
+  const float* rope_cos;  // [d_R/2] for this step's position
+  const float* rope_sin;  // [d_R/2]
+  float* open_acc;        // [B][r] fp32 running sum of the open slot
+  void* cache;            // [max_batch][max_slots][r + d_R]
+  void* q_t;              // [B][n_h*d_h] query in storage type (input of the absorption GEMM)
+  void* qt;               // [B][n_h][r + d_R] absorbed query; this kernel writes the RoPE tail
+  int n_heads, head_dim, r, dr, dw;
+  int max_slots, slot;    // slot = 0-based slot index receiving this token
+  int new_slot;           // 1 when the token opens the slot (tokens mod s == 0)
+  int use_gate;           // 0 at s == 1 (w = 1)
+  float ln_eps;
+  float q_scale;          // log2(e) / sqrt(d_h), folded into the absorbed query
+};
+
+// One CTA of 256 threads per sequence.  Section 4.1: c_i = LayerNorm(x_i W_r); Eq. 13 gate;
+// slot update (open: c_hat_j = w c, else c_hat_j += w c); Section 4.3: RoPE key replaces
+// the slot's key, RoPE queries are rotated and written behind the absorbed query.
+template <typename T>
+__global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
+  __shared__ float c_s[512];
+  __shared__ float part_s[256];
+  __shared__ float red_s[33];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const float* row = a.p1 + (long long)b * a.proj.width;
+
+  // LayerNorm over r (two-pass variance).
+  float s = 0.f;
+  for (int i = tid; i < a.r; i += 256) {
+    const float v = row[a.proj.off_c + i];
+    c_s[i] = v;
+    s += v;
+  }
+  const float mean = block_sum(s, red_s) / a.r;
+  float sq = 0.f;
+  for (int i = tid; i < a.r; i += 256) {
+    const float dlt = c_s[i] - mean;
+    sq += dlt * dlt;
+  }
+  __syncthreads();
+  const float rstd = rsqrtf(block_sum(sq, red_s) / a.r + a.ln_eps);
+  for (int i = tid; i < a.r; i += 256) c_s[i] = (c_s[i] - mean) * rstd * a.gamma[i] + a.beta[i];
+  __syncthreads();
+
+  // Hyper-network gate: w = sigmoid(<c A + a, Linear(pe_j)>).
+  float w = 1.f;
+  if (a.use_gate) {
+    const int parts = 256 / a.dw > 0 ? 256 / a.dw : 1;
+    float h = 0.f;
+    if (tid < parts * a.dw) {
+      const int n = tid % a.dw, part = tid / a.dw;
+      const int per = ceil_div(a.r, parts);
+      const int lo = part * per, hi = min(a.r, lo + per);
+      for (int i = lo; i < hi; ++i) h = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], h);
+    }
+    part_s[tid] = h;
+    __syncthreads();
+    float prod = 0.f;
+    if (tid < a.dw) {
+      float hn = a.hyp_c_b[tid];
+      for (int p = 0; p < parts; ++p) hn += part_s[p * a.dw + tid];
+      prod = hn * a.gate_pe[tid];
+    }
+    const float logit = block_sum(prod, red_s);
+    w = 1.f / (1.f + expf(-logit));
+  }
+
+  // Slot update: fp32 running sum, stored to the cache in the storage type.
+  const int W = a.r + a.dr;
+  T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + a.slot) * W;
+  float* acc = a.open_acc + (long long)b * a.r;
+  for (int i = tid; i < a.r; i += 256) {
+    const float v = (a.new_slot ? 0.f : acc[i]) + w * c_s[i];
+    acc[i] = v;
+    slot_row[i] = Elem<T>::from_float(v);
+  }
+  // RoPE key of this token replaces the slot's key.
+  for (int k = tid; k < a.dr / 2; k += 256) {
+    const float x0 = row[a.proj.off_kr + 2 * k], x1 = row[a.proj.off_kr + 2 * k + 1];
+    const float cs = a.rope_cos[k], sn = a.rope_sin[k];
+    slot_row[a.r + 2 * k] = Elem<T>::from_float(x0 * cs - x1 * sn);
+    slot_row[a.r + 2 * k + 1] = Elem<T>::from_float(x0 * sn + x1 * cs);
+  }
+  // Query in storage type for the absorption GEMM; rotated, pre-scaled RoPE queries.
+  T* q_t = static_cast<T*>(a.q_t) + (long long)b * a.n_heads * a.head_dim;
+  for (int i = tid; i < a.n_heads * a.head_dim; i += 256)
+    q_t[i] = Elem<T>::from_float(row[a.proj.off_q + i]);
+  T* qt = static_cast<T*>(a.qt) + (long long)b * a.n_heads * W;
+  const int half = a.dr / 2;
+  for (int i = tid; i < a.n_heads * half; i += 256) {
+    const int h = i / half, k = i % half;
+    const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k];
+    const float x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
+    const float cs = a.rope_cos[k], sn = a.rope_sin[k];
+    qt[h * W + a.r + 2 * k] = Elem<T>::from_float((x0 * cs - x1 * sn) * a.q_scale);
+    qt[h * W + a.r + 2 * k + 1] = Elem<T>::from_float((x0 * sn + x1 * cs) * a.q_scale);
+  }
+}
+
+struct AttnArgs {
+  const void* qt;      // [B][n_h][r + d_R], pre-scaled by log2(e)/sqrt(d_h)
+  const void* cache;   // [max_batch][max_slots][r + d_R]
+  float* o_part;       // [B * n_split][n_h][r] un-normalised partial outputs
+  float* ml_part;      // [B * n_split][n_h][2]: running max (log2 units), sum
+  int n_heads, r, dr, max_slots, n_slots, slots_per_split, n_split;
+};
+
+constexpr int kAttnFmaTile = 16;
+
+inline size_t attn_fma_smem_bytes(int nh_padded, int r, int dr) {
+  const int W = r + dr;
+  return sizeof(float) * ((size_t)nh_padded * W + (size_t)kAttnFmaTile * (W + 1) +
+                          (size_t)kAttnFmaTile * nh_padded + 3 * nh_padded);
+}
+
+// CUDA-core split-K decode attention in the absorbed form (Eq. 12 / Eq. 17): one CTA per
+// (split, sequence) streams its slot range once; every head reuses the staged tile.
+// NH = head count padded to the template instance, RPT = latent columns per thread.
+template <typename T, int NH, int RPT>
+__global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
+  extern __shared__ float smem[];
+  constexpr int TS = kAttnFmaTile;
+  constexpr int V = Elem<T>::kVec;
+  const int W = a.r + a.dr, WS = W + 1;
+  float* qs = smem;
+  float* tile = qs + NH * W;
+  float* ps = tile + TS * WS;
+  float* m_s = ps + TS * NH;
+  float* fac_s = m_s + NH;
+  const int tid = threadIdx.x, b = blockIdx.y, split = blockIdx.x;
+  const int slot0 = split * a.slots_per_split;
+  const int slot1 = min(a.n_slots, slot0 + a.slots_per_split);
+  const T* qt = static_cast<const T*>(a.qt) + (long long)b * a.n_heads * W;
+  const T* cache = static_cast<const T*>(a.cache) + (long long)b * a.max_slots * W;
+
+  for (int v = tid; v < NH * (W / V); v += 256) {
+    const int h = v / (W / V), kv = (v % (W / V)) * V;
+    float tmp[V];
+    if (h < a.n_heads) {
+      load_vec(qt + h * W + kv, tmp);
+    } else {
+#pragma unroll
+      for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < V; ++e) qs[h * W + kv + e] = tmp[e];
+  }
+  if (tid < NH) m_s[tid] = -INFINITY;
+  float acc[NH][RPT];
+#pragma unroll
+  for (int h = 0; h < NH; ++h)
+#pragma unroll
+    for (int q = 0; q < RPT; ++q) acc[h][q] = 0.f;
+  float l_run = 0.f;  // threads < NH: running softmax denominator of head tid
+
+  for (int t0 = slot0; t0 < slot1; t0 += TS) {
+    __syncthreads();
+    for (int v = tid; v < TS * (W / V); v += 256) {
+      const int sl = v / (W / V), kv = (v % (W / V)) * V;
+      float tmp[V];
+      if (t0 + sl < slot1) {
+        load_vec(cache + (long long)(t0 + sl) * W + kv, tmp);
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) tile[sl * WS + kv + e] = tmp[e];
+    }
+    __syncthreads();
+    for (int idx = tid; idx < NH * TS; idx += 256) {
+      const int sl = idx % TS, h = idx / TS;
+      const float* qrow = qs + h * W;
+      const float* trow = tile + sl * WS;
+      float d0 = 0.f, d1 = 0.f;
+      for (int k = 0; k < W; k += 2) {
+        d0 = fmaf(qrow[k], trow[k], d0);
+        d1 = fmaf(qrow[k + 1], trow[k + 1], d1);
+      }
+      ps[sl * NH + h] = (t0 + sl < slot1) ? d0 + d1 : -INFINITY;
+    }
+    __syncthreads();
+    if (tid < NH) {
+      float m_new = m_s[tid];
+#pragma unroll
+      for (int sl = 0; sl < TS; ++sl) m_new = fmaxf(m_new, ps[sl * NH + tid]);
+      fac_s[tid] = exp2f(m_s[tid] - m_new);  // 0 on the first tile (m = -inf)
+      m_s[tid] = m_new;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < NH * TS; idx += 256) {
+      const int h = idx % NH;
+      ps[idx] = exp2f(ps[idx] - m_s[h]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+      const float f = fac_s[h];
+#pragma unroll
+      for (int q = 0; q < RPT; ++q) acc[h][q] *= f;
+    }
+    for (int sl = 0; sl < TS; ++sl) {
+      float cv[RPT];
+#pragma unroll
+      for (int q = 0; q < RPT; ++q) {
+        const int col = tid + 256 * q;
+        cv[q] = col < a.r ? tile[sl * WS + col] : 0.f;
+      }
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        const float p = ps[sl * NH + h];
+#pragma unroll
+        for (int q = 0; q < RPT; ++q) acc[h][q] = fmaf(p, cv[q], acc[h][q]);
+      }
+    }
+    if (tid < NH) {
+      float sum = 0.f;
+#pragma unroll
+      for (int sl = 0; sl < TS; ++sl) sum += ps[sl * NH + tid];
+      l_run = l_run * fac_s[tid] + sum;
+    }
+  }
+
+  const long long unit = (long long)b * a.n_split + split;
+  float* o_part = a.o_part + unit * a.n_heads * a.r;
+#pragma unroll
+  for (int h = 0; h < NH; ++h) {
+    if (h >= a.n_heads) break;
+#pragma unroll
+    for (int q = 0; q < RPT; ++q) {
+      const int col = tid + 256 * q;
+      if (col < a.r) o_part[h * a.r + col] = acc[h][q];
+    }
+  }
+  if (tid < a.n_heads) {
+    a.ml_part[(unit * a.n_heads + tid) * 2] = m_s[tid];
+    a.ml_part[(unit * a.n_heads + tid) * 2 + 1] = l_run;
+  }
+}
+
+struct CombineArgs {
+  const float* o_part;   // [B * n_split][n_h][r]
+  const float* ml_part;  // [B * n_split][n_h][2]
+  void* o;               // [B][n_h][r] normalised attention output in latent space
+  int n_heads, r, n_split;
+};
+
+// Cross-split combine: rescales each split's partial by 2^(m_split - m) and normalises.
+// Grid (n_h, B), 128 threads over r.
+template <typename T>
+__global__ void __launch_bounds__(128) decode_combine_kernel(CombineArgs a) {
+  const int h = blockIdx.x, b = blockIdx.y;
+  float m = -INFINITY;
+  for (int sp = 0; sp < a.n_split; ++sp)
+    m = fmaxf(m, a.ml_part[(((long long)b * a.n_split + sp) * a.n_heads + h) * 2]);
+  float denom = 0.f;
+  for (int sp = 0; sp < a.n_split; ++sp) {
+    const float* ml = a.ml_part + (((long long)b * a.n_split + sp) * a.n_heads + h) * 2;
+    denom += exp2f(ml[0] - m) * ml[1];
+  }
+  const float inv = 1.f / denom;
+  T* o = static_cast<T*>(a.o) + ((long long)b * a.n_heads + h) * a.r;
+  for (int col = threadIdx.x; col < a.r; col += 128) {
+    float sum = 0.f;
+    for (int sp = 0; sp < a.n_split; ++sp) {
+      const long long unit = (long long)b * a.n_split + sp;
+      const float wgt = exp2f(a.ml_part[(unit * a.n_heads + h) * 2] - m);
+      sum = fmaf(wgt, a.o_part[(unit * a.n_heads + h) * a.r + col], sum);
+    }
+    o[col] = Elem<T>::from_float(sum * inv);
+  }
+}
+
+}  // namespace mtla

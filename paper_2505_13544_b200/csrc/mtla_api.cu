@@ -1,0 +1,567 @@
+// C ABI of the MTLA library (see include/mtla.h): validation, arena carving, weight
+// repacking and the launch sequences of the decode step and the prefill.
+#include "mtla.h"
+
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+#include "decode_kernels.cuh"
+#include "gemm_fma.cuh"
+#include "prefill_kernels.cuh"
+#include "setup_kernels.cuh"
+
+using namespace mtla;
+
+namespace {
+
+constexpr int kTargetCtas = 296;     // two CTAs per SM on a 148-SM part
+constexpr int kMinSlotsPerSplit = 64;
+
+struct ArenaPlan {
+  size_t wcat_t, w_k, w_kv_t, w_o_t;
+  size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
+  size_t cache, open_acc, err_flag;
+  size_t p1, q_t, qt, o_part, ml_part, o, v, x_stage, y_stage;
+  size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
+  size_t total;
+};
+
+struct Dims {
+  int d, nh, dh, r, dr, dw, s, W, ntot, max_slots, max_units;
+  size_t elem;
+  ProjLayout proj;
+};
+
+bool normalise(const mtla_config* in, mtla_config* out, Dims* dm) {
+  if (!in) return false;
+  mtla_config c = *in;
+  if (c.hyper_dim == 0) c.hyper_dim = c.latent_rank / 4;
+  if (c.ln_eps == 0.f) c.ln_eps = 1e-5f;
+  if (c.rope_theta == 0.f) c.rope_theta = 10000.f;
+  if (c.d_model <= 0 || c.d_model % 8) return false;
+  if (c.n_heads < 1 || c.n_heads > 32) return false;
+  if (c.head_dim != 64 && c.head_dim != 128) return false;
+  if (c.latent_rank < 64 || c.latent_rank > 512 || c.latent_rank % 64) return false;
+  if (c.rope_dim != 32 && c.rope_dim != 64) return false;
+  if (c.stride < 1) return false;
+  if (c.hyper_dim < 1 || c.hyper_dim > 256) return false;
+  if (c.max_batch < 1 || c.max_tokens < 1 || c.max_prefill_tokens < 0) return false;
+  if (c.dtype != MTLA_DTYPE_FP32 && c.dtype != MTLA_DTYPE_BF16) return false;
+  if (!(c.ln_eps > 0.f) || !(c.rope_theta > 0.f)) return false;
+  if ((long long)c.max_batch * c.max_tokens > (1ll << 31)) return false;
+  *out = c;
+  dm->d = c.d_model; dm->nh = c.n_heads; dm->dh = c.head_dim; dm->r = c.latent_rank;
+  dm->dr = c.rope_dim; dm->dw = c.hyper_dim; dm->s = c.stride;
+  dm->W = dm->r + dm->dr;
+  dm->elem = c.dtype == MTLA_DTYPE_BF16 ? 2 : 4;
+  dm->proj.off_q = 0;
+  dm->proj.off_qr = dm->nh * dm->dh;
+  dm->proj.off_c = dm->proj.off_qr + dm->nh * dm->dr;
+  dm->proj.off_kr = dm->proj.off_c + dm->r;
+  dm->proj.width = dm->proj.off_kr + dm->dr;
+  dm->ntot = dm->proj.width;
+  dm->max_slots = ceil_div(c.max_tokens, c.stride);
+  dm->max_units = kTargetCtas + c.max_batch;
+  return true;
+}
+
+void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes, 1024);
+    return at;
+  };
+  const size_t e = dm.elem, B = c.max_batch;
+  const size_t hd = (size_t)dm.nh * dm.dh;
+  p->wcat_t = take((size_t)dm.ntot * dm.d * e);
+  p->w_k = take((size_t)dm.r * hd * e);
+  p->w_kv_t = take(2 * hd * dm.r * e);
+  p->w_o_t = take((size_t)dm.d * hd * e);
+  p->gamma = take(dm.r * 4);
+  p->beta = take(dm.r * 4);
+  p->hyp_c_w = take((size_t)dm.r * dm.dw * 4);
+  p->hyp_c_b = take(dm.dw * 4);
+  p->hyp_pe_w = take((size_t)dm.r * dm.dw * 4);
+  p->hyp_pe_b = take(dm.dw * 4);
+  p->gate_pe = take((size_t)dm.max_slots * dm.dw * 4);
+  p->rope_cos = take((size_t)c.max_tokens * (dm.dr / 2) * 4);
+  p->rope_sin = take((size_t)c.max_tokens * (dm.dr / 2) * 4);
+  p->cache = take(B * dm.max_slots * dm.W * e);
+  p->open_acc = take(B * dm.r * 4);
+  p->err_flag = take(16);
+  p->p1 = take(B * dm.ntot * 4);
+  p->q_t = take(B * hd * e);
+  p->qt = take(B * dm.nh * dm.W * e);
+  p->o_part = take((size_t)dm.max_units * dm.nh * dm.r * 4);
+  p->ml_part = take((size_t)dm.max_units * dm.nh * 2 * 4);
+  p->o = take(B * dm.nh * dm.r * e);
+  p->v = take(B * hd * e);
+  p->x_stage = take(B * dm.d * e);
+  p->y_stage = take(B * dm.d * e);
+  const size_t rows = B * (size_t)c.max_prefill_tokens;
+  p->pf_p1 = take(rows * dm.ntot * 4);
+  p->pf_qcat = take(rows * dm.nh * (dm.dh + dm.dr) * e);
+  p->pf_cprime = take(rows * dm.r * e);
+  p->pf_kr = take(rows * dm.dr * e);
+  p->pf_kv = take(rows * 2 * hd * e);
+  p->pf_attn = take(rows * hd * e);
+  p->total = off;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+struct mtla_handle {
+  mtla_config cfg;
+  Dims dm;
+  ArenaPlan plan;
+  char* arena;
+  int tokens;   // tokens consumed per sequence
+  int batch;    // 0 while the cache is empty and no batch has been fixed
+  int64_t launches;
+  bool attn_smem_ready, pf_smem_ready;
+
+  template <typename P> P* at(size_t off) const { return reinterpret_cast<P*>(arena + off); }
+};
+
+namespace {
+
+#define MTLA_CUDA(call)                       \
+  do {                                        \
+    if ((call) != cudaSuccess) return MTLA_ERR_CUDA; \
+  } while (0)
+
+template <typename T>
+int launch_transpose(mtla_handle* h, const void* src, void* dst, int K, int N, int ld_src,
+                     int ld_dst, cudaStream_t st) {
+  dim3 grid(ceil_div(N, 32), ceil_div(K, 32)), block(32, 8);
+  transpose_kernel<T><<<grid, block, 0, st>>>(static_cast<const T*>(src), static_cast<T*>(dst),
+                                              K, N, ld_src, ld_dst);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+template <typename T>
+int launch_widen(mtla_handle* h, const void* src, float* dst, long long n, cudaStream_t st) {
+  widen_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(static_cast<const T*>(src), dst, n);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+template <typename TIn, typename TOut>
+int gemm(mtla_handle* h, const void* a, const void* bt, void* c, int m, int n, int k, int lda,
+         int ldb, int ldc, float alpha, int batches, long long za, long long zb, long long zc,
+         cudaStream_t st) {
+  GemmArgs g;
+  g.a = a; g.bt = bt; g.c = c; g.m = m; g.n = n; g.k = k;
+  g.lda = lda; g.ldb = ldb; g.ldc = ldc; g.za = za; g.zb = zb; g.zc = zc; g.alpha = alpha;
+  h->launches++;
+  return launch_gemm_nt_fma<TIn, TOut>(g, batches, st) == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+#define MTLA_TRY(expr)            \
+  do {                            \
+    const int rc_ = (expr);       \
+    if (rc_ != MTLA_OK) return rc_; \
+  } while (0)
+
+template <typename T>
+int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
+  const Dims& dm = h->dm;
+  const ArenaPlan& p = h->plan;
+  const int hd = dm.nh * dm.dh;
+  T* wcat = h->at<T>(p.wcat_t);
+  // Fused input projection, stored [out][in]: rows [ q | q^R | c | k^R ].
+  MTLA_TRY(launch_transpose<T>(h, w->w_q, wcat + (size_t)dm.proj.off_q * dm.d, dm.d, hd, hd, dm.d, st));
+  MTLA_TRY(launch_transpose<T>(h, w->w_qr, wcat + (size_t)dm.proj.off_qr * dm.d, dm.d,
+                               dm.nh * dm.dr, dm.nh * dm.dr, dm.d, st));
+  MTLA_TRY(launch_transpose<T>(h, w->w_r, wcat + (size_t)dm.proj.off_c * dm.d, dm.d, dm.r, dm.r, dm.d, st));
+  MTLA_TRY(launch_transpose<T>(h, w->w_kr, wcat + (size_t)dm.proj.off_kr * dm.d, dm.d, dm.dr, dm.dr, dm.d, st));
+  // W_K as given serves the query absorption ([r][n_h*d_h]: out = r, in = d_h per head).
+  MTLA_CUDA(cudaMemcpyAsync(h->at<T>(p.w_k), w->w_k, (size_t)dm.r * hd * sizeof(T),
+                            cudaMemcpyDeviceToDevice, st));
+  // [W_K^T ; W_V^T] stored [out][in] = [2*n_h*d_h][r] for the up-projections.
+  MTLA_TRY(launch_transpose<T>(h, w->w_k, h->at<T>(p.w_kv_t), dm.r, hd, hd, dm.r, st));
+  MTLA_TRY(launch_transpose<T>(h, w->w_v, h->at<T>(p.w_kv_t) + (size_t)hd * dm.r, dm.r, hd, hd, dm.r, st));
+  MTLA_TRY(launch_transpose<T>(h, w->w_o, h->at<T>(p.w_o_t), hd, dm.d, dm.d, hd, st));
+  MTLA_TRY(launch_widen<T>(h, w->ln_gamma, h->at<float>(p.gamma), dm.r, st));
+  MTLA_TRY(launch_widen<T>(h, w->ln_beta, h->at<float>(p.beta), dm.r, st));
+  MTLA_TRY(launch_widen<T>(h, w->hyp_c_w, h->at<float>(p.hyp_c_w), (long long)dm.r * dm.dw, st));
+  MTLA_TRY(launch_widen<T>(h, w->hyp_c_b, h->at<float>(p.hyp_c_b), dm.dw, st));
+  MTLA_TRY(launch_widen<T>(h, w->hyp_pe_w, h->at<float>(p.hyp_pe_w), (long long)dm.r * dm.dw, st));
+  MTLA_TRY(launch_widen<T>(h, w->hyp_pe_b, h->at<float>(p.hyp_pe_b), dm.dw, st));
+  gate_pe_table_kernel<<<dm.max_slots, 256, 0, st>>>(h->at<float>(p.hyp_pe_w), h->at<float>(p.hyp_pe_b),
+                                                     h->at<float>(p.gate_pe), dm.r, dm.dw);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  const long long n_rope = (long long)h->cfg.max_tokens * (dm.dr / 2);
+  rope_table_kernel<<<(unsigned)((n_rope + 255) / 256), 256, 0, st>>>(
+      h->at<float>(p.rope_cos), h->at<float>(p.rope_sin), h->cfg.max_tokens, dm.dr / 2,
+      (double)h->cfg.rope_theta);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.err_flag), 0, 16, st));
+  return MTLA_OK;
+}
+
+template <typename T, int NH>
+int launch_attn_fma_rpt(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
+  const size_t smem = attn_fma_smem_bytes(NH, a.r, a.dr);
+  dim3 grid(a.n_split, B);
+  if (a.r <= 256) {
+    if (!h->attn_smem_ready)
+      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, NH, 1>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    decode_attn_fma_kernel<T, NH, 1><<<grid, 256, smem, st>>>(a);
+  } else {
+    if (!h->attn_smem_ready)
+      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, NH, 2>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    decode_attn_fma_kernel<T, NH, 2><<<grid, 256, smem, st>>>(a);
+  }
+  h->attn_smem_ready = true;
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  return MTLA_OK;
+}
+
+template <typename T>
+int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
+  if (a.n_heads <= 4) return launch_attn_fma_rpt<T, 4>(h, a, B, st);
+  if (a.n_heads <= 8) return launch_attn_fma_rpt<T, 8>(h, a, B, st);
+  if (a.n_heads <= 16) return launch_attn_fma_rpt<T, 16>(h, a, B, st);
+  return launch_attn_fma_rpt<T, 32>(h, a, B, st);
+}
+
+// The decode step (Section 4.1): a1 fused projection, a2-a5 post kernel, a6 absorption,
+// a7 split-K attention + combine, a8 value and output projections.
+template <typename T>
+int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) {
+  const Dims& dm = h->dm;
+  const ArenaPlan& p = h->plan;
+  const int hd = dm.nh * dm.dh;
+  const int i0 = h->tokens;            // 0-based index of this token
+  const int slot = i0 / dm.s;
+  const int n_slots = slot + 1;
+
+  MTLA_TRY((gemm<T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d, dm.d,
+                           dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+
+  PostArgs pa;
+  pa.p1 = h->at<float>(p.p1);
+  pa.proj = dm.proj;
+  pa.gamma = h->at<float>(p.gamma);
+  pa.beta = h->at<float>(p.beta);
+  pa.hyp_c_w = h->at<float>(p.hyp_c_w);
+  pa.hyp_c_b = h->at<float>(p.hyp_c_b);
+  pa.gate_pe = h->at<float>(p.gate_pe) + (size_t)slot * dm.dw;
+  pa.rope_cos = h->at<float>(p.rope_cos) + (size_t)i0 * (dm.dr / 2);
+  pa.rope_sin = h->at<float>(p.rope_sin) + (size_t)i0 * (dm.dr / 2);
+  pa.open_acc = h->at<float>(p.open_acc);
+  pa.cache = h->at<void>(p.cache);
+  pa.q_t = h->at<void>(p.q_t);
+  pa.qt = h->at<void>(p.qt);
+  pa.n_heads = dm.nh; pa.head_dim = dm.dh; pa.r = dm.r; pa.dr = dm.dr; pa.dw = dm.dw;
+  pa.max_slots = dm.max_slots; pa.slot = slot;
+  pa.new_slot = (i0 % dm.s) == 0;
+  pa.use_gate = dm.s > 1;
+  pa.ln_eps = h->cfg.ln_eps;
+  pa.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+  decode_post_kernel<T><<<B, 256, 0, st>>>(pa);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+
+  // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head.
+  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.q_t), h->at<T>(p.w_k), h->at<T>(p.qt), B, dm.r, dm.dh, hd, hd,
+                       dm.nh * dm.W, pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
+
+  AttnArgs aa;
+  aa.qt = h->at<void>(p.qt);
+  aa.cache = h->at<void>(p.cache);
+  aa.o_part = h->at<float>(p.o_part);
+  aa.ml_part = h->at<float>(p.ml_part);
+  aa.n_heads = dm.nh; aa.r = dm.r; aa.dr = dm.dr; aa.max_slots = dm.max_slots;
+  aa.n_slots = n_slots;
+  int want = ceil_div(kTargetCtas, B);
+  int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
+  if (n_split < 1) n_split = 1;
+  aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
+  aa.n_split = ceil_div(n_slots, aa.slots_per_split);
+  MTLA_TRY(launch_attn_fma<T>(h, aa, B, st));
+
+  CombineArgs ca;
+  ca.o_part = aa.o_part; ca.ml_part = aa.ml_part; ca.o = h->at<void>(p.o);
+  ca.n_heads = dm.nh; ca.r = dm.r; ca.n_split = aa.n_split;
+  decode_combine_kernel<T><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+
+  // a8: v_h = o_h W_{V,h} per head, then y = concat_h(v_h) W_O.
+  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r, h->at<T>(p.v), B,
+                       dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f, dm.nh, dm.r,
+                       (long long)dm.dh * dm.r, dm.dh, st)));
+  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.v), h->at<T>(p.w_o_t), y, B, dm.d, hd, hd, hd, dm.d, 1.f, 1, 0,
+                       0, 0, st)));
+  return MTLA_OK;
+}
+
+template <typename T>
+int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaStream_t st) {
+  const Dims& dm = h->dm;
+  const ArenaPlan& p = h->plan;
+  const int hd = dm.nh * dm.dh;
+  const int rows = B * T_len;
+  const float q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+
+  MTLA_TRY((gemm<T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot, dm.d,
+                           dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  PrefillPostArgs pa;
+  pa.p1 = h->at<float>(p.pf_p1);
+  pa.proj = dm.proj;
+  pa.gamma = h->at<float>(p.gamma);
+  pa.beta = h->at<float>(p.beta);
+  pa.hyp_c_w = h->at<float>(p.hyp_c_w);
+  pa.hyp_c_b = h->at<float>(p.hyp_c_b);
+  pa.gate_pe = h->at<float>(p.gate_pe);
+  pa.rope_cos = h->at<float>(p.rope_cos);
+  pa.rope_sin = h->at<float>(p.rope_sin);
+  pa.open_acc = h->at<float>(p.open_acc);
+  pa.cache = h->at<void>(p.cache);
+  pa.qcat = h->at<void>(p.pf_qcat);
+  pa.cprime = h->at<void>(p.pf_cprime);
+  pa.kr = h->at<void>(p.pf_kr);
+  pa.n_heads = dm.nh; pa.head_dim = dm.dh; pa.r = dm.r; pa.dr = dm.dr; pa.dw = dm.dw;
+  pa.stride = dm.s; pa.T = T_len; pa.max_slots = dm.max_slots;
+  pa.use_gate = dm.s > 1;
+  pa.ln_eps = h->cfg.ln_eps;
+  pa.q_scale = q_scale;
+  prefill_post_kernel<T><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  if (!y) return MTLA_OK;
+
+  // Eq. 9-10 on the running-state sequence: keys and values of every column.
+  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<T>(p.pf_kv), rows,
+                       2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
+  PrefillAttnArgs aa;
+  aa.qcat = pa.qcat; aa.kv = h->at<void>(p.pf_kv); aa.kr = pa.kr; aa.out = h->at<void>(p.pf_attn);
+  aa.n_heads = dm.nh; aa.dr = dm.dr; aa.stride = dm.s; aa.T = T_len;
+  const size_t smem = prefill_attn_fma_smem_bytes(dm.dh, dm.dr);
+  dim3 grid(ceil_div(T_len, kPfTile), dm.nh, B);
+  if (dm.dh == 64) {
+    if (!h->pf_smem_ready)
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<T, 64>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    prefill_attn_fma_kernel<T, 64><<<grid, 256, smem, st>>>(aa);
+  } else {
+    if (!h->pf_smem_ready)
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<T, 128>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    prefill_attn_fma_kernel<T, 128><<<grid, 256, smem, st>>>(aa);
+  }
+  h->pf_smem_ready = true;
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd, hd, dm.d,
+                       1.f, 1, 0, 0, 0, st)));
+  return MTLA_OK;
+}
+
+int check_step_args(mtla_handle* h, const void* x, int32_t B, const void* y) {
+  if (!h || !x || !y || B <= 0) return MTLA_ERR_INVALID_ARG;
+  if (h->batch == 0) {
+    if (B > h->cfg.max_batch) return MTLA_ERR_CAPACITY;
+  } else if (B != h->batch) {
+    return MTLA_ERR_BATCH_MISMATCH;
+  }
+  if (h->tokens + 1 > h->cfg.max_tokens) return MTLA_ERR_CAPACITY;
+  return MTLA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mtla_arena_bytes(const mtla_config* cfg) {
+  mtla_config c;
+  Dims dm;
+  if (!normalise(cfg, &c, &dm)) return 0;
+  ArenaPlan p;
+  plan_arena(c, dm, &p);
+  return p.total;
+}
+
+int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size_t arena_bytes,
+                void* stream, mtla_handle** out) {
+  if (!cfg || !w || !arena || !out) return MTLA_ERR_INVALID_ARG;
+  mtla_config c;
+  Dims dm;
+  if (!normalise(cfg, &c, &dm)) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  const void* required[] = {w->w_q, w->w_qr, w->w_r, w->w_kr, w->ln_gamma, w->ln_beta,
+                            w->w_k, w->w_v, w->w_o, w->hyp_c_w, w->hyp_pe_w};
+  for (const void* ptr : required)
+    if (!ptr || !aligned16(ptr)) return MTLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(arena) & 1023) return MTLA_ERR_INVALID_ARG;
+  ArenaPlan p;
+  plan_arena(c, dm, &p);
+  if (arena_bytes < p.total) return MTLA_ERR_ARENA_TOO_SMALL;
+  mtla_handle* h = new (std::nothrow) mtla_handle();
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
+  h->tokens = 0; h->batch = 0; h->launches = 0;
+  h->attn_smem_ready = false; h->pf_smem_ready = false;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int rc = c.dtype == MTLA_DTYPE_BF16 ? create_impl<bf16>(h, w, st) : create_impl<float>(h, w, st);
+  if (rc != MTLA_OK) {
+    delete h;
+    return rc;
+  }
+  *out = h;
+  return MTLA_OK;
+}
+
+int mtla_prefill(mtla_handle* h, const void* x, int32_t B, int32_t T, void* y, void* stream) {
+  if (!h || !x || B <= 0 || T <= 0) return MTLA_ERR_INVALID_ARG;
+  if (!aligned16(x) || (y && !aligned16(y))) return MTLA_ERR_INVALID_ARG;
+  if (h->tokens != 0) return MTLA_ERR_STATE;
+  if (B > h->cfg.max_batch || T > h->cfg.max_prefill_tokens || T > h->cfg.max_tokens)
+    return MTLA_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? prefill_impl<bf16>(h, x, B, T, y, st)
+                                                 : prefill_impl<float>(h, x, B, T, y, st);
+  if (rc != MTLA_OK) return rc;
+  h->tokens = T;
+  h->batch = B;
+  return MTLA_OK;
+}
+
+int mtla_decode_step(mtla_handle* h, const void* x, int32_t B, void* y, void* stream) {
+  const int chk = check_step_args(h, x, B, y);
+  if (chk != MTLA_OK) return chk;
+  if (!aligned16(x) || !aligned16(y)) return MTLA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? decode_impl<bf16>(h, x, B, y, st)
+                                                 : decode_impl<float>(h, x, B, y, st);
+  if (rc != MTLA_OK) return rc;
+  h->tokens += 1;
+  h->batch = B;
+  return MTLA_OK;
+}
+
+int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y_host,
+                          void* stream) {
+  const int chk = check_step_args(h, x_host, B, y_host);
+  if (chk != MTLA_OK) return chk;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)B * h->dm.d * h->dm.elem;
+  void* xs = h->at<void>(h->plan.x_stage);
+  void* ys = h->at<void>(h->plan.y_stage);
+  MTLA_CUDA(cudaMemcpyAsync(xs, x_host, bytes, cudaMemcpyHostToDevice, st));
+  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? decode_impl<bf16>(h, xs, B, ys, st)
+                                                 : decode_impl<float>(h, xs, B, ys, st);
+  if (rc != MTLA_OK) return rc;
+  MTLA_CUDA(cudaMemcpyAsync(y_host, ys, bytes, cudaMemcpyDeviceToHost, st));
+  h->tokens += 1;
+  h->batch = B;
+  return MTLA_OK;
+}
+
+size_t mtla_cache_bytes(const mtla_handle* h) {
+  if (!h) return 0;
+  return (size_t)h->batch * ceil_div(h->tokens, h->dm.s) * h->dm.W * h->dm.elem;
+}
+
+int mtla_destroy(mtla_handle* h) {
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  delete h;
+  return MTLA_OK;
+}
+
+int mtla_reset(mtla_handle* h) {
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  h->tokens = 0;
+  h->batch = 0;
+  return MTLA_OK;
+}
+
+int mtla_position(const mtla_handle* h, int32_t* tokens, int32_t* slots, int32_t* batch) {
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  if (tokens) *tokens = h->tokens;
+  if (slots) *slots = ceil_div(h->tokens, h->dm.s);
+  if (batch) *batch = h->batch;
+  return MTLA_OK;
+}
+
+int mtla_cache_export(mtla_handle* h, void* dst, size_t bytes, void* stream) {
+  if (!h || !dst) return MTLA_ERR_INVALID_ARG;
+  const size_t need = mtla_cache_bytes(h);
+  if (bytes < need) return MTLA_ERR_CAPACITY;
+  if (need == 0) return MTLA_OK;
+  const size_t row = (size_t)ceil_div(h->tokens, h->dm.s) * h->dm.W * h->dm.elem;
+  const size_t pitch = (size_t)h->dm.max_slots * h->dm.W * h->dm.elem;
+  MTLA_CUDA(cudaMemcpy2DAsync(dst, row, h->at<char>(h->plan.cache), pitch, row, h->batch,
+                              cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+  return MTLA_OK;
+}
+
+int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens, void* stream) {
+  if (!h || !src || B <= 0 || tokens <= 0 || !aligned16(src)) return MTLA_ERR_INVALID_ARG;
+  if (B > h->cfg.max_batch || tokens > h->cfg.max_tokens) return MTLA_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_slots = ceil_div(tokens, h->dm.s);
+  const size_t row = (size_t)n_slots * h->dm.W * h->dm.elem;
+  const size_t pitch = (size_t)h->dm.max_slots * h->dm.W * h->dm.elem;
+  MTLA_CUDA(cudaMemcpy2DAsync(h->at<char>(h->plan.cache), pitch, src, row, row, B,
+                              cudaMemcpyDeviceToDevice, st));
+  if (tokens % h->dm.s != 0) {
+    if (h->cfg.dtype == MTLA_DTYPE_BF16)
+      open_acc_from_cache_kernel<bf16><<<B, 256, 0, st>>>(h->at<bf16>(h->plan.cache),
+                                                          h->at<float>(h->plan.open_acc), h->dm.r,
+                                                          h->dm.W, h->dm.max_slots, n_slots - 1);
+    else
+      open_acc_from_cache_kernel<float><<<B, 256, 0, st>>>(h->at<float>(h->plan.cache),
+                                                           h->at<float>(h->plan.open_acc), h->dm.r,
+                                                           h->dm.W, h->dm.max_slots, n_slots - 1);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
+  h->tokens = tokens;
+  h->batch = B;
+  return MTLA_OK;
+}
+
+int mtla_check(mtla_handle* h, void* stream) {
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  MTLA_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  int flag[4] = {0, 0, 0, 0};
+  MTLA_CUDA(cudaMemcpy(flag, h->at<char>(h->plan.err_flag), sizeof(flag), cudaMemcpyDeviceToHost));
+  return flag[0] ? MTLA_ERR_DEVICE_TIMEOUT : MTLA_OK;
+}
+
+int64_t mtla_launch_count(const mtla_handle* h) { return h ? h->launches : 0; }
+
+const char* mtla_attention_variant(const mtla_handle* h) {
+  (void)h;
+  return "fma";
+}
+
+const char* mtla_error_string(int status) {
+  switch (status) {
+    case MTLA_OK: return "ok";
+    case MTLA_ERR_INVALID_ARG: return "invalid argument";
+    case MTLA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case MTLA_ERR_ARENA_TOO_SMALL: return "arena too small";
+    case MTLA_ERR_CAPACITY: return "capacity exceeded";
+    case MTLA_ERR_BATCH_MISMATCH: return "batch mismatch";
+    case MTLA_ERR_CUDA: return "CUDA error";
+    case MTLA_ERR_STATE: return "call not valid in this state";
+    case MTLA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,304 @@
+// Prefill kernels that are not GEMMs: the per-chunk LayerNorm / gate / running-merge kernel
+// and the CUDA-core attention under the stride-aware causal mask (Section 4.2).
+#pragma once
+
+#include <math.h>
+
+#include "common.cuh"
+#include "decode_kernels.cuh"
+
+namespace mtla {
+
+struct PrefillPostArgs {
+  const float* p1;        // [B*T][proj.width] fused input projection (fp32)
+  ProjLayout proj;
+  const float* gamma;
+  const float* beta;
+  const float* hyp_c_w;   // [r][d_w]
+  const float* hyp_c_b;   // [d_w]
+  const float* gate_pe;   // [max_slots][d_w]; row j0 is Linear(pe_{j0+1})
+  const float* rope_cos;  // [max_tokens][d_R/2]
+  const float* rope_sin;
+  float* open_acc;        // [B][r]
+  void* cache;            // [max_batch][max_slots][r + d_R]
+  void* qcat;             // [B*T][n_h][d_h + d_R]: scaled query and rotated RoPE query
+  void* cprime;           // [B*T][r]: running merge state after each token (Eq. 14's sequence)
+  void* kr;               // [B*T][d_R]: rotated RoPE key of each token
+  int n_heads, head_dim, r, dr, dw, stride, T, max_slots;
+  int use_gate;
+  float ln_eps, q_scale;
+};
+
+// One CTA per (chunk, sequence): walks the chunk's <= s tokens in order so that the running
+// sum is formed exactly as the decode steps would form it, and leaves the chunk's final
+// state in the cache (the last chunk also leaves the fp32 accumulator for later decoding).
+template <typename T>
+__global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
+  __shared__ float c_s[512];
+  __shared__ float acc_s[512];
+  __shared__ float part_s[256];
+  __shared__ float red_s[33];
+  const int chunk = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int W = a.r + a.dr, DQ = a.head_dim + a.dr, half = a.dr / 2;
+  const int tok0 = chunk * a.stride, tok1 = min(a.T, tok0 + a.stride);
+  const float* gate_pe = a.gate_pe + (long long)chunk * a.dw;
+  for (int i = tid; i < a.r; i += 256) acc_s[i] = 0.f;
+
+  for (int tok = tok0; tok < tok1; ++tok) {
+    const long long rowi = (long long)b * a.T + tok;
+    const float* row = a.p1 + rowi * a.proj.width;
+    __syncthreads();
+    float s = 0.f;
+    for (int i = tid; i < a.r; i += 256) {
+      const float v = row[a.proj.off_c + i];
+      c_s[i] = v;
+      s += v;
+    }
+    const float mean = block_sum(s, red_s) / a.r;
+    float sq = 0.f;
+    for (int i = tid; i < a.r; i += 256) {
+      const float dlt = c_s[i] - mean;
+      sq += dlt * dlt;
+    }
+    __syncthreads();
+    const float rstd = rsqrtf(block_sum(sq, red_s) / a.r + a.ln_eps);
+    for (int i = tid; i < a.r; i += 256)
+      c_s[i] = (c_s[i] - mean) * rstd * a.gamma[i] + a.beta[i];
+    __syncthreads();
+
+    float w = 1.f;
+    if (a.use_gate) {
+      const int parts = 256 / a.dw > 0 ? 256 / a.dw : 1;
+      float h = 0.f;
+      if (tid < parts * a.dw) {
+        const int n = tid % a.dw, part = tid / a.dw;
+        const int per = ceil_div(a.r, parts);
+        const int lo = part * per, hi = min(a.r, lo + per);
+        for (int i = lo; i < hi; ++i) h = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], h);
+      }
+      part_s[tid] = h;
+      __syncthreads();
+      float prod = 0.f;
+      if (tid < a.dw) {
+        float hn = a.hyp_c_b[tid];
+        for (int p = 0; p < parts; ++p) hn += part_s[p * a.dw + tid];
+        prod = hn * gate_pe[tid];
+      }
+      const float logit = block_sum(prod, red_s);
+      w = 1.f / (1.f + expf(-logit));
+    }
+
+    T* cp = static_cast<T*>(a.cprime) + rowi * a.r;
+    for (int i = tid; i < a.r; i += 256) {
+      const float v = acc_s[i] + w * c_s[i];
+      acc_s[i] = v;
+      cp[i] = Elem<T>::from_float(v);
+    }
+    const float* cs_row = a.rope_cos + (long long)tok * half;
+    const float* sn_row = a.rope_sin + (long long)tok * half;
+    T* kr = static_cast<T*>(a.kr) + rowi * a.dr;
+    for (int k = tid; k < half; k += 256) {
+      const float x0 = row[a.proj.off_kr + 2 * k], x1 = row[a.proj.off_kr + 2 * k + 1];
+      kr[2 * k] = Elem<T>::from_float(x0 * cs_row[k] - x1 * sn_row[k]);
+      kr[2 * k + 1] = Elem<T>::from_float(x0 * sn_row[k] + x1 * cs_row[k]);
+    }
+    T* qc = static_cast<T*>(a.qcat) + rowi * a.n_heads * DQ;
+    for (int i = tid; i < a.n_heads * a.head_dim; i += 256) {
+      const int h = i / a.head_dim, e = i % a.head_dim;
+      qc[h * DQ + e] = Elem<T>::from_float(row[a.proj.off_q + i] * a.q_scale);
+    }
+    for (int i = tid; i < a.n_heads * half; i += 256) {
+      const int h = i / half, k = i % half;
+      const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k];
+      const float x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
+      qc[h * DQ + a.head_dim + 2 * k] =
+          Elem<T>::from_float((x0 * cs_row[k] - x1 * sn_row[k]) * a.q_scale);
+      qc[h * DQ + a.head_dim + 2 * k + 1] =
+          Elem<T>::from_float((x0 * sn_row[k] + x1 * cs_row[k]) * a.q_scale);
+    }
+  }
+  __syncthreads();
+
+  // The chunk's state after its last available token is what the cache holds.
+  const long long last = (long long)b * a.T + (tok1 - 1);
+  T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + chunk) * W;
+  const T* kr = static_cast<const T*>(a.kr) + last * a.dr;
+  for (int i = tid; i < a.r; i += 256) slot_row[i] = Elem<T>::from_float(acc_s[i]);
+  for (int i = tid; i < a.dr; i += 256) slot_row[a.r + i] = kr[i];
+  if (tok1 == a.T)
+    for (int i = tid; i < a.r; i += 256) a.open_acc[(long long)b * a.r + i] = acc_s[i];
+}
+
+struct PrefillAttnArgs {
+  const void* qcat;   // [B*T][n_h][d_h + d_R], pre-scaled by log2(e)/sqrt(d_h)
+  const void* kv;     // [B*T][2*n_h*d_h]: keys then values up-projected from cprime (Eq. 9-10)
+  const void* kr;     // [B*T][d_R]
+  void* out;          // [B*T][n_h*d_h] per-head attention outputs (input of W_O)
+  int n_heads, dr, stride, T;
+};
+
+constexpr int kPfTile = 64;
+
+inline size_t prefill_attn_fma_smem_bytes(int dh, int dr) {
+  const int DQ = dh + dr;
+  return sizeof(float) * ((size_t)2 * DQ * kPfTile + (size_t)kPfTile * dh +
+                          (size_t)kPfTile * (kPfTile + 1));
+}
+
+// CUDA-core flash-style attention for the prefill.  Row m (0-based token) sees the closed
+// slots j < floor(m/s), each represented by the state and RoPE key of its last token
+// j*s + s - 1, plus its own running state at column m: exactly the columns the
+// stride-aware mask of Section 4.2 admits.  The mask is a predicate on (m, j).
+// Grid (ceil(T/64), n_h, B), 256 threads as 16 x 16, each owning a 4 x 4 score patch.
+template <typename T, int DH>
+__global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a) {
+  extern __shared__ float smem[];
+  constexpr int BT = kPfTile, V = Elem<T>::kVec, OC = DH / 16;
+  const int DQ = DH + a.dr;
+  float* qs = smem;                 // [DQ][BT]  (transposed: k-major)
+  float* ks = qs + DQ * BT;         // [DQ][BT]
+  float* vs = ks + DQ * BT;         // [BT][DH]
+  float* ps = vs + BT * DH;         // [BT][BT+1]
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int q0 = blockIdx.x * BT, h = blockIdx.y, b = blockIdx.z;
+  const T* qcat = static_cast<const T*>(a.qcat);
+  const T* kv = static_cast<const T*>(a.kv);
+  const T* kr = static_cast<const T*>(a.kr);
+  const long long base = (long long)b * a.T;
+  const int kvw = 2 * a.n_heads * DH;
+
+  for (int v = tid; v < BT * (DQ / V); v += 256) {
+    const int row = v / (DQ / V), kk = (v % (DQ / V)) * V;
+    float tmp[V];
+    if (q0 + row < a.T) {
+      load_vec(qcat + ((base + q0 + row) * a.n_heads + h) * DQ + kk, tmp);
+    } else {
+#pragma unroll
+      for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < V; ++e) qs[(kk + e) * BT + row] = tmp[e];
+  }
+
+  float m_run[4], l_run[4], o[4][OC];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    m_run[i] = -INFINITY;
+    l_run[i] = 0.f;
+#pragma unroll
+    for (int c = 0; c < OC; ++c) o[i][c] = 0.f;
+  }
+
+  const int last_row = min(a.T, q0 + BT) - 1;
+  const int n_closed = last_row / a.stride;         // closed slots visible to the last row
+  const int n_tiles = ceil_div(n_closed, BT);
+  // Tiles 0..n_tiles-1 walk the closed slots; tile n_tiles is the diagonal (own state).
+  for (int t = 0; t <= n_tiles; ++t) {
+    const bool diag = (t == n_tiles);
+    __syncthreads();
+    for (int v = tid; v < BT * (DQ / V); v += 256) {
+      const int col = v / (DQ / V), kk = (v % (DQ / V)) * V;
+      const int j = t * BT + col;
+      const long long tok = diag ? (long long)(q0 + col) : (long long)j * a.stride + a.stride - 1;
+      const bool ok = diag ? (q0 + col < a.T) : (j < n_closed);
+      float tmp[V];
+      if (ok) {
+        if (kk < DH) load_vec(kv + (base + tok) * kvw + h * DH + kk, tmp);
+        else load_vec(kr + (base + tok) * a.dr + (kk - DH), tmp);
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) ks[(kk + e) * BT + col] = tmp[e];
+    }
+    for (int v = tid; v < BT * (DH / V); v += 256) {
+      const int col = v / (DH / V), kk = (v % (DH / V)) * V;
+      const int j = t * BT + col;
+      const long long tok = diag ? (long long)(q0 + col) : (long long)j * a.stride + a.stride - 1;
+      const bool ok = diag ? (q0 + col < a.T) : (j < n_closed);
+      float tmp[V];
+      if (ok) {
+        load_vec(kv + (base + tok) * kvw + a.n_heads * DH + h * DH + kk, tmp);
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) vs[col * DH + kk + e] = tmp[e];
+    }
+    __syncthreads();
+
+    float sc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sc[i][j] = 0.f;
+    for (int k = 0; k < DQ; ++k) {
+      const float4 q4 = *reinterpret_cast<const float4*>(qs + k * BT + ty * 4);
+      const float4 k4 = *reinterpret_cast<const float4*>(ks + k * BT + tx * 4);
+      const float qv[4] = {q4.x, q4.y, q4.z, q4.w}, kv4[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sc[i][j] = fmaf(qv[i], kv4[j], sc[i][j]);
+    }
+    // Stride-aware mask as a predicate, then the online softmax update per row.
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = q0 + ty * 4 + i;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int col = tx * 4 + j;
+        const bool allowed = diag ? (col == ty * 4 + i && row < a.T)
+                                  : (t * BT + col < row / a.stride);
+        sc[i][j] = allowed ? sc[i][j] : -INFINITY;
+        mx = fmaxf(mx, sc[i][j]);
+      }
+#pragma unroll
+      for (int off = 8; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      const float m_new = fmaxf(m_run[i], mx);
+      const float fac = (m_new == -INFINITY) ? 1.f : exp2f(m_run[i] - m_new);
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float p = (m_new == -INFINITY) ? 0.f : exp2f(sc[i][j] - m_new);
+        ps[(ty * 4 + i) * (BT + 1) + tx * 4 + j] = p;
+        sum += p;
+      }
+#pragma unroll
+      for (int off = 8; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+      l_run[i] = l_run[i] * fac + sum;
+      m_run[i] = m_new;
+#pragma unroll
+      for (int c = 0; c < OC; ++c) o[i][c] *= fac;
+    }
+    __syncthreads();
+    for (int k = 0; k < BT; ++k) {
+      float vv[OC];
+#pragma unroll
+      for (int c = 0; c < OC; ++c) vv[c] = vs[k * DH + tx * OC + c];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float p = ps[(ty * 4 + i) * (BT + 1) + k];
+#pragma unroll
+        for (int c = 0; c < OC; ++c) o[i][c] = fmaf(p, vv[c], o[i][c]);
+      }
+    }
+  }
+
+  T* out = static_cast<T*>(a.out);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = q0 + ty * 4 + i;
+    if (row >= a.T) continue;
+    const float inv = 1.f / l_run[i];
+#pragma unroll
+    for (int c = 0; c < OC; ++c)
+      out[(base + row) * a.n_heads * DH + h * DH + tx * OC + c] =
+          Elem<T>::from_float(o[i][c] * inv);
+  }
+}
+
+}  // namespace mtla

@@ -1,0 +1,78 @@
+// One-time kernels run by mtla_create: weight repacking and the positional tables.
+#pragma once
+
+#include <math.h>
+
+#include "common.cuh"
+
+namespace mtla {
+
+// dst[n][k] = src[k][n] for a row-major src [K][N] (leading dimension ld_src); dst has
+// leading dimension ld_dst.  Grid (ceil(N/32), ceil(K/32)), block (32, 8).
+template <typename T>
+__global__ void transpose_kernel(const T* src, T* dst, int K, int N, int ld_src, int ld_dst) {
+  __shared__ T tile[32][33];
+  const int n0 = blockIdx.x * 32, k0 = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int k = k0 + i, n = n0 + threadIdx.x;
+    if (k < K && n < N) tile[i][threadIdx.x] = src[(long long)k * ld_src + n];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int n = n0 + i, k = k0 + threadIdx.x;
+    if (k < K && n < N) dst[(long long)n * ld_dst + k] = tile[threadIdx.x][i];
+  }
+}
+
+// dst (fp32) = src (T); src == nullptr fills zeros.
+template <typename T>
+__global__ void widen_kernel(const T* src, float* dst, long long n) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src ? Elem<T>::to_float(src[i]) : 0.f;
+}
+
+// Row j0 of the table is Linear(pe_j) of Eq. 13 for the 1-based slot number j = j0 + 1:
+// pe_j is the sinusoidal embedding of dimension r (sin at even, cos at odd indices,
+// wavelengths 10000^(2k/r)), evaluated in fp64.  One CTA per slot number.
+__global__ void __launch_bounds__(256) gate_pe_table_kernel(const float* w /*[r][d_w]*/,
+                                                            const float* bias /*[d_w]*/,
+                                                            float* table /*[slots][d_w]*/,
+                                                            int r, int dw) {
+  __shared__ double pe[512];
+  const int j = blockIdx.x + 1;
+  for (int k = threadIdx.x; k < r / 2; k += blockDim.x) {
+    const double angle = (double)j / pow(10000.0, 2.0 * k / r);
+    pe[2 * k] = sin(angle);
+    pe[2 * k + 1] = cos(angle);
+  }
+  __syncthreads();
+  for (int n = threadIdx.x; n < dw; n += blockDim.x) {
+    double acc = bias[n];
+    for (int i = 0; i < r; ++i) acc += pe[i] * (double)w[(long long)i * dw + n];
+    table[(long long)blockIdx.x * dw + n] = (float)acc;
+  }
+}
+
+// cos/sin of pos * theta^(-2k/d_R) for every position and pair index (Section 4.3), fp64
+// evaluation rounded to fp32.
+__global__ void rope_table_kernel(float* cos_t, float* sin_t, int positions, int half,
+                                  double theta) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)positions * half) return;
+  const int pos = (int)(i / half), k = (int)(i % half);
+  const double angle = (double)pos * pow(theta, -2.0 * k / (2.0 * half));
+  cos_t[i] = (float)cos(angle);
+  sin_t[i] = (float)sin(angle);
+}
+
+// Initialises the fp32 accumulator of the open slot from a stored cache row.
+template <typename T>
+__global__ void open_acc_from_cache_kernel(const T* cache, float* open_acc, int r, int W,
+                                           int max_slots, int slot) {
+  const int b = blockIdx.x;
+  const T* row = cache + ((long long)b * max_slots + slot) * W;
+  for (int i = threadIdx.x; i < r; i += blockDim.x)
+    open_acc[(long long)b * r + i] = Elem<T>::to_float(row[i]);
+}
+
+}  // namespace mtla

@@ -1,0 +1,63 @@
+"""Shared test plumbing: build an oracle Params and a GPU handle from the same seeded tensors."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import mtla_oracle as O
+from paper_2505_13544_b200 import synth
+
+# Tolerances of the benchmark specification: fp32 max-abs 1e-4; bf16 max-abs 2e-2 and
+# relative L2 1e-2.  Slot counts and cache lengths must match exactly.
+FP32_MAX_ABS = 1e-4
+BF16_MAX_ABS = 2e-2
+BF16_REL_L2 = 1e-2
+
+
+def dims_of(w: synth.Workload) -> dict:
+    return dict(d_model=w.d_model, n_heads=w.n_heads, head_dim=w.head_dim,
+                latent_rank=w.latent_rank, rope_dim=w.rope_dim, hyper_dim=w.hyper_dim,
+                stride=w.stride)
+
+
+def oracle_params(w: synth.Workload, weights: dict) -> O.Params:
+    return O.params_from_tensors(dims_of(w), {k: v.double().numpy() for k, v in weights.items()},
+                                 ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+
+
+def gpu_handle(w: synth.Workload, weights: dict, max_batch=None, max_tokens=None,
+               max_prefill_tokens=None, device="cuda:0"):
+    from paper_2505_13544_b200 import binding as M
+    cfg = M.make_config(**dims_of(w), max_batch=max_batch or w.batch,
+                        max_tokens=max_tokens or w.max_tokens,
+                        max_prefill_tokens=(w.prefill_tokens if max_prefill_tokens is None
+                                            else max_prefill_tokens),
+                        dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    dev_weights = {k: v.to(device) for k, v in weights.items()}
+    return M.mtla_create(cfg, dev_weights, device=device)
+
+
+def assert_close(got: torch.Tensor, want: np.ndarray, dtype: str, what: str = "y") -> None:
+    """Applies the specification's tolerance for the storage type."""
+    g = got.detach().double().cpu().numpy()
+    want = np.asarray(want, dtype=np.float64)
+    assert g.shape == want.shape, (what, g.shape, want.shape)
+    assert np.isfinite(g).all(), f"{what}: non-finite values"
+    err = np.abs(g - want).max() if g.size else 0.0
+    if dtype == "fp32":
+        assert err <= FP32_MAX_ABS, f"{what}: max abs err {err:.3e} > {FP32_MAX_ABS}"
+    else:
+        rel = np.linalg.norm(g - want) / max(np.linalg.norm(want), 1e-30)
+        assert err <= BF16_MAX_ABS, f"{what}: max abs err {err:.3e} > {BF16_MAX_ABS}"
+        assert rel <= BF16_REL_L2, f"{what}: rel L2 err {rel:.3e} > {BF16_REL_L2}"
+
+
+def assert_cache_close(got: torch.Tensor, want: np.ndarray, dtype: str) -> None:
+    """Cache contents: fp32 to 1e-4; bf16 to a few storage ulps (2^-7 relative, 2^-7 absolute)."""
+    g = got.detach().double().cpu().numpy()
+    want = np.asarray(want, dtype=np.float64)
+    assert g.shape == want.shape, (g.shape, want.shape)
+    if dtype == "fp32":
+        assert np.abs(g - want).max() <= FP32_MAX_ABS
+    else:
+        assert (np.abs(g - want) <= 2.0 ** -7 * (1.0 + np.abs(want))).all()
