@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the MTLA decode step (and, as extras, the prefill) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one full decode step (input projections, LayerNorm + gate + slot update,
+query absorption, attention over the compressed cache, output projections) for the whole
+batch; the metric is decode tokens/s = B * K / time.  With N > 1 every rank runs an
+independent replica of the workload on its own GPU (sequences never interact, so there is
+no collective on the data path) and the value is the sum over ranks divided by the
+slowest rank's device time.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2505_13544_b200 import synth  # noqa: E402
+
+METRIC = "mtla_decode_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0          # the "~8 TB/s" the benchmark specification quotes
+
+
+def measured_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+def algorithmic_work(w: synth.Workload, n_slots: float) -> dict:
+    """Bytes and FLOP one decode step must move/compute (weights once, cache once)."""
+    e = 2 if w.dtype == "bf16" else 4
+    d, nh, dh, r, dr, dw = (w.d_model, w.n_heads, w.head_dim, w.latent_rank, w.rope_dim,
+                            w.hyper_dim)
+    params = (d * nh * dh + d * nh * dr + d * r + d * dr + 2 * r + 2 * r * nh * dh
+              + nh * dh * d + 2 * (r * dw + dw))
+    cache = w.batch * n_slots * (r + dr) * e
+    return {"weight_bytes": params * e, "cache_bytes": cache,
+            "attn_flop": w.batch * nh * n_slots * (2 * (r + dr) + 2 * r),
+            "proj_flop": 2 * w.batch * params}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nvml = None
+
+    def _run(self):
+        n = self._nvml
+        names = {
+            "sw_power_cap": getattr(n, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_slowdown": getattr(n, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "sw_thermal_slowdown": getattr(n, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "hw_thermal_slowdown": getattr(n, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "hw_power_brake": getattr(n, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_SM))
+                try:
+                    mask = n.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    mask = n.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for name, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self._nvml is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self) -> dict:
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
+                "reasons": sorted(self.reasons)}
+
+
+def dims_of(w: synth.Workload) -> dict:
+    return dict(d_model=w.d_model, n_heads=w.n_heads, head_dim=w.head_dim,
+                latent_rank=w.latent_rank, rope_dim=w.rope_dim, hyper_dim=w.hyper_dim,
+                stride=w.stride)
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_decode_sample(w: synth.Workload, n_seq: int, budget_s: float, max_steps: int,
+                         exact_steps: int | None = None) -> dict:
+    """Times the CPU oracle's decode step, as it stands, on a bounded sample: n_seq sequences
+    at the workload's full context, as many steps as fit the budget.  State building (the
+    prompt or the imported cache) is outside the timed region, like the GPU's."""
+    from oracle import mtla_oracle as O
+    from threadpoolctl import threadpool_info
+
+    weights = synth.make_weights(w)
+    p = O.params_from_tensors(dims_of(w), {k: v.double().numpy() for k, v in weights.items()},
+                              ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    states = []
+    for b in range(n_seq):
+        if w.context_tokens:
+            cache = synth.context_cache_row(w, b).double().numpy()
+            states.append(O.state_from_cache(cache, w.context_tokens, p))
+        else:
+            prompt = synth.normal(w.seed, f"prompt/{b}", (w.prefill_tokens, w.d_model))
+            prompt = synth.stored(prompt, w.dtype).double().numpy()
+            _, st = O.decode_sequence(p, prompt, rows=[])
+            states.append(st)
+    steps, t0 = 0, time.perf_counter()
+    limit = exact_steps if exact_steps is not None else max_steps
+    while steps < limit:
+        x = synth.decode_input(w, steps, batch=n_seq).double().numpy()
+        for b in range(n_seq):
+            O.decode_step(p, states[b], x[b])
+        steps += 1
+        if exact_steps is None and time.perf_counter() - t0 >= budget_s:
+            break
+    elapsed = time.perf_counter() - t0
+    cores = max([int(i.get("num_threads", 1)) for i in threadpool_info()] + [1])
+    return {"value": n_seq * steps / elapsed, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n_seq} of {w.batch} sequences x {steps} decode steps at full context "
+                      f"({states[0].n_slots} slots), {elapsed:.1f} s",
+            "seconds": elapsed, "steps": steps}
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.WORKLOADS[args.workload]
+    n_seq = 1 if w.batch * w.latent_rank >= 8192 else min(w.batch, 4)
+    # warm-up steps are run and discarded, then exactly --steps sample steps are timed
+    oracle_decode_sample(w, n_seq, 0.0, 0, exact_steps=min(args.warmup, 1))
+    res = oracle_decode_sample(w, n_seq, 0.0, 0, exact_steps=args.steps)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": res["seconds"] / max(res["steps"], 1) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": n_seq, "of_batch": w.batch,
+                   "note": "CPU oracle on host cores; each step is one decode step of a bounded "
+                           "sample of sequences at full context"},
+        "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU arm
+
+def build_layer(w: synth.Workload, extra_steps: int, device):
+    from paper_2505_13544_b200 import binding as M
+    weights = synth.make_weights(w)
+    cfg = M.make_config(**dims_of(w), max_batch=w.batch,
+                        max_tokens=w.prefill_tokens + w.context_tokens + extra_steps,
+                        max_prefill_tokens=w.prefill_tokens, dtype=w.dtype, ln_eps=w.ln_eps,
+                        rope_theta=w.rope_theta)
+    h = M.mtla_create(cfg, {k: v.to(device) for k, v in weights.items()}, device=device)
+    return M, h
+
+
+def fill_context(M, h, w: synth.Workload, device) -> dict:
+    """Brings the cache to the workload's context: a timed parallel prefill, or an import."""
+    info = {}
+    if w.prefill_tokens:
+        x = torch.empty(w.batch, w.prefill_tokens, w.d_model, dtype=synth.torch_dtype(w.dtype),
+                        device=device)
+        for b in range(w.batch):
+            x[b].copy_(synth.stored(synth.normal(w.seed, f"prompt/{b}",
+                                                 (w.prefill_tokens, w.d_model)), w.dtype))
+        y = torch.empty_like(x)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(device)
+        ev0.record()
+        M.mtla_prefill(h, x, y)
+        ev1.record()
+        torch.cuda.synchronize(device)
+        ms = ev0.elapsed_time(ev1)
+        info = {"prefill_tokens_per_s": w.batch * w.prefill_tokens / (ms * 1e-3),
+                "prefill_ms": ms, "prefill_tokens": w.prefill_tokens, "timed_runs": 1}
+        del x, y
+    elif w.context_tokens:
+        n_slots = -(-w.context_tokens // w.stride)
+        cache = torch.empty(w.batch, n_slots, w.slot_width, dtype=synth.torch_dtype(w.dtype),
+                            device=device)
+        for b in range(w.batch):
+            cache[b].copy_(synth.context_cache_row(w, b))
+        M.mtla_cache_import(h, cache, w.context_tokens)
+        torch.cuda.synchronize(device)
+        del cache
+    torch.cuda.empty_cache()
+    return info
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--workload", default="large", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch.distributed as dist
+    from paper_2505_13544_b200 import replicas
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier(device_ids=[local])
+        torch.cuda.synchronize(device)
+
+    w = synth.WORKLOADS[args.workload]
+    K, W = args.steps, max(args.warmup, 3)
+    M, h = build_layer(w, extra_steps=2 * (K + W), device=device)
+    extras = fill_context(M, h, w, device)
+    dt = synth.torch_dtype(w.dtype)
+    xs = [synth.decode_input(w, i).to(device) for i in range(8)]
+    y = torch.empty(w.batch, w.d_model, dtype=dt, device=device)
+
+    # ---- device-resident timing: K decode steps, inputs already in HBM
+    for i in range(W):
+        M.mtla_decode_step(h, xs[i % 8], y)
+    slots_begin = M.mtla_position(h)[1]
+    launches0 = M.mtla_launch_count(h)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    M.mtla_profile_begin(h, K)
+    with ClockSampler(local) as clocks:
+        barrier()
+        ev0.record()
+        for i in range(K):
+            M.mtla_decode_step(h, xs[i % 8], y)
+        ev1.record()
+        barrier()
+    local_ms = ev0.elapsed_time(ev1)
+    attn_ms, attn_steps = M.mtla_profile_end(h)
+    launches = M.mtla_launch_count(h) - launches0
+    slots_end = M.mtla_position(h)[1]
+    M.mtla_check(h)
+    value, ms = replicas.throughput(w.batch * K, local_ms, device)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    xh = [synth.decode_input(w, i).pin_memory() for i in range(8)]
+    yh = torch.empty(w.batch, w.d_model, dtype=dt).pin_memory()
+    for i in range(W):
+        M.mtla_decode_step_host(h, xh[i % 8], yh)
+    barrier()
+    ev0.record()
+    for i in range(K):
+        M.mtla_decode_step_host(h, xh[i % 8], yh)
+    ev1.record()
+    barrier()
+    e2e_value, _ = replicas.throughput(w.batch * K, ev0.elapsed_time(ev1), device)
+    assert torch.isfinite(yh.float()).all()
+    M.mtla_check(h)
+
+    if rank != 0:
+        M.mtla_destroy(h)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    n_slots = 0.5 * (slots_begin + 1 + slots_end)
+    work = algorithmic_work(w, n_slots)
+    attn_launch_s = attn_ms * 1e-3 / max(attn_steps, 1)
+    achieved_gbs = work["cache_bytes"] / attn_launch_s / 1e9
+    step_s = local_ms * 1e-3 / K
+    hbm_time = (work["weight_bytes"] + work["cache_bytes"]) / (peaks["hbm_gbs"] * 1e9)
+    tensor_time = (work["attn_flop"] + work["proj_flop"]) / (peaks["bf16_tflops_sustained"] * 1e12)
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        t = json.load(open(tpath)).get(M.mtla_attention_variant(h), {})
+        if t.get("dram_bytes_per_cache_byte") is not None:
+            traffic = t["dram_bytes_per_cache_byte"] * work["cache_bytes"]
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "d_model": w.d_model,
+                   "n_heads": w.n_heads, "head_dim": w.head_dim, "latent_rank": w.latent_rank,
+                   "rope_dim": w.rope_dim, "stride": w.stride,
+                   "context_slots": [slots_begin, slots_end],
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2: every step streams the whole cache "
+                         f"({work['cache_bytes'] / 1e6:.0f} MB) and the weights"
+                         if work["cache_bytes"] > 126e6 else
+                         "cache smaller than L2: bandwidth figures are effective, not DRAM",
+                   "attention_variant": M.mtla_attention_variant(h)},
+        "roofline": {"bound": "hbm", "kernel": "decode attention (a7)",
+                     "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved_gbs / peaks["hbm_gbs"],
+                     "peak_source": f"of {peaks['source']}",
+                     "frac_of_nominal_8TBs": achieved_gbs / NOMINAL_HBM_GBS,
+                     "launch_ms": attn_launch_s * 1e3, "traffic": traffic},
+        "step_roofline": {"hbm_time_ms": hbm_time * 1e3, "tensor_time_ms": tensor_time * 1e3,
+                          "frac": max(hbm_time, tensor_time) / step_s,
+                          "frac_of_nominal_8TBs": max(
+                              (work["weight_bytes"] + work["cache_bytes"]) / (NOMINAL_HBM_GBS * 1e9),
+                              tensor_time) / step_s},
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": w.batch * w.d_model * (2 if w.dtype == "bf16" else 4),
+                "d2h_bytes_per_step": w.batch * w.d_model * (2 if w.dtype == "bf16" else 4)},
+        "gpu_launches": int(launches),
+        "clocks": clocks.summary(),
+    }
+    if extras:
+        line["prefill"] = extras
+    M.mtla_destroy(h)
+    del h
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_cpu_baseline:
+        n_seq = 1 if w.batch * w.latent_rank >= 8192 else min(w.batch, 4)
+        res = oracle_decode_sample(w, n_seq, budget_s=12.0, max_steps=64)
+        line["cpu_baseline"] = {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

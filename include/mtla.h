@@ -144,6 +144,14 @@ int mtla_check(mtla_handle* h, void* stream);
 /* Number of kernels the library has launched on behalf of this handle since creation. */
 int64_t mtla_launch_count(const mtla_handle* h);
 
+/* Kernel timing for benchmarks.  After mtla_profile_begin, each of the next max_steps
+ * decode steps records a CUDA event pair on its stream around the decode-attention kernel
+ * (step a7, the kernel that streams the cache).  mtla_profile_end waits for those events,
+ * returns their summed duration in milliseconds and the number of steps covered, and
+ * releases the events. */
+int mtla_profile_begin(mtla_handle* h, int32_t max_steps);
+int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps);
+
 /* Name of the decode-attention kernel variant the handle dispatches to ("fma" or "tcgen05"). */
 const char* mtla_attention_variant(const mtla_handle* h);
 

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "mtla_arena_bytes", "mtla_create", "mtla_prefill", "mtla_decode_step",
     "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
     "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
-    "mtla_attention_variant", "mtla_error_string")
+    "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end")
 
 
 class MTLAError(RuntimeError):
@@ -74,6 +74,9 @@ def load_library() -> ctypes.CDLL:
         "mtla_check": (ctypes.c_int, [vp, vp]),
         "mtla_launch_count": (ctypes.c_int64, [vp]),
         "mtla_attention_variant": (ctypes.c_char_p, [vp]),
+        "mtla_profile_begin": (ctypes.c_int, [vp, i32]),
+        "mtla_profile_end": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
+                                            ctypes.POINTER(i32)]),
         "mtla_error_string": (ctypes.c_char_p, [ctypes.c_int]),
     }
     for name, (res, args) in sigs.items():
@@ -247,3 +250,15 @@ def mtla_launch_count(h: Handle) -> int:
 
 def mtla_attention_variant(h: Handle) -> str:
     return load_library().mtla_attention_variant(h.ptr).decode()
+
+
+def mtla_profile_begin(h: Handle, max_steps: int) -> None:
+    _check(load_library().mtla_profile_begin(h.ptr, max_steps), "mtla_profile_begin")
+
+
+def mtla_profile_end(h: Handle) -> tuple[float, int]:
+    """(summed decode-attention kernel time in ms, steps covered)."""
+    ms, steps = ctypes.c_double(), ctypes.c_int32()
+    _check(load_library().mtla_profile_end(h.ptr, ctypes.byref(ms), ctypes.byref(steps)),
+           "mtla_profile_end")
+    return ms.value, steps.value

@@ -26,7 +26,6 @@ struct PostArgs {
   const float* rope_sin;  // [d_R/2]
   float* open_acc;        // [B][r] fp32 running sum of the open slot
   void* cache;            // [max_batch][max_slots][r + d_R]
-  void* q_t;              // [B][n_h*d_h] query in storage type (input of the absorption GEMM)
   void* qt;               // [B][n_h][r + d_R] absorbed query; this kernel writes the RoPE tail
   int n_heads, head_dim, r, dr, dw;
   int max_slots, slot;    // slot = 0-based slot index receiving this token
@@ -39,7 +38,8 @@ struct PostArgs {
 // One CTA of 256 threads per sequence.  Section 4.1: c_i = LayerNorm(x_i W_r); Eq. 13 gate;
 // slot update (open: c_hat_j = w c, else c_hat_j += w c); Section 4.3: RoPE key replaces
 // the slot's key, RoPE queries are rotated and written behind the absorbed query.
-template <typename T>
+// T is the cache element type, TQ the element type of the absorbed-query buffer.
+template <typename T, typename TQ>
 __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   __shared__ float c_s[512];
   __shared__ float part_s[256];
@@ -104,19 +104,16 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
     slot_row[a.r + 2 * k] = Elem<T>::from_float(x0 * cs - x1 * sn);
     slot_row[a.r + 2 * k + 1] = Elem<T>::from_float(x0 * sn + x1 * cs);
   }
-  // Query in storage type for the absorption GEMM; rotated, pre-scaled RoPE queries.
-  T* q_t = static_cast<T*>(a.q_t) + (long long)b * a.n_heads * a.head_dim;
-  for (int i = tid; i < a.n_heads * a.head_dim; i += 256)
-    q_t[i] = Elem<T>::from_float(row[a.proj.off_q + i]);
-  T* qt = static_cast<T*>(a.qt) + (long long)b * a.n_heads * W;
+  // Rotated, pre-scaled RoPE queries behind the (separately computed) absorbed query.
+  TQ* qt = static_cast<TQ*>(a.qt) + (long long)b * a.n_heads * W;
   const int half = a.dr / 2;
   for (int i = tid; i < a.n_heads * half; i += 256) {
     const int h = i / half, k = i % half;
     const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k];
     const float x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
     const float cs = a.rope_cos[k], sn = a.rope_sin[k];
-    qt[h * W + a.r + 2 * k] = Elem<T>::from_float((x0 * cs - x1 * sn) * a.q_scale);
-    qt[h * W + a.r + 2 * k + 1] = Elem<T>::from_float((x0 * sn + x1 * cs) * a.q_scale);
+    qt[h * W + a.r + 2 * k] = Elem<TQ>::from_float((x0 * cs - x1 * sn) * a.q_scale);
+    qt[h * W + a.r + 2 * k + 1] = Elem<TQ>::from_float((x0 * sn + x1 * cs) * a.q_scale);
   }
 }
 
@@ -138,12 +135,13 @@ inline size_t attn_fma_smem_bytes(int nh_padded, int r, int dr) {
 
 // CUDA-core split-K decode attention in the absorbed form (Eq. 12 / Eq. 17): one CTA per
 // (split, sequence) streams its slot range once; every head reuses the staged tile.
-// NH = head count padded to the template instance, RPT = latent columns per thread.
-template <typename T, int NH, int RPT>
+// T = cache element type, TQ = absorbed-query element type, NH = head count padded to the
+// template instance, RPT = latent columns per thread.
+template <typename T, typename TQ, int NH, int RPT>
 __global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
   extern __shared__ float smem[];
   constexpr int TS = kAttnFmaTile;
-  constexpr int V = Elem<T>::kVec;
+  constexpr int V = Elem<T>::kVec, VQ = Elem<TQ>::kVec;
   const int W = a.r + a.dr, WS = W + 1;
   float* qs = smem;
   float* tile = qs + NH * W;
@@ -153,20 +151,20 @@ __global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
   const int tid = threadIdx.x, b = blockIdx.y, split = blockIdx.x;
   const int slot0 = split * a.slots_per_split;
   const int slot1 = min(a.n_slots, slot0 + a.slots_per_split);
-  const T* qt = static_cast<const T*>(a.qt) + (long long)b * a.n_heads * W;
+  const TQ* qt = static_cast<const TQ*>(a.qt) + (long long)b * a.n_heads * W;
   const T* cache = static_cast<const T*>(a.cache) + (long long)b * a.max_slots * W;
 
-  for (int v = tid; v < NH * (W / V); v += 256) {
-    const int h = v / (W / V), kv = (v % (W / V)) * V;
-    float tmp[V];
+  for (int v = tid; v < NH * (W / VQ); v += 256) {
+    const int h = v / (W / VQ), kv = (v % (W / VQ)) * VQ;
+    float tmp[VQ];
     if (h < a.n_heads) {
       load_vec(qt + h * W + kv, tmp);
     } else {
 #pragma unroll
-      for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+      for (int e = 0; e < VQ; ++e) tmp[e] = 0.f;
     }
 #pragma unroll
-    for (int e = 0; e < V; ++e) qs[h * W + kv + e] = tmp[e];
+    for (int e = 0; e < VQ; ++e) qs[h * W + kv + e] = tmp[e];
   }
   if (tid < NH) m_s[tid] = -INFINITY;
   float acc[NH][RPT];

@@ -21,15 +21,15 @@ struct GemmArgs {
 
 // Tile: BM x 64 outputs per CTA of 256 threads, BK = 32.  Thread (ty, tx) of a 16 x 16
 // grid owns rows ty + 16*i (i < BM/16) and columns tx*4 .. tx*4+3.
-template <typename TIn, typename TOut, int BM>
+template <typename TA, typename TB, typename TOut, int BM>
 __global__ void __launch_bounds__(256) gemm_nt_fma_kernel(GemmArgs g) {
   constexpr int BN = 64, BK = 32, TM = BM / 16, TN = 4;
-  constexpr int V = Elem<TIn>::kVec;
+  constexpr int VA = Elem<TA>::kVec, VB = Elem<TB>::kVec;
   __shared__ float as[BK][BM + 4];
   __shared__ float bs[BK][BN + 4];
 
-  const TIn* a = static_cast<const TIn*>(g.a) + (long long)blockIdx.z * g.za;
-  const TIn* bt = static_cast<const TIn*>(g.bt) + (long long)blockIdx.z * g.zb;
+  const TA* a = static_cast<const TA*>(g.a) + (long long)blockIdx.z * g.za;
+  const TB* bt = static_cast<const TB*>(g.bt) + (long long)blockIdx.z * g.zb;
   TOut* c = static_cast<TOut*>(g.c) + (long long)blockIdx.z * g.zc;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -42,29 +42,29 @@ __global__ void __launch_bounds__(256) gemm_nt_fma_kernel(GemmArgs g) {
 
   for (int k0 = 0; k0 < g.k; k0 += BK) {
     // Stage A and Bt tiles (transposed to [k][row]) as fp32.
-    for (int v = tid; v < BM * (BK / V); v += 256) {
-      const int row = v / (BK / V), kv = (v % (BK / V)) * V;
-      float tmp[V];
+    for (int v = tid; v < BM * (BK / VA); v += 256) {
+      const int row = v / (BK / VA), kv = (v % (BK / VA)) * VA;
+      float tmp[VA];
       if (m0 + row < g.m && k0 + kv < g.k) {
         load_vec(a + (long long)(m0 + row) * g.lda + k0 + kv, tmp);
       } else {
 #pragma unroll
-        for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+        for (int e = 0; e < VA; ++e) tmp[e] = 0.f;
       }
 #pragma unroll
-      for (int e = 0; e < V; ++e) as[kv + e][row] = tmp[e];
+      for (int e = 0; e < VA; ++e) as[kv + e][row] = tmp[e];
     }
-    for (int v = tid; v < BN * (BK / V); v += 256) {
-      const int row = v / (BK / V), kv = (v % (BK / V)) * V;
-      float tmp[V];
+    for (int v = tid; v < BN * (BK / VB); v += 256) {
+      const int row = v / (BK / VB), kv = (v % (BK / VB)) * VB;
+      float tmp[VB];
       if (n0 + row < g.n && k0 + kv < g.k) {
         load_vec(bt + (long long)(n0 + row) * g.ldb + k0 + kv, tmp);
       } else {
 #pragma unroll
-        for (int e = 0; e < V; ++e) tmp[e] = 0.f;
+        for (int e = 0; e < VB; ++e) tmp[e] = 0.f;
       }
 #pragma unroll
-      for (int e = 0; e < V; ++e) bs[kv + e][row] = tmp[e];
+      for (int e = 0; e < VB; ++e) bs[kv + e][row] = tmp[e];
     }
     __syncthreads();
 #pragma unroll
@@ -96,19 +96,19 @@ __global__ void __launch_bounds__(256) gemm_nt_fma_kernel(GemmArgs g) {
 }
 
 // Launches the NT GEMM over `batches` z-slices.  K must be a multiple of the 16-byte
-// vector width of TIn and all row starts 16-byte aligned (checked by the caller).
-template <typename TIn, typename TOut>
+// vector widths of TA and TB and all row starts 16-byte aligned (guaranteed by the caller).
+template <typename TA, typename TB, typename TOut>
 inline cudaError_t launch_gemm_nt_fma(const GemmArgs& g, int batches, cudaStream_t st) {
   if (g.m <= 0 || g.n <= 0 || batches <= 0) return cudaSuccess;
   if (g.m <= 16) {
     dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 16), batches);
-    gemm_nt_fma_kernel<TIn, TOut, 16><<<grid, 256, 0, st>>>(g);
+    gemm_nt_fma_kernel<TA, TB, TOut, 16><<<grid, 256, 0, st>>>(g);
   } else if (g.m <= 64) {
     dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 64), batches);
-    gemm_nt_fma_kernel<TIn, TOut, 64><<<grid, 256, 0, st>>>(g);
+    gemm_nt_fma_kernel<TA, TB, TOut, 64><<<grid, 256, 0, st>>>(g);
   } else {
     dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 128), batches);
-    gemm_nt_fma_kernel<TIn, TOut, 128><<<grid, 256, 0, st>>>(g);
+    gemm_nt_fma_kernel<TA, TB, TOut, 128><<<grid, 256, 0, st>>>(g);
   }
   return cudaGetLastError();
 }

@@ -5,6 +5,7 @@
 #include <math.h>
 #include <new>
 #include <string.h>
+#include <vector>
 
 #include "common.cuh"
 #include "decode_kernels.cuh"
@@ -23,7 +24,7 @@ struct ArenaPlan {
   size_t wcat_t, w_k, w_kv_t, w_o_t;
   size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
   size_t cache, open_acc, err_flag;
-  size_t p1, q_t, qt, o_part, ml_part, o, v, x_stage, y_stage;
+  size_t p1, qt, o_part, ml_part, o, v, x_stage, y_stage;
   size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
   size_t total;
 };
@@ -93,21 +94,20 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->open_acc = take(B * dm.r * 4);
   p->err_flag = take(16);
   p->p1 = take(B * dm.ntot * 4);
-  p->q_t = take(B * hd * e);
-  p->qt = take(B * dm.nh * dm.W * e);
+  p->qt = take(B * dm.nh * dm.W * 4);
   p->o_part = take((size_t)dm.max_units * dm.nh * dm.r * 4);
   p->ml_part = take((size_t)dm.max_units * dm.nh * 2 * 4);
-  p->o = take(B * dm.nh * dm.r * e);
-  p->v = take(B * hd * e);
+  p->o = take(B * dm.nh * dm.r * 4);
+  p->v = take(B * hd * 4);
   p->x_stage = take(B * dm.d * e);
   p->y_stage = take(B * dm.d * e);
   const size_t rows = B * (size_t)c.max_prefill_tokens;
   p->pf_p1 = take(rows * dm.ntot * 4);
-  p->pf_qcat = take(rows * dm.nh * (dm.dh + dm.dr) * e);
+  p->pf_qcat = take(rows * dm.nh * (dm.dh + dm.dr) * 4);
   p->pf_cprime = take(rows * dm.r * e);
-  p->pf_kr = take(rows * dm.dr * e);
-  p->pf_kv = take(rows * 2 * hd * e);
-  p->pf_attn = take(rows * hd * e);
+  p->pf_kr = take(rows * dm.dr * 4);
+  p->pf_kv = take(rows * 2 * hd * 4);
+  p->pf_attn = take(rows * hd * 4);
   p->total = off;
 }
 
@@ -124,6 +124,9 @@ struct mtla_handle {
   int batch;    // 0 while the cache is empty and no batch has been fixed
   int64_t launches;
   bool attn_smem_ready, pf_smem_ready;
+  // Optional timing of the decode-attention kernel: one event pair per profiled step.
+  std::vector<cudaEvent_t> prof_events;
+  int prof_used;
 
   template <typename P> P* at(size_t off) const { return reinterpret_cast<P*>(arena + off); }
 };
@@ -152,7 +155,7 @@ int launch_widen(mtla_handle* h, const void* src, float* dst, long long n, cudaS
   return cudaGetLastError() == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
-template <typename TIn, typename TOut>
+template <typename TA, typename TB, typename TOut>
 int gemm(mtla_handle* h, const void* a, const void* bt, void* c, int m, int n, int k, int lda,
          int ldb, int ldc, float alpha, int batches, long long za, long long zb, long long zc,
          cudaStream_t st) {
@@ -160,7 +163,7 @@ int gemm(mtla_handle* h, const void* a, const void* bt, void* c, int m, int n, i
   g.a = a; g.bt = bt; g.c = c; g.m = m; g.n = n; g.k = k;
   g.lda = lda; g.ldb = ldb; g.ldc = ldc; g.za = za; g.zb = zb; g.zc = zc; g.alpha = alpha;
   h->launches++;
-  return launch_gemm_nt_fma<TIn, TOut>(g, batches, st) == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
+  return launch_gemm_nt_fma<TA, TB, TOut>(g, batches, st) == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
 #define MTLA_TRY(expr)            \
@@ -208,20 +211,20 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   return MTLA_OK;
 }
 
-template <typename T, int NH>
+template <typename T, typename TQ, int NH>
 int launch_attn_fma_rpt(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
   const size_t smem = attn_fma_smem_bytes(NH, a.r, a.dr);
   dim3 grid(a.n_split, B);
   if (a.r <= 256) {
     if (!h->attn_smem_ready)
-      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, NH, 1>,
+      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, TQ, NH, 1>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_attn_fma_kernel<T, NH, 1><<<grid, 256, smem, st>>>(a);
+    decode_attn_fma_kernel<T, TQ, NH, 1><<<grid, 256, smem, st>>>(a);
   } else {
     if (!h->attn_smem_ready)
-      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, NH, 2>,
+      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, TQ, NH, 2>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_attn_fma_kernel<T, NH, 2><<<grid, 256, smem, st>>>(a);
+    decode_attn_fma_kernel<T, TQ, NH, 2><<<grid, 256, smem, st>>>(a);
   }
   h->attn_smem_ready = true;
   h->launches++;
@@ -229,12 +232,12 @@ int launch_attn_fma_rpt(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t s
   return MTLA_OK;
 }
 
-template <typename T>
+template <typename T, typename TQ>
 int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
-  if (a.n_heads <= 4) return launch_attn_fma_rpt<T, 4>(h, a, B, st);
-  if (a.n_heads <= 8) return launch_attn_fma_rpt<T, 8>(h, a, B, st);
-  if (a.n_heads <= 16) return launch_attn_fma_rpt<T, 16>(h, a, B, st);
-  return launch_attn_fma_rpt<T, 32>(h, a, B, st);
+  if (a.n_heads <= 4) return launch_attn_fma_rpt<T, TQ, 4>(h, a, B, st);
+  if (a.n_heads <= 8) return launch_attn_fma_rpt<T, TQ, 8>(h, a, B, st);
+  if (a.n_heads <= 16) return launch_attn_fma_rpt<T, TQ, 16>(h, a, B, st);
+  return launch_attn_fma_rpt<T, TQ, 32>(h, a, B, st);
 }
 
 // The decode step (Section 4.1): a1 fused projection, a2-a5 post kernel, a6 absorption,
@@ -248,8 +251,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   const int slot = i0 / dm.s;
   const int n_slots = slot + 1;
 
-  MTLA_TRY((gemm<T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d, dm.d,
-                           dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d,
+                              dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
 
   PostArgs pa;
   pa.p1 = h->at<float>(p.p1);
@@ -263,7 +266,6 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   pa.rope_sin = h->at<float>(p.rope_sin) + (size_t)i0 * (dm.dr / 2);
   pa.open_acc = h->at<float>(p.open_acc);
   pa.cache = h->at<void>(p.cache);
-  pa.q_t = h->at<void>(p.q_t);
   pa.qt = h->at<void>(p.qt);
   pa.n_heads = dm.nh; pa.head_dim = dm.dh; pa.r = dm.r; pa.dr = dm.dr; pa.dw = dm.dw;
   pa.max_slots = dm.max_slots; pa.slot = slot;
@@ -271,13 +273,14 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
-  decode_post_kernel<T><<<B, 256, 0, st>>>(pa);
+  decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
 
-  // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head.
-  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.q_t), h->at<T>(p.w_k), h->at<T>(p.qt), B, dm.r, dm.dh, hd, hd,
-                       dm.nh * dm.W, pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
+  // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection.
+  MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
+                                  h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
+                                  pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
 
   AttnArgs aa;
   aa.qt = h->at<void>(p.qt);
@@ -291,21 +294,27 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   if (n_split < 1) n_split = 1;
   aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
   aa.n_split = ceil_div(n_slots, aa.slots_per_split);
-  MTLA_TRY(launch_attn_fma<T>(h, aa, B, st));
+  const bool prof = h->prof_used + 2 <= (int)h->prof_events.size();
+  if (prof) MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used], st));
+  MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st)));
+  if (prof) {
+    MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used + 1], st));
+    h->prof_used += 2;
+  }
 
   CombineArgs ca;
   ca.o_part = aa.o_part; ca.ml_part = aa.ml_part; ca.o = h->at<void>(p.o);
   ca.n_heads = dm.nh; ca.r = dm.r; ca.n_split = aa.n_split;
-  decode_combine_kernel<T><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
+  decode_combine_kernel<float><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
 
   // a8: v_h = o_h W_{V,h} per head, then y = concat_h(v_h) W_O.
-  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r, h->at<T>(p.v), B,
-                       dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f, dm.nh, dm.r,
-                       (long long)dm.dh * dm.r, dm.dh, st)));
-  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.v), h->at<T>(p.w_o_t), y, B, dm.d, hd, hd, hd, dm.d, 1.f, 1, 0,
-                       0, 0, st)));
+  MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r,
+                                  h->at<float>(p.v), B, dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f,
+                                  dm.nh, dm.r, (long long)dm.dh * dm.r, dm.dh, st)));
+  MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.v), h->at<T>(p.w_o_t), y, B, dm.d, hd, hd, hd,
+                              dm.d, 1.f, 1, 0, 0, 0, st)));
   return MTLA_OK;
 }
 
@@ -317,8 +326,8 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   const int rows = B * T_len;
   const float q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
 
-  MTLA_TRY((gemm<T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot, dm.d,
-                           dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot,
+                              dm.d, dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
   PrefillPostArgs pa;
   pa.p1 = h->at<float>(p.pf_p1);
   pa.proj = dm.proj;
@@ -339,14 +348,14 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = q_scale;
-  prefill_post_kernel<T><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
+  prefill_post_kernel<T, float><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
   if (!y) return MTLA_OK;
 
   // Eq. 9-10 on the running-state sequence: keys and values of every column.
-  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<T>(p.pf_kv), rows,
-                       2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
+  MTLA_TRY((gemm<T, T, float>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<float>(p.pf_kv),
+                              rows, 2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
   PrefillAttnArgs aa;
   aa.qcat = pa.qcat; aa.kv = h->at<void>(p.pf_kv); aa.kr = pa.kr; aa.out = h->at<void>(p.pf_attn);
   aa.n_heads = dm.nh; aa.dr = dm.dr; aa.stride = dm.s; aa.T = T_len;
@@ -354,20 +363,20 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   dim3 grid(ceil_div(T_len, kPfTile), dm.nh, B);
   if (dm.dh == 64) {
     if (!h->pf_smem_ready)
-      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<T, 64>,
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, 64>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    prefill_attn_fma_kernel<T, 64><<<grid, 256, smem, st>>>(aa);
+    prefill_attn_fma_kernel<float, 64><<<grid, 256, smem, st>>>(aa);
   } else {
     if (!h->pf_smem_ready)
-      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<T, 128>,
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, 128>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    prefill_attn_fma_kernel<T, 128><<<grid, 256, smem, st>>>(aa);
+    prefill_attn_fma_kernel<float, 128><<<grid, 256, smem, st>>>(aa);
   }
   h->pf_smem_ready = true;
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
-  MTLA_TRY((gemm<T, T>(h, h->at<T>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd, hd, dm.d,
-                       1.f, 1, 0, 0, 0, st)));
+  MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd,
+                              hd, dm.d, 1.f, 1, 0, 0, 0, st)));
   return MTLA_OK;
 }
 
@@ -414,6 +423,7 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
   h->tokens = 0; h->batch = 0; h->launches = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
+  h->prof_used = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int rc = c.dtype == MTLA_DTYPE_BF16 ? create_impl<bf16>(h, w, st) : create_impl<float>(h, w, st);
   if (rc != MTLA_OK) {
@@ -477,6 +487,7 @@ size_t mtla_cache_bytes(const mtla_handle* h) {
 
 int mtla_destroy(mtla_handle* h) {
   if (!h) return MTLA_ERR_INVALID_ARG;
+  for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
   delete h;
   return MTLA_OK;
 }
@@ -543,6 +554,36 @@ int mtla_check(mtla_handle* h, void* stream) {
 }
 
 int64_t mtla_launch_count(const mtla_handle* h) { return h ? h->launches : 0; }
+
+int mtla_profile_begin(mtla_handle* h, int32_t max_steps) {
+  if (!h || max_steps <= 0) return MTLA_ERR_INVALID_ARG;
+  for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+  h->prof_events.clear();
+  h->prof_used = 0;
+  for (int i = 0; i < 2 * max_steps; ++i) {
+    cudaEvent_t e;
+    MTLA_CUDA(cudaEventCreate(&e));
+    h->prof_events.push_back(e);
+  }
+  return MTLA_OK;
+}
+
+int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps) {
+  if (!h || !attention_ms || !steps) return MTLA_ERR_INVALID_ARG;
+  double total = 0.0;
+  for (int i = 0; i + 1 < h->prof_used; i += 2) {
+    MTLA_CUDA(cudaEventSynchronize(h->prof_events[i + 1]));
+    float ms = 0.f;
+    MTLA_CUDA(cudaEventElapsedTime(&ms, h->prof_events[i], h->prof_events[i + 1]));
+    total += ms;
+  }
+  *attention_ms = total;
+  *steps = h->prof_used / 2;
+  for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+  h->prof_events.clear();
+  h->prof_used = 0;
+  return MTLA_OK;
+}
 
 const char* mtla_attention_variant(const mtla_handle* h) {
   (void)h;

@@ -23,7 +23,7 @@ struct PrefillPostArgs {
   void* cache;            // [max_batch][max_slots][r + d_R]
   void* qcat;             // [B*T][n_h][d_h + d_R]: scaled query and rotated RoPE query
   void* cprime;           // [B*T][r]: running merge state after each token (Eq. 14's sequence)
-  void* kr;               // [B*T][d_R]: rotated RoPE key of each token
+  void* kr;               // [B*T][d_R]: rotated RoPE key of each token (query element type)
   int n_heads, head_dim, r, dr, dw, stride, T, max_slots;
   int use_gate;
   float ln_eps, q_scale;
@@ -32,7 +32,8 @@ struct PrefillPostArgs {
 // One CTA per (chunk, sequence): walks the chunk's <= s tokens in order so that the running
 // sum is formed exactly as the decode steps would form it, and leaves the chunk's final
 // state in the cache (the last chunk also leaves the fp32 accumulator for later decoding).
-template <typename T>
+// T is the cache / state element type, TQ the element type of the query buffer.
+template <typename T, typename TQ>
 __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
   __shared__ float c_s[512];
   __shared__ float acc_s[512];
@@ -96,25 +97,28 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
     }
     const float* cs_row = a.rope_cos + (long long)tok * half;
     const float* sn_row = a.rope_sin + (long long)tok * half;
-    T* kr = static_cast<T*>(a.kr) + rowi * a.dr;
+    // Keys are rounded to the cache type (what decoding would read back), held as TQ.
+    TQ* kr = static_cast<TQ*>(a.kr) + rowi * a.dr;
     for (int k = tid; k < half; k += 256) {
       const float x0 = row[a.proj.off_kr + 2 * k], x1 = row[a.proj.off_kr + 2 * k + 1];
-      kr[2 * k] = Elem<T>::from_float(x0 * cs_row[k] - x1 * sn_row[k]);
-      kr[2 * k + 1] = Elem<T>::from_float(x0 * sn_row[k] + x1 * cs_row[k]);
+      const T k0 = Elem<T>::from_float(x0 * cs_row[k] - x1 * sn_row[k]);
+      const T k1 = Elem<T>::from_float(x0 * sn_row[k] + x1 * cs_row[k]);
+      kr[2 * k] = Elem<TQ>::from_float(Elem<T>::to_float(k0));
+      kr[2 * k + 1] = Elem<TQ>::from_float(Elem<T>::to_float(k1));
     }
-    T* qc = static_cast<T*>(a.qcat) + rowi * a.n_heads * DQ;
+    TQ* qc = static_cast<TQ*>(a.qcat) + rowi * a.n_heads * DQ;
     for (int i = tid; i < a.n_heads * a.head_dim; i += 256) {
       const int h = i / a.head_dim, e = i % a.head_dim;
-      qc[h * DQ + e] = Elem<T>::from_float(row[a.proj.off_q + i] * a.q_scale);
+      qc[h * DQ + e] = Elem<TQ>::from_float(row[a.proj.off_q + i] * a.q_scale);
     }
     for (int i = tid; i < a.n_heads * half; i += 256) {
       const int h = i / half, k = i % half;
       const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k];
       const float x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
       qc[h * DQ + a.head_dim + 2 * k] =
-          Elem<T>::from_float((x0 * cs_row[k] - x1 * sn_row[k]) * a.q_scale);
+          Elem<TQ>::from_float((x0 * cs_row[k] - x1 * sn_row[k]) * a.q_scale);
       qc[h * DQ + a.head_dim + 2 * k + 1] =
-          Elem<T>::from_float((x0 * sn_row[k] + x1 * cs_row[k]) * a.q_scale);
+          Elem<TQ>::from_float((x0 * sn_row[k] + x1 * cs_row[k]) * a.q_scale);
     }
   }
   __syncthreads();
@@ -122,9 +126,10 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
   // The chunk's state after its last available token is what the cache holds.
   const long long last = (long long)b * a.T + (tok1 - 1);
   T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + chunk) * W;
-  const T* kr = static_cast<const T*>(a.kr) + last * a.dr;
+  const TQ* kr = static_cast<const TQ*>(a.kr) + last * a.dr;
   for (int i = tid; i < a.r; i += 256) slot_row[i] = Elem<T>::from_float(acc_s[i]);
-  for (int i = tid; i < a.dr; i += 256) slot_row[a.r + i] = kr[i];
+  for (int i = tid; i < a.dr; i += 256)
+    slot_row[a.r + i] = Elem<T>::from_float(Elem<TQ>::to_float(kr[i]));
   if (tok1 == a.T)
     for (int i = tid; i < a.r; i += 256) a.open_acc[(long long)b * a.r + i] = acc_s[i];
 }
@@ -150,10 +155,11 @@ inline size_t prefill_attn_fma_smem_bytes(int dh, int dr) {
 // j*s + s - 1, plus its own running state at column m: exactly the columns the
 // stride-aware mask of Section 4.2 admits.  The mask is a predicate on (m, j).
 // Grid (ceil(T/64), n_h, B), 256 threads as 16 x 16, each owning a 4 x 4 score patch.
-template <typename T, int DH>
+// TQ = element type of queries, keys, values, RoPE keys and outputs.
+template <typename TQ, int DH>
 __global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a) {
   extern __shared__ float smem[];
-  constexpr int BT = kPfTile, V = Elem<T>::kVec, OC = DH / 16;
+  constexpr int BT = kPfTile, V = Elem<TQ>::kVec, OC = DH / 16;
   const int DQ = DH + a.dr;
   float* qs = smem;                 // [DQ][BT]  (transposed: k-major)
   float* ks = qs + DQ * BT;         // [DQ][BT]
@@ -161,9 +167,9 @@ __global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a
   float* ps = vs + BT * DH;         // [BT][BT+1]
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int q0 = blockIdx.x * BT, h = blockIdx.y, b = blockIdx.z;
-  const T* qcat = static_cast<const T*>(a.qcat);
-  const T* kv = static_cast<const T*>(a.kv);
-  const T* kr = static_cast<const T*>(a.kr);
+  const TQ* qcat = static_cast<const TQ*>(a.qcat);
+  const TQ* kv = static_cast<const TQ*>(a.kv);
+  const TQ* kr = static_cast<const TQ*>(a.kr);
   const long long base = (long long)b * a.T;
   const int kvw = 2 * a.n_heads * DH;
 
@@ -288,7 +294,7 @@ __global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a
     }
   }
 
-  T* out = static_cast<T*>(a.out);
+  TQ* out = static_cast<TQ*>(a.out);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int row = q0 + ty * 4 + i;
@@ -297,7 +303,7 @@ __global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a
 #pragma unroll
     for (int c = 0; c < OC; ++c)
       out[(base + row) * a.n_heads * DH + h * DH + tx * OC + c] =
-          Elem<T>::from_float(o[i][c] * inv);
+          Elem<TQ>::from_float(o[i][c] * inv);
   }
 }
 
