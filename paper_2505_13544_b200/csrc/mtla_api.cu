@@ -2,12 +2,15 @@
 // repacking and the launch sequences of the decode step and the prefill.
 #include "mtla.h"
 
+#include <cuda.h>
 #include <math.h>
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 #include <vector>
 
 #include "common.cuh"
+#include "decode_attn_tc.cuh"
 #include "decode_kernels.cuh"
 #include "gemm_fma.cuh"
 #include "prefill_kernels.cuh"
@@ -17,6 +20,7 @@ using namespace mtla;
 
 namespace {
 
+constexpr int kSmCount = 148;        // B200
 constexpr int kTargetCtas = 296;     // two CTAs per SM on a 148-SM part
 constexpr int kMinSlotsPerSplit = 64;
 
@@ -124,6 +128,9 @@ struct mtla_handle {
   int batch;    // 0 while the cache is empty and no batch has been fixed
   int64_t launches;
   bool attn_smem_ready, pf_smem_ready;
+  // Tensor-core decode attention (bf16, r a multiple of 128): TMA view of the cache.
+  bool use_tc;
+  CUtensorMap cache_map;
   // Optional timing of the decode-attention kernel: one event pair per profiled step.
   std::vector<cudaEvent_t> prof_events;
   int prof_used;
@@ -172,6 +179,55 @@ int gemm(mtla_handle* h, const void* a, const void* bt, void* c, int m, int n, i
     if (rc_ != MTLA_OK) return rc_; \
   } while (0)
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// TMA view of the bf16 cache [max_batch][max_slots][r + d_R]: boxes of 128 slots x 64
+// columns (128 bytes, the swizzle span), zero fill outside the tensor.
+int make_cache_map(mtla_handle* h) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn)
+    return MTLA_ERR_CUDA;
+  const Dims& dm = h->dm;
+  const cuuint64_t dims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.max_slots, (cuuint64_t)h->cfg.max_batch};
+  const cuuint64_t strides[2] = {(cuuint64_t)dm.W * 2, (cuuint64_t)dm.max_slots * dm.W * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult rc = reinterpret_cast<EncodeTiledFn>(fn)(
+      &h->cache_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->at<void>(h->plan.cache), dims, strides,
+      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+template <int NHP>
+int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int B, cudaStream_t st) {
+  dim3 grid(a.n_split, B);
+#define MTLA_TC_CASE(RP)                                                                       \
+  case RP:                                                                                     \
+    if (!h->attn_smem_ready)                                                                   \
+      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP>,                           \
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes)); \
+    decode_attn_tc_kernel<NHP, RP><<<grid, 256, tc::kSmemBytes, st>>>(h->cache_map, a);         \
+    break;
+  switch (a.r / 128) {
+    MTLA_TC_CASE(1)
+    MTLA_TC_CASE(2)
+    MTLA_TC_CASE(3)
+    MTLA_TC_CASE(4)
+    default: return MTLA_ERR_UNSUPPORTED_SHAPE;
+  }
+#undef MTLA_TC_CASE
+  h->attn_smem_ready = true;
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  return MTLA_OK;
+}
+
 template <typename T>
 int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   const Dims& dm = h->dm;
@@ -208,6 +264,11 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.err_flag), 0, 16, st));
+  // Unused cache rows must hold finite values: the tensor-core kernel multiplies rows
+  // beyond the valid range by a zero probability.
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.cache), 0,
+                            (size_t)h->cfg.max_batch * dm.max_slots * dm.W * dm.elem, st));
+  if (h->use_tc) MTLA_TRY(make_cache_map(h));
   return MTLA_OK;
 }
 
@@ -273,14 +334,21 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
-  decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
+  if (h->use_tc) decode_post_kernel<T, bf16><<<B, 256, 0, st>>>(pa);
+  else decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
 
-  // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection.
-  MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
-                                  h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
-                                  pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
+  // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection
+  // (bf16 output where the tensor-core attention consumes it).
+  if (h->use_tc)
+    MTLA_TRY((gemm<float, T, bf16>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
+                                   h->at<bf16>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
+                                   pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
+  else
+    MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
+                                    h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
+                                    pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
 
   AttnArgs aa;
   aa.qt = h->at<void>(p.qt);
@@ -289,14 +357,30 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   aa.ml_part = h->at<float>(p.ml_part);
   aa.n_heads = dm.nh; aa.r = dm.r; aa.dr = dm.dr; aa.max_slots = dm.max_slots;
   aa.n_slots = n_slots;
-  int want = ceil_div(kTargetCtas, B);
-  int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
-  if (n_split < 1) n_split = 1;
-  aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
-  aa.n_split = ceil_div(n_slots, aa.slots_per_split);
   const bool prof = h->prof_used + 2 <= (int)h->prof_events.size();
-  if (prof) MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used], st));
-  MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st)));
+  if (h->use_tc) {
+    // One CTA per SM: as many splits per sequence as keep B * n_split within the SM count.
+    int n_split = min(max(1, kSmCount / B), ceil_div(n_slots, tc::kTile));
+    aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), tc::kTile) * tc::kTile;
+    aa.n_split = ceil_div(n_slots, aa.slots_per_split);
+    AttnTcArgs ta;
+    ta.qt = h->at<bf16>(p.qt);
+    ta.o_part = aa.o_part; ta.ml_part = aa.ml_part;
+    ta.error_word = h->at<int>(p.err_flag);
+    ta.n_heads = dm.nh; ta.r = dm.r; ta.dr = dm.dr; ta.n_slots = n_slots;
+    ta.slots_per_split = aa.slots_per_split; ta.n_split = aa.n_split;
+    if (prof) MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used], st));
+    if (dm.nh <= 16) MTLA_TRY(launch_attn_tc_rp<16>(h, ta, B, st));
+    else MTLA_TRY(launch_attn_tc_rp<32>(h, ta, B, st));
+  } else {
+    int want = ceil_div(kTargetCtas, B);
+    int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
+    if (n_split < 1) n_split = 1;
+    aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
+    aa.n_split = ceil_div(n_slots, aa.slots_per_split);
+    if (prof) MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used], st));
+    MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st)));
+  }
   if (prof) {
     MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used + 1], st));
     h->prof_used += 2;
@@ -424,6 +508,10 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   h->tokens = 0; h->batch = 0; h->launches = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
+  // The tensor-core attention needs bf16 and whole 128-column latent blocks; the
+  // MTLA_ATTENTION=fma environment override keeps the CUDA-core kernel for comparisons.
+  const char* force = getenv("MTLA_ATTENTION");
+  h->use_tc = c.dtype == MTLA_DTYPE_BF16 && dm.r % 128 == 0 && !(force && !strcmp(force, "fma"));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int rc = c.dtype == MTLA_DTYPE_BF16 ? create_impl<bf16>(h, w, st) : create_impl<float>(h, w, st);
   if (rc != MTLA_OK) {
@@ -586,8 +674,7 @@ int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps) {
 }
 
 const char* mtla_attention_variant(const mtla_handle* h) {
-  (void)h;
-  return "fma";
+  return (h && h->use_tc) ? "tcgen05" : "fma";
 }
 
 const char* mtla_error_string(int status) {
