@@ -161,11 +161,22 @@ def oracle_decode_sample(w: synth.Workload, n_seq: int, budget_s: float, max_ste
             "seconds": elapsed, "steps": steps}
 
 
+def pick_workload(args) -> synth.Workload:
+    """The named workload, optionally shrunk (the name then says how)."""
+    w = synth.WORKLOADS[args.workload]
+    if args.batch:
+        w = w.scaled(batch=args.batch, name=f"{w.name}[batch={args.batch}]")
+    if args.context_tokens and w.context_tokens:
+        w = w.scaled(context_tokens=args.context_tokens,
+                     name=f"{w.name}[context_tokens={args.context_tokens}]")
+    return w
+
+
 def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = synth.WORKLOADS[args.workload]
+    w = pick_workload(args)
     n_seq = 1 if w.batch * w.latent_rank >= 8192 else min(w.batch, 4)
     # warm-up steps are run and discarded, then exactly --steps sample steps are timed
     oracle_decode_sample(w, n_seq, 0.0, 0, exact_steps=min(args.warmup, 1))
@@ -241,6 +252,10 @@ def main() -> None:
     ap.add_argument("--workload", default="large", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch (profiling-sized variants)")
+    ap.add_argument("--context-tokens", type=int, default=0,
+                    help="override the workload's imported context length")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -262,7 +277,7 @@ def main() -> None:
             dist.barrier(device_ids=[local])
         torch.cuda.synchronize(device)
 
-    w = synth.WORKLOADS[args.workload]
+    w = pick_workload(args)
     K, W = args.steps, max(args.warmup, 3)
     M, h = build_layer(w, extra_steps=2 * (K + W), device=device)
     extras = fill_context(M, h, w, device)

@@ -27,6 +27,8 @@ struct PostArgs {
   float* open_acc;        // [B][r] fp32 running sum of the open slot
   void* cache;            // [max_batch][max_slots][r + d_R]
   void* qt;               // [B][n_h][r + d_R] absorbed query; this kernel writes the RoPE tail
+  bf16* q16;              // [B][2*n_h*d_h]: q as bf16 [hi | lo] halves (q = hi + lo) for the
+                          // tensor-core absorption, or nullptr
   int n_heads, head_dim, r, dr, dw;
   int max_slots, slot;    // slot = 0-based slot index receiving this token
   int new_slot;           // 1 when the token opens the slot (tokens mod s == 0)
@@ -103,6 +105,17 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
     const float cs = a.rope_cos[k], sn = a.rope_sin[k];
     slot_row[a.r + 2 * k] = Elem<T>::from_float(x0 * cs - x1 * sn);
     slot_row[a.r + 2 * k + 1] = Elem<T>::from_float(x0 * sn + x1 * cs);
+  }
+  if (a.q16) {
+    const int hd = a.n_heads * a.head_dim;
+    for (int i = tid * 2; i < hd; i += 512) {
+      const float q0 = row[a.proj.off_q + i], q1 = row[a.proj.off_q + i + 1];
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(q0, q1);
+      bf16* dst = a.q16 + (long long)b * 2 * hd + i;
+      *reinterpret_cast<__nv_bfloat162*>(dst) = hi;
+      *reinterpret_cast<__nv_bfloat162*>(dst + hd) =
+          __floats2bfloat162_rn(q0 - __low2float(hi), q1 - __high2float(hi));
+    }
   }
   // Rotated, pre-scaled RoPE queries behind the (separately computed) absorbed query.
   TQ* qt = static_cast<TQ*>(a.qt) + (long long)b * a.n_heads * W;
@@ -262,7 +275,8 @@ __global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
 struct CombineArgs {
   const float* o_part;   // [B * n_split][n_h][r]
   const float* ml_part;  // [B * n_split][n_h][2]
-  void* o;               // [B][n_h][r] normalised attention output in latent space
+  void* o;               // [B][n_h][r] normalised attention output in latent space; for bf16
+                         // rows are [2][n_h][r]: hi halves, then the rounding remainders
   int n_heads, r, n_split;
 };
 
@@ -280,7 +294,9 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(CombineArgs a) {
     denom += exp2f(ml[0] - m) * ml[1];
   }
   const float inv = 1.f / denom;
-  T* o = static_cast<T*>(a.o) + ((long long)b * a.n_heads + h) * a.r;
+  constexpr bool kSplit = sizeof(T) == 2;
+  const long long lo_off = (long long)a.n_heads * a.r;
+  T* o = static_cast<T*>(a.o) + ((long long)b * (kSplit ? 2 : 1) * a.n_heads + h) * a.r;
   for (int col = threadIdx.x; col < a.r; col += 128) {
     float sum = 0.f;
     for (int sp = 0; sp < a.n_split; ++sp) {
@@ -288,7 +304,10 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(CombineArgs a) {
       const float wgt = exp2f(a.ml_part[(unit * a.n_heads + h) * 2] - m);
       sum = fmaf(wgt, a.o_part[(unit * a.n_heads + h) * a.r + col], sum);
     }
-    o[col] = Elem<T>::from_float(sum * inv);
+    const float val = sum * inv;
+    const T hi = Elem<T>::from_float(val);
+    o[col] = hi;
+    if (kSplit) o[lo_off + col] = Elem<T>::from_float(val - Elem<T>::to_float(hi));
   }
 }
 

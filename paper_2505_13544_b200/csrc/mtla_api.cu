@@ -13,6 +13,7 @@
 #include "decode_attn_tc.cuh"
 #include "decode_kernels.cuh"
 #include "gemm_fma.cuh"
+#include "gemm_tc.cuh"
 #include "prefill_kernels.cuh"
 #include "setup_kernels.cuh"
 
@@ -23,12 +24,21 @@ namespace {
 constexpr int kSmCount = 148;        // B200
 constexpr int kTargetCtas = 296;     // two CTAs per SM on a 148-SM part
 constexpr int kMinSlotsPerSplit = 64;
+constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill projections
+constexpr int kGemmSlots = 2 * kSmCount;   // CTAs a split-K GEMM may spread one product over
+
+// Rows of the activation-side TMA box (the MMA's N) for a decode batch of B sequences.
+int act_box_rows(int B) {
+  for (int bn = 16; bn < 256; bn *= 2)
+    if (B <= bn) return bn;
+  return 256;
+}
 
 struct ArenaPlan {
   size_t wcat_t, w_k, w_kv_t, w_o_t;
   size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
   size_t cache, open_acc, err_flag;
-  size_t p1, qt, o_part, ml_part, o, v, x_stage, y_stage;
+  size_t p1, q16, qt, o_part, ml_part, o, v, x_stage, y_stage, gemm_part, gemm_tickets;
   size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
   size_t total;
 };
@@ -98,6 +108,7 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->open_acc = take(B * dm.r * 4);
   p->err_flag = take(16);
   p->p1 = take(B * dm.ntot * 4);
+  p->q16 = take(B * 2 * hd * 2);
   p->qt = take(B * dm.nh * dm.W * 4);
   p->o_part = take((size_t)dm.max_units * dm.nh * dm.r * 4);
   p->ml_part = take((size_t)dm.max_units * dm.nh * 2 * 4);
@@ -105,6 +116,10 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->v = take(B * hd * 4);
   p->x_stage = take(B * dm.d * e);
   p->y_stage = take(B * dm.d * e);
+  // Split-K workspace of the tensor-core GEMMs: at most kGemmSlots CTAs hold a partial tile.
+  p->gemm_part = take(c.dtype == MTLA_DTYPE_BF16
+                          ? (size_t)kGemmSlots * gtc::kBM * act_box_rows(c.max_batch) * 4 : 0);
+  p->gemm_tickets = take((size_t)kGemmSlots * 4 * sizeof(int));
   const size_t rows = B * (size_t)c.max_prefill_tokens;
   p->pf_p1 = take(rows * dm.ntot * 4);
   p->pf_qcat = take(rows * dm.nh * (dm.dh + dm.dr) * 4);
@@ -131,6 +146,12 @@ struct mtla_handle {
   // Tensor-core decode attention (bf16, r a multiple of 128): TMA view of the cache.
   bool use_tc;
   CUtensorMap cache_map;
+  // Tensor-core projections (bf16): weight panels as 128-row boxes, serving as the MMA's M side
+  // in the decode step and as its N side in the prefill; decode activations as act_bn-row boxes.
+  CUtensorMap map_wcat, map_wk, map_wkvt, map_wvt, map_wot;
+  CUtensorMap map_q16, map_o16, map_v16;
+  int act_bn;               // box rows the three activation maps were encoded with (0: none yet)
+  unsigned gemm_attr_mask;  // kernel instances whose shared-memory limit has been raised
   // Optional timing of the decode-attention kernel: one event pair per profiled step.
   std::vector<cudaEvent_t> prof_events;
   int prof_used;
@@ -184,24 +205,107 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// TMA view of the bf16 cache [max_batch][max_slots][r + d_R]: boxes of 128 slots x 64
-// columns (128 bytes, the swizzle span), zero fill outside the tensor.
-int make_cache_map(mtla_handle* h) {
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn cached = nullptr;
+  if (cached) return cached;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess || !fn)
-    return MTLA_ERR_CUDA;
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  cached = reinterpret_cast<EncodeTiledFn>(fn);
+  return cached;
+}
+
+// TMA view of the bf16 cache [max_batch][max_slots][r + d_R]: boxes of 128 slots x 64
+// columns (128 bytes, the swizzle span), zero fill outside the tensor.
+int make_cache_map(mtla_handle* h) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return MTLA_ERR_CUDA;
   const Dims& dm = h->dm;
   const cuuint64_t dims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.max_slots, (cuuint64_t)h->cfg.max_batch};
   const cuuint64_t strides[2] = {(cuuint64_t)dm.W * 2, (cuuint64_t)dm.max_slots * dm.W * 2};
   const cuuint32_t box[3] = {64, 128, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult rc = reinterpret_cast<EncodeTiledFn>(fn)(
+  const CUresult rc = fn(
       &h->cache_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->at<void>(h->plan.cache), dims, strides,
       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+// TMA view of a row-major bf16 matrix [rows][cols] with leading dimension ld (elements):
+// boxes of box_rows rows x 64 columns (128 bytes, the swizzle span), zero fill outside.
+int make_map_2d(CUtensorMap* map, const void* ptr, long long rows, long long cols, long long ld,
+                int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return MTLA_ERR_CUDA;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims,
+                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+template <int BN, int STAGES, typename OutT>
+int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
+                        const GemmTcArgs& g, dim3 grid, cudaStream_t st) {
+  constexpr int smem = gtc::smem_bytes(BN, STAGES);
+  if (!(h->gemm_attr_mask & (1u << inst))) {
+    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    h->gemm_attr_mask |= 1u << inst;
+  }
+  gemm_tc_kernel<BN, STAGES, OutT><<<grid, 192, smem, st>>>(ma, mb, g);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  return MTLA_OK;
+}
+
+// D[z][i][j] = alpha * sum_k A[z][i][k] B[z][j][k] on the tensor cores (see gemm_tc.cuh).
+// `bn` is the row count of map_b's box.  With allow_split the reduction is spread over
+// several CTAs when the tile count alone would leave most SMs idle.
+template <typename OutT>
+int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTcArgs g, int bn,
+            int batches, bool allow_split, cudaStream_t st) {
+  const int m_tiles = ceil_div(g.m, gtc::kBM);
+  g.m_tiles = m_tiles;
+  g.n_tiles = ceil_div(g.n, bn);
+  const long long tiles = (long long)m_tiles * g.n_tiles * batches;
+  const int kb_total = ceil_div(g.k, gtc::kBK);
+  int n_split = 1;
+  if (allow_split && tiles < kGemmSlots)
+    n_split = max(1, min(kb_total / 4, (int)(kGemmSlots / tiles)));
+  g.kb_per_split = ceil_div(kb_total, n_split);
+  g.n_split = ceil_div(kb_total, g.kb_per_split);
+  g.partial = h->at<float>(h->plan.gemm_part);
+  g.tickets = h->at<int>(h->plan.gemm_tickets);
+  g.error_word = h->at<int>(h->plan.err_flag);
+  const size_t osz = sizeof(OutT);
+  g.vec_ok = (reinterpret_cast<uintptr_t>(g.c) % 16 == 0) && (g.c_sm * osz % 16 == 0) &&
+             (g.c_sz * osz % 16 == 0);
+  if ((long long)m_tiles * g.n_tiles * g.n_split > 0x7fffffffll) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
+  constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
+  switch (bn) {
+    case 16: return launch_gemm_tc_inst<16, 4, OutT>(h, 0 + o, ma, mb, g, grid, st);
+    case 32: return launch_gemm_tc_inst<32, 4, OutT>(h, 2 + o, ma, mb, g, grid, st);
+    case 64: return launch_gemm_tc_inst<64, 4, OutT>(h, 4 + o, ma, mb, g, grid, st);
+    case 128: return launch_gemm_tc_inst<128, 3, OutT>(h, 6 + o, ma, mb, g, grid, st);
+    case 256: return launch_gemm_tc_inst<256, 4, OutT>(h, 8 + o, ma, mb, g, grid, st);
+    default: return MTLA_ERR_UNSUPPORTED_SHAPE;
+  }
+}
+
+GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, int k, float alpha) {
+  GemmTcArgs g;
+  memset(&g, 0, sizeof(g));
+  g.c = c; g.c_sm = c_sm; g.c_sn = c_sn; g.m = m; g.n = n; g.k = k; g.alpha = alpha;
+  return g;
 }
 
 template <int NHP>
@@ -268,7 +372,31 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   // beyond the valid range by a zero probability.
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.cache), 0,
                             (size_t)h->cfg.max_batch * dm.max_slots * dm.W * dm.elem, st));
-  if (h->use_tc) MTLA_TRY(make_cache_map(h));
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.gemm_tickets), 0, (size_t)kGemmSlots * 4 * sizeof(int), st));
+  if (h->use_tc) {
+    MTLA_TRY(make_cache_map(h));
+    MTLA_TRY(make_map_2d(&h->map_wcat, h->at<void>(p.wcat_t), dm.ntot, dm.d, dm.d, gtc::kBM));
+    MTLA_TRY(make_map_2d(&h->map_wk, h->at<void>(p.w_k), dm.r, hd, hd, gtc::kBM));
+    MTLA_TRY(make_map_2d(&h->map_wkvt, h->at<void>(p.w_kv_t), 2 * hd, dm.r, dm.r, gtc::kBM));
+    MTLA_TRY(make_map_2d(&h->map_wvt, h->at<T>(p.w_kv_t) + (size_t)hd * dm.r, hd, dm.r, dm.r, gtc::kBM));
+    MTLA_TRY(make_map_2d(&h->map_wot, h->at<void>(p.w_o_t), dm.d, hd, hd, gtc::kBM));
+  }
+  return MTLA_OK;
+}
+
+// (Re-)encodes the TMA views of the decode step's bf16 intermediates for a batch of B rows.
+int ensure_activation_maps(mtla_handle* h, int B) {
+  const int bn = act_box_rows(B);
+  if (h->act_bn == bn) return MTLA_OK;
+  const Dims& dm = h->dm;
+  const ArenaPlan& p = h->plan;
+  const int hd = dm.nh * dm.dh, mb = h->cfg.max_batch;
+  // Each intermediate row holds the bf16 [hi | lo] halves of an fp32 activation.
+  const long long onr = (long long)dm.nh * dm.r;
+  MTLA_TRY(make_map_2d(&h->map_q16, h->at<void>(p.q16), mb, 2 * hd, 2 * hd, bn));
+  MTLA_TRY(make_map_2d(&h->map_o16, h->at<void>(p.o), mb, 2 * onr, 2 * onr, bn));
+  MTLA_TRY(make_map_2d(&h->map_v16, h->at<void>(p.v), mb, 2 * hd, 2 * hd, bn));
+  h->act_bn = bn;
   return MTLA_OK;
 }
 
@@ -312,8 +440,19 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   const int slot = i0 / dm.s;
   const int n_slots = slot + 1;
 
-  MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d,
-                              dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  const int bn = act_box_rows(B);
+  if (h->use_tc) {
+    // a1 on the tensor cores: weights stream through the MMA's M side, the batch sits in N.
+    MTLA_TRY(ensure_activation_maps(h, B));
+    CUtensorMap map_x;
+    MTLA_TRY(make_map_2d(&map_x, x, B, dm.d, dm.d, bn));
+    MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x,
+                            gemm_tc_args(h->at<float>(p.p1), 1, dm.ntot, dm.ntot, B, dm.d, 1.f), bn, 1,
+                            true, st));
+  } else {
+    MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d,
+                                dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  }
 
   PostArgs pa;
   pa.p1 = h->at<float>(p.p1);
@@ -328,6 +467,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   pa.open_acc = h->at<float>(p.open_acc);
   pa.cache = h->at<void>(p.cache);
   pa.qt = h->at<void>(p.qt);
+  pa.q16 = h->use_tc ? h->at<bf16>(p.q16) : nullptr;
   pa.n_heads = dm.nh; pa.head_dim = dm.dh; pa.r = dm.r; pa.dr = dm.dr; pa.dw = dm.dw;
   pa.max_slots = dm.max_slots; pa.slot = slot;
   pa.new_slot = (i0 % dm.s) == 0;
@@ -341,11 +481,11 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
 
   // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection
   // (bf16 output where the tensor-core attention consumes it).
-  if (h->use_tc)
-    MTLA_TRY((gemm<float, T, bf16>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
-                                   h->at<bf16>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
-                                   pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
-  else
+  if (h->use_tc) {
+    GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.qt), 1, (long long)dm.nh * dm.W, dm.r, B, dm.dh, pa.q_scale);
+    g.c_sz = dm.W; g.a_col_z = dm.dh; g.b_col_z = dm.dh; g.b_lo_col = hd;
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wk, h->map_q16, g, bn, dm.nh, true, st));
+  } else
     MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
                                     h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
                                     pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
@@ -389,11 +529,21 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   CombineArgs ca;
   ca.o_part = aa.o_part; ca.ml_part = aa.ml_part; ca.o = h->at<void>(p.o);
   ca.n_heads = dm.nh; ca.r = dm.r; ca.n_split = aa.n_split;
-  decode_combine_kernel<float><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
+  if (h->use_tc) decode_combine_kernel<bf16><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
+  else decode_combine_kernel<float><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
 
   // a8: v_h = o_h W_{V,h} per head, then y = concat_h(v_h) W_O.
+  if (h->use_tc) {
+    GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.v), 1, 2 * hd, dm.dh, B, dm.r, 1.f);
+    g.c_sz = dm.dh; g.a_row_z = dm.dh; g.b_col_z = dm.r; g.b_lo_col = dm.nh * dm.r; g.c_lo_off = hd;
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wvt, h->map_o16, g, bn, dm.nh, true, st));
+    g = gemm_tc_args(y, 1, dm.d, dm.d, B, hd, 1.f);
+    g.b_lo_col = hd;
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, h->map_v16, g, bn, 1, true, st));
+    return MTLA_OK;
+  }
   MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r,
                                   h->at<float>(p.v), B, dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f,
                                   dm.nh, dm.r, (long long)dm.dh * dm.r, dm.dh, st)));
@@ -410,8 +560,18 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   const int rows = B * T_len;
   const float q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
 
-  MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot,
-                              dm.d, dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  if (h->use_tc) {
+    // Weights on the MMA's M side, 128 prompt rows per CTA on its N side: neighbouring CTAs
+    // share an activation panel while the (small) weight matrix stays in L2.
+    CUtensorMap map_x;
+    MTLA_TRY(make_map_2d(&map_x, x, rows, dm.d, dm.d, kPrefillBn));
+    MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x,
+                            gemm_tc_args(h->at<float>(p.pf_p1), 1, dm.ntot, dm.ntot, rows, dm.d, 1.f),
+                            kPrefillBn, 1, false, st));
+  } else {
+    MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot,
+                                dm.d, dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+  }
   PrefillPostArgs pa;
   pa.p1 = h->at<float>(p.pf_p1);
   pa.proj = dm.proj;
@@ -438,29 +598,47 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   if (!y) return MTLA_OK;
 
   // Eq. 9-10 on the running-state sequence: keys and values of every column.
-  MTLA_TRY((gemm<T, T, float>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<float>(p.pf_kv),
-                              rows, 2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
+  if (h->use_tc) {
+    CUtensorMap map_c;
+    MTLA_TRY(make_map_2d(&map_c, h->at<void>(p.pf_cprime), rows, dm.r, dm.r, kPrefillBn));
+    MTLA_TRY(gemm_tc<float>(h, h->map_wkvt, map_c,
+                            gemm_tc_args(h->at<float>(p.pf_kv), 1, 2 * hd, 2 * hd, rows, dm.r, 1.f),
+                            kPrefillBn, 1, false, st));
+  } else {
+    MTLA_TRY((gemm<T, T, float>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<float>(p.pf_kv),
+                                rows, 2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
+  }
   PrefillAttnArgs aa;
   aa.qcat = pa.qcat; aa.kv = h->at<void>(p.pf_kv); aa.kr = pa.kr; aa.out = h->at<void>(p.pf_attn);
   aa.n_heads = dm.nh; aa.dr = dm.dr; aa.stride = dm.s; aa.T = T_len;
   const size_t smem = prefill_attn_fma_smem_bytes(dm.dh, dm.dr);
   dim3 grid(ceil_div(T_len, kPfTile), dm.nh, B);
-  if (dm.dh == 64) {
-    if (!h->pf_smem_ready)
-      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, 64>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    prefill_attn_fma_kernel<float, 64><<<grid, 256, smem, st>>>(aa);
+#define MTLA_PF_ATTN(TOUT, DH)                                                               \
+  do {                                                                                       \
+    if (!h->pf_smem_ready)                                                                   \
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, TOUT, DH>,               \
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+    prefill_attn_fma_kernel<float, TOUT, DH><<<grid, 256, smem, st>>>(aa);                   \
+  } while (0)
+  if (h->use_tc) {
+    if (dm.dh == 64) MTLA_PF_ATTN(bf16, 64); else MTLA_PF_ATTN(bf16, 128);
   } else {
-    if (!h->pf_smem_ready)
-      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, 128>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    prefill_attn_fma_kernel<float, 128><<<grid, 256, smem, st>>>(aa);
+    if (dm.dh == 64) MTLA_PF_ATTN(float, 64); else MTLA_PF_ATTN(float, 128);
   }
+#undef MTLA_PF_ATTN
   h->pf_smem_ready = true;
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
-  MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd,
-                              hd, dm.d, 1.f, 1, 0, 0, 0, st)));
+  if (h->use_tc) {
+    CUtensorMap map_a;
+    MTLA_TRY(make_map_2d(&map_a, h->at<void>(p.pf_attn), rows, 2 * hd, 2 * hd, kPrefillBn));
+    GemmTcArgs g = gemm_tc_args(y, 1, dm.d, dm.d, rows, hd, 1.f);
+    g.b_lo_col = hd;
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, map_a, g, kPrefillBn, 1, false, st));
+  } else {
+    MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd,
+                                hd, dm.d, 1.f, 1, 0, 0, 0, st)));
+  }
   return MTLA_OK;
 }
 
@@ -508,6 +686,8 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   h->tokens = 0; h->batch = 0; h->launches = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
+  h->act_bn = 0;
+  h->gemm_attr_mask = 0;
   // The tensor-core attention needs bf16 and whole 128-column latent blocks; the
   // MTLA_ATTENTION=fma environment override keeps the CUDA-core kernel for comparisons.
   const char* force = getenv("MTLA_ATTENTION");

@@ -138,7 +138,8 @@ struct PrefillAttnArgs {
   const void* qcat;   // [B*T][n_h][d_h + d_R], pre-scaled by log2(e)/sqrt(d_h)
   const void* kv;     // [B*T][2*n_h*d_h]: keys then values up-projected from cprime (Eq. 9-10)
   const void* kr;     // [B*T][d_R]
-  void* out;          // [B*T][n_h*d_h] per-head attention outputs (input of W_O)
+  void* out;          // [B*T][n_h*d_h] per-head attention outputs (input of W_O); bf16 rows
+                      // are [2][n_h*d_h]: hi halves, then the rounding remainders
   int n_heads, dr, stride, T;
 };
 
@@ -155,8 +156,8 @@ inline size_t prefill_attn_fma_smem_bytes(int dh, int dr) {
 // j*s + s - 1, plus its own running state at column m: exactly the columns the
 // stride-aware mask of Section 4.2 admits.  The mask is a predicate on (m, j).
 // Grid (ceil(T/64), n_h, B), 256 threads as 16 x 16, each owning a 4 x 4 score patch.
-// TQ = element type of queries, keys, values, RoPE keys and outputs.
-template <typename TQ, int DH>
+// TQ = element type of queries, keys, values and RoPE keys; TOut = element type of the outputs.
+template <typename TQ, typename TOut, int DH>
 __global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a) {
   extern __shared__ float smem[];
   constexpr int BT = kPfTile, V = Elem<TQ>::kVec, OC = DH / 16;
@@ -294,16 +295,22 @@ __global__ void __launch_bounds__(256) prefill_attn_fma_kernel(PrefillAttnArgs a
     }
   }
 
-  TQ* out = static_cast<TQ*>(a.out);
+  TOut* out = static_cast<TOut*>(a.out);
+  constexpr bool kSplit = sizeof(TOut) == 2;
+  const long long hdw = (long long)a.n_heads * DH;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int row = q0 + ty * 4 + i;
     if (row >= a.T) continue;
     const float inv = 1.f / l_run[i];
+    TOut* orow = out + (base + row) * (kSplit ? 2 : 1) * hdw + h * DH + tx * OC;
 #pragma unroll
-    for (int c = 0; c < OC; ++c)
-      out[(base + row) * a.n_heads * DH + h * DH + tx * OC + c] =
-          Elem<TQ>::from_float(o[i][c] * inv);
+    for (int c = 0; c < OC; ++c) {
+      const float val = o[i][c] * inv;
+      const TOut hi = Elem<TOut>::from_float(val);
+      orow[c] = hi;
+      if (kSplit) orow[hdw + c] = Elem<TOut>::from_float(val - Elem<TOut>::to_float(hi));
+    }
   }
 }
 
