@@ -45,6 +45,8 @@ struct GemmTcArgs {
   int m_tiles, n_tiles;       // tiles along A / B rows: gridDim.x = m_tiles * n_tiles * n_split,
                               // A tiles fastest (neighbouring CTAs share the B panel)
   int vec_ok;                 // 1: c, c_sm, c_sz keep 16-byte alignment for the row-major path
+  int vec4_ok;                // 1: c_sm == 1, m % 4 == 0 and every column start is 16-byte aligned,
+                              // so the split-K reduction may store four rows at once
   float alpha;
   float* partial;             // [tiles][n_split][BN][128] fp32 (split-K only)
   int* tickets;               // [tiles][4], zero between launches (split-K only)
@@ -101,6 +103,22 @@ __device__ __forceinline__ void store_row32<bf16>(bf16* p, const uint32_t (&v)[3
       }
       *reinterpret_cast<uint4*>(p + j) = make_uint4(w[0], w[1], w[2], w[3]);
     }
+}
+
+// Stores four consecutive outputs (and, for bf16 with lo_off > 0, their rounding remainders).
+__device__ __forceinline__ void store4(float* p, const float (&v)[4], long long) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store4(bf16* p, const float (&v)[4], long long lo_off) {
+  const __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&h0),
+                                            *reinterpret_cast<const uint32_t*>(&h1));
+  if (lo_off > 0) {
+    const __nv_bfloat162 l0 = __floats2bfloat162_rn(v[0] - __low2float(h0), v[1] - __high2float(h0));
+    const __nv_bfloat162 l1 = __floats2bfloat162_rn(v[2] - __low2float(h1), v[3] - __high2float(h1));
+    *reinterpret_cast<uint2*>(p + lo_off) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0),
+                                                       *reinterpret_cast<const uint32_t*>(&l1));
+  }
 }
 
 }  // namespace gtc
@@ -251,18 +269,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
           __threadfence();
-          const float* all = g.partial + tile * g.n_split * (long long)(BN * kBM);
+          // This warp sums its 32-row quarter over the splits, in split order.  Lane l owns
+          // rows 4*(l%8)..+3 of column (l/8) in each group of four columns, so every load is
+          // a 16-byte vector and a warp instruction covers 512 contiguous bytes; several
+          // column groups and splits are in flight per thread to cover the L2 latency.
+          const float* all = g.partial + tile * g.n_split * (long long)(BN * kBM) + q * 32;
+          const int r4 = 4 * (lane & 7), cs = lane >> 3;
+          constexpr int U = BN >= 16 ? 4 : 1;          // column groups per step (BN / 4 >= U)
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += CH) {
-            uint32_t v[32];
+          for (int jb = 0; jb < BN; jb += 4 * U) {
+            float4 acc[U];
 #pragma unroll
-            for (int j = 0; j < CH; ++j) {
-              float sum = 0.f;
-              for (int sp = 0; sp < g.n_split; ++sp)
-                sum += __ldcg(all + (long long)sp * (BN * kBM) + (c0 + j) * kBM + row_local);
-              v[j] = __float_as_uint(sum);
+            for (int u = 0; u < U; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+            for (int sp0 = 0; sp0 < g.n_split; sp0 += 4) {
+              float4 t[4][U];
+#pragma unroll
+              for (int s4 = 0; s4 < 4; ++s4)
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                  t[s4][u] = sp0 + s4 < g.n_split
+                                 ? __ldcg(reinterpret_cast<const float4*>(
+                                       all + (long long)(sp0 + s4) * (BN * kBM) +
+                                       (jb + u * 4 + cs) * kBM + r4))
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int s4 = 0; s4 < 4; ++s4)
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                  acc[u].x += t[s4][u].x; acc[u].y += t[s4][u].y;
+                  acc[u].z += t[s4][u].z; acc[u].w += t[s4][u].w;
+                }
             }
-            emit(v, c0);
+            const int i0 = mt * kBM + q * 32 + r4;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              const int j = nt * BN + jb + u * 4 + cs;
+              if (j >= g.n || i0 >= g.m) continue;
+              const float val[4] = {g.alpha * acc[u].x, g.alpha * acc[u].y, g.alpha * acc[u].z,
+                                    g.alpha * acc[u].w};
+              OutT* p = c + (long long)j * g.c_sn + (long long)i0 * g.c_sm;
+              if (g.vec4_ok) {
+                store4(p, val, g.c_lo_off);
+              } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (i0 + e < g.m) put(p + (long long)e * g.c_sm, val[e]);
+              }
+            }
           }
         }
       }

@@ -289,6 +289,8 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   g.vec_ok = (reinterpret_cast<uintptr_t>(g.c) % 16 == 0) && (g.c_sm * osz % 16 == 0) &&
              (g.c_sz * osz % 16 == 0);
   if ((long long)m_tiles * g.n_tiles * g.n_split > 0x7fffffffll) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  g.vec4_ok = g.c_sm == 1 && g.m % 4 == 0 && reinterpret_cast<uintptr_t>(g.c) % 16 == 0 &&
+              g.c_sn * osz % 16 == 0 && g.c_sz * osz % 16 == 0 && g.c_lo_off * osz % 8 == 0;
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
   switch (bn) {
