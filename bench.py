@@ -279,7 +279,7 @@ def main() -> None:
 
     w = pick_workload(args)
     K, W = args.steps, max(args.warmup, 3)
-    M, h = build_layer(w, extra_steps=2 * (K + W), device=device)
+    M, h = build_layer(w, extra_steps=3 * (K + W), device=device)
     extras = fill_context(M, h, w, device)
     dt = synth.torch_dtype(w.dtype)
     xs = [synth.decode_input(w, i).to(device) for i in range(8)]
@@ -300,11 +300,20 @@ def main() -> None:
         ev1.record()
         barrier()
     local_ms = ev0.elapsed_time(ev1)
-    attn_ms, attn_steps = M.mtla_profile_end(h)
+    stage_ms, attn_steps = M.mtla_profile_end_stages(h)
+    attn_ms = stage_ms["attention"]
     launches = M.mtla_launch_count(h) - launches0
     slots_end = M.mtla_position(h)[1]
     M.mtla_check(h)
     value, ms = replicas.throughput(w.batch * K, local_ms, device)
+    # The same K steps once more without the per-kernel events, to show what they cost.
+    torch.cuda.synchronize(device)
+    ev0.record()
+    for i in range(K):
+        M.mtla_decode_step(h, xs[i % 8], y)
+    ev1.record()
+    torch.cuda.synchronize(device)
+    plain_ms = ev0.elapsed_time(ev1)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     xh = [synth.decode_input(w, i).pin_memory() for i in range(8)]
@@ -371,6 +380,8 @@ def main() -> None:
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": w.batch * w.d_model * (2 if w.dtype == "bf16" else 4),
                 "d2h_bytes_per_step": w.batch * w.d_model * (2 if w.dtype == "bf16" else 4)},
+        "ms_per_step_without_stage_events": plain_ms / K,
+        "stage_us": {k: v * 1e3 / max(attn_steps, 1) for k, v in stage_ms.items()},
         "gpu_launches": int(launches),
         "clocks": clocks.summary(),
     }

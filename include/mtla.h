@@ -144,13 +144,18 @@ int mtla_check(mtla_handle* h, void* stream);
 /* Number of kernels the library has launched on behalf of this handle since creation. */
 int64_t mtla_launch_count(const mtla_handle* h);
 
-/* Kernel timing for benchmarks.  After mtla_profile_begin, each of the next max_steps
- * decode steps records a CUDA event pair on its stream around the decode-attention kernel
- * (step a7, the kernel that streams the cache).  mtla_profile_end waits for those events,
- * returns their summed duration in milliseconds and the number of steps covered, and
- * releases the events. */
+/* Kernel timing for benchmarks.  After mtla_profile_begin, each of the next max_steps decode
+ * steps records CUDA events on its stream between its kernels, in the order of Section 4.1:
+ * stage 0 input projections (Eq. 7, Eq. 8, RoPE projections), 1 LayerNorm + gate (Eq. 13) + slot
+ * update + RoPE, 2 query absorption (Eq. 12), 3 attention over the cache (Eq. 17; the kernel
+ * that streams the cache), 4 cross-split combine, 5 value up-projection (Eq. 10), 6 output
+ * projection (Eq. 11).  mtla_profile_end_stages waits for those events, returns the summed
+ * duration of every stage in milliseconds (stage_ms host [MTLA_DECODE_STAGES]) and the number
+ * of steps covered, and releases the events; mtla_profile_end returns the attention stage only. */
+enum { MTLA_DECODE_STAGES = 7, MTLA_STAGE_ATTENTION = 3 };
 int mtla_profile_begin(mtla_handle* h, int32_t max_steps);
 int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps);
+int mtla_profile_end_stages(mtla_handle* h, double* stage_ms, int32_t* steps);
 
 /* Name of the decode-attention kernel variant the handle dispatches to ("fma" or "tcgen05"). */
 const char* mtla_attention_variant(const mtla_handle* h);

@@ -26,7 +26,11 @@ EXPORTED_SYMBOLS = (
     "mtla_arena_bytes", "mtla_create", "mtla_prefill", "mtla_decode_step",
     "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
     "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
-    "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end")
+    "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
+    "mtla_profile_end_stages")
+
+DECODE_STAGES = ("input_proj", "norm_gate_update", "absorb", "attention", "combine", "value_proj",
+                 "output_proj")
 
 
 class MTLAError(RuntimeError):
@@ -77,6 +81,8 @@ def load_library() -> ctypes.CDLL:
         "mtla_profile_begin": (ctypes.c_int, [vp, i32]),
         "mtla_profile_end": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(i32)]),
+        "mtla_profile_end_stages": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
+                                                   ctypes.POINTER(i32)]),
         "mtla_error_string": (ctypes.c_char_p, [ctypes.c_int]),
     }
     for name, (res, args) in sigs.items():
@@ -262,3 +268,11 @@ def mtla_profile_end(h: Handle) -> tuple[float, int]:
     _check(load_library().mtla_profile_end(h.ptr, ctypes.byref(ms), ctypes.byref(steps)),
            "mtla_profile_end")
     return ms.value, steps.value
+
+
+def mtla_profile_end_stages(h: Handle) -> tuple[dict, int]:
+    """({stage name: summed milliseconds}, steps covered) for the decode step's kernels."""
+    ms, steps = (ctypes.c_double * len(DECODE_STAGES))(), ctypes.c_int32()
+    _check(load_library().mtla_profile_end_stages(h.ptr, ms, ctypes.byref(steps)),
+           "mtla_profile_end_stages")
+    return dict(zip(DECODE_STAGES, list(ms))), steps.value

@@ -1,28 +1,51 @@
 // Tensor-core (tcgen05 / TMEM / TMA) split-K decode attention over the compressed cache in
-// the absorbed form (Eq. 12 / Eq. 17), bf16 operands, fp32 accumulation.
+// the absorbed form (Eq. 12 / Eq. 17), bf16 operands, fp32 accumulation, with the
+// cross-split combine fused in.
 //
-// Work unit: one CTA per (split, sequence) streams its slot range in tiles of 128 slots.
-// A tile is brought in by TMA as 64-column sub-tiles [128 slots x 128 B] with the 128-byte
+// Work is cut into tiles of 64 slots.  The B * ceil(n_slots / 64) tiles of a step form one
+// list (sequence-major) that is dealt out in equal contiguous shares to one persistent CTA per
+// SM, so a CTA's share may end one sequence and start the next ("segments").  Each segment
+// yields a partial (reference maximum, denominator, un-normalised output) and the CTA that
+// delivers a sequence's last partial combines them (an atomic ticket, never a wait).
+//
+// A tile is brought in by TMA as 64-column sub-tiles [64 slots x 128 B] with the 128-byte
 // swizzle; the SAME shared-memory bytes feed both contractions, so every cache byte is read
 // from HBM exactly once per step:
-//   scores  S^T[128 slots x heads]  = tile[128 x (r+d_R)] . q~^T      A = tile, K-major
-//   values  O^T[r x heads]         += tile[:, :r]^T . P^T[128 x heads] A = tile, MN-major
-// Heads sit in the MMA's N dimension (16 or 32), slots / latent columns in M = 128, so no
-// padding of heads up to M is paid for.  Accumulators live in TMEM: two score buffers and
-// r/128 output blocks.  Warp roles: warp 0 = TMA producer (one thread), warp 1 = MMA issuer
-// (one thread) and TMEM owner, warps 4-7 = softmax (one thread per slot of the tile).
+//   scores  S^T[64 slots x heads]  = tile[64 x (r+d_R)] . q~^T        A = tile, K-major, M = 64
+//   values  O^T[r x heads]        += tile[:, :r]^T . P^T[64 x heads]  A = tile, MN-major, M = 128
+// Heads sit in the MMA's N dimension (16 or 32), so no padding of heads up to M is paid for.
+// Accumulators live in TMEM: two score buffers and r/128 output blocks.  With M = 64 the score
+// of slot i sits in TMEM lane 32*(i/16) + i%16, i.e. in the first 16 lanes of each warp's
+// quarter, so lanes 0-15 of each softmax warp own one slot each.
 //
-// Shared memory: a ring of five 32 KB "pairs" (two adjacent 64-column sub-tiles = one
-// 128-row MN-major operand block) + one 16 KB sub-tile for the RoPE-key columns + q~ as the
-// K-major B operand + the bf16 probabilities P.  A tile needs r/128 pairs; with r = 512 the
-// fifth pair lets the next tile's first loads overlap this tile's softmax and value MMAs.
+// An MMA that accumulates into the tile a previous MMA wrote cannot start before that one has
+// drained, and with N this small the drain latency dwarfs the arithmetic.  So consecutive MMAs
+// never share an accumulator: a score buffer is four partial accumulators (k-step ks of every
+// 64-column chunk goes to partial ks; the softmax threads add the four), and the value MMAs
+// rotate over the r/128 output blocks.
 //
-// The online softmax rescales lazily: the reference maximum of a head is only raised when a
-// tile exceeds it by more than 2^8, so the TMEM read-modify-write of O is rare.  Results are
-// exact either way because the same reference enters numerator and denominator.
+// Shared memory: a ring of nine 16 KB "pairs" (two adjacent sub-tiles = a 128-row MN-major
+// operand block), three 8 KB sub-tiles for the RoPE-key columns, q~ as a K-major swizzled B
+// operand (TMA-loaded per segment), and two bf16 probability buffers.  The ring holds more
+// than two tiles, and the MMA warp issues whichever of "score the next tile" / "accumulate the
+// tile whose probabilities are ready" can go, so loads stay in flight through every phase.
 //
-// Every wait is bounded (see sm100_ptx.cuh); on a timeout the CTA raises its abort word, all
-// roles unwind, and the host sees MTLA_ERR_DEVICE_TIMEOUT from mtla_check.
+// The online softmax raises a head's reference maximum only when a tile exceeds it by more
+// than 2^8: the common tile needs one barrier-with-OR and no cross-thread reduction, and the
+// TMEM read-modify-write of O is rare.  Results are exact either way because the same
+// reference enters numerator and denominator.
+//
+// One thread can issue a tcgen05.mma only about every hundred cycles, far slower than these
+// small-N MMAs execute, so issue is spread over six single-thread issuers in six warps: four
+// for the scores (issuer k owns partial accumulator k) and two for the values (output blocks
+// of even / odd index).  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
+// warps 5-6 = value issuers, warp 7 idle, warps 8-11 = softmax and epilogue.  The first two
+// warpgroups give most of their registers to the third (setmaxnreg).
+//
+// Every mbarrier wait is bounded (see sm100_ptx.cuh); on a timeout the CTA raises its abort
+// word, all roles unwind, and the host sees MTLA_ERR_DEVICE_TIMEOUT from mtla_check.  The
+// named barrier among the softmax warps is reached by all of them in every iteration, and
+// carries the abort state in its OR.
 #pragma once
 
 #include <math.h>
@@ -33,43 +56,52 @@
 namespace mtla {
 
 struct AttnTcArgs {
-  const bf16* qt;      // [B][n_h][r + d_R] bf16, pre-scaled by log2(e)/sqrt(d_h)
-  float* o_part;       // [B * n_split][n_h][r]
-  float* ml_part;      // [B * n_split][n_h][2]
+  float* o_part;       // [B + grid][n_h][r] un-normalised partial outputs
+  float* ml_part;      // [B + grid][n_h][2]: reference maximum (log2 units), denominator
+  bf16* o16;           // [B][2][n_h][r]: combined output as bf16 hi halves, then remainders
+  int* tickets;        // [B], zero between launches
   int* error_word;
-  int n_heads, r, dr, n_slots, slots_per_split, n_split;
+  int n_heads, r, dr, n_slots, batch;
+  int tiles_per_seq;   // ceil(n_slots / 64)
 };
 
 namespace tc {
 
-constexpr int kTile = 128;            // slots per tile
-constexpr int kSubBytes = 128 * 128;  // one 64-column sub-tile
+constexpr int kTile = 64;                  // slots per tile
+constexpr int kThreads = 384;
+constexpr int kQkIssuers = 4, kPvIssuers = 2;
+constexpr int kSubBytes = kTile * 128;     // one 64-column sub-tile
 constexpr int kPairBytes = 2 * kSubBytes;
-constexpr int kPairs = 5;
-constexpr int kTmemCols = 256;
-constexpr int kColS = 0;              // two score buffers at columns 0 and 32
-constexpr int kColO = 64;             // output blocks at 64 + 32 * block
+constexpr int kPairs = 9;
+constexpr int kKrBufs = 3;
+constexpr int kTmemCols = 512;
+constexpr int kSParts = 4;                 // independent partial score accumulators per buffer
+constexpr int kColS = 0;                   // score buffer b, partial k at column (b * 4 + k) * 32
+constexpr int kColO = 2 * kSParts * 32;    // output blocks at 256 + 32 * block
 constexpr float kRescaleThreshold = 8.f;
 
 constexpr int kOffPairs = 0;
 constexpr int kOffKr = kPairs * kPairBytes;
-constexpr int kOffQ = kOffKr + kSubBytes;
-constexpr int kMaxQBytes = 32 * 576 * 2;
+constexpr int kOffQ = kOffKr + kKrBufs * kSubBytes;
+constexpr int kMaxQBytes = 9 * 32 * 128;   // (2 * 4 + 1) chunks x 32 heads x 128 B
 constexpr int kOffP = kOffQ + kMaxQBytes;
-constexpr int kPBytes = 32 * kTile * 2;
-constexpr int kOffMisc = kOffP + kPBytes;
-constexpr int kMiscBytes = 2048;
+constexpr int kPBytes = 32 * kTile * 2;    // one probability buffer
+constexpr int kOffMisc = kOffP + 2 * kPBytes;
+constexpr int kMiscBytes = 3072;
 constexpr int kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + slack for 1024-byte alignment
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 struct Misc {
   unsigned long long full_pair[kPairs], empty_pair[kPairs];
-  unsigned long long full_kr, empty_kr, s_full[2], s_empty[2], p_full, pv_done, group_sync;
+  unsigned long long full_kr[kKrBufs], empty_kr[kKrBufs];
+  unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], q_full, q_empty;
   uint32_t tmem_base;
   int abort_word;
-  int flag[2];
+  int last_flag;
   float wmax[4][32];
-  float cand_m[32], fac[32], m_cur[32];
+  float m_new[32], fac[32];
   float lsum[4][32];
+  float comb_w[8][32];     // combine: weight of part p for head h (first 8 parts cached)
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
 
@@ -90,18 +122,29 @@ __device__ __forceinline__ float transposed_reduce(float (&v)[32], int lane, Op 
   return v[0];
 }
 
+// Share of the tile list owned by CTA c of G: [c * total / G, (c + 1) * total / G).
+__host__ __device__ inline long long share_begin(long long c, long long total, long long G) {
+  return c * total / G;
+}
+// The CTA whose share contains tile g.
+__host__ __device__ inline long long share_owner(long long g, long long total, long long G) {
+  return ((g + 1) * G - 1) / total;
+}
+
 }  // namespace tc
 
 // NHP: heads padded to the MMA's N (16 or 32).  RP: r / 128 (pairs per tile).
 template <int NHP, int RP>
-__global__ void __launch_bounds__(256, 1)
-decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map, AttnTcArgs a) {
+__global__ void __launch_bounds__(tc::kThreads, 1)
+decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
+                      const __grid_constant__ CUtensorMap q_map, AttnTcArgs a) {
   using namespace tc;
   using namespace ptx;
-  constexpr int WP = (2 * RP + 1) * 64;          // q~ width padded to whole 64-column chunks
-  constexpr uint32_t SBOQ = (WP / 8) * 128;      // bytes between 8-head groups of q~
-  constexpr uint32_t IDESC_QK = make_idesc_bf16(128, NHP, 0, 0);
+  constexpr int NCH = 2 * RP + 1;                // 64-column chunks of q~ (latent + RoPE)
+  constexpr uint32_t QCHUNK = NHP * 128;         // bytes of one q~ chunk
+  constexpr uint32_t IDESC_QK = make_idesc_bf16(64, NHP, 0, 0);
   constexpr uint32_t IDESC_PV = make_idesc_bf16(128, NHP, 1, 0);
+  constexpr uint32_t PSBO = (kTile / 8) * 128;   // bytes between 8-head groups of P^T
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -118,20 +161,23 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map, AttnTcArgs 
       mbar_init(bar(&misc->full_pair[i]), 1);
       mbar_init(bar(&misc->empty_pair[i]), 1);
     }
-    mbar_init(bar(&misc->full_kr), 1);
-    mbar_init(bar(&misc->empty_kr), 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(&misc->s_full[i]), 1);
-      mbar_init(bar(&misc->s_empty[i]), 128);
+    for (int i = 0; i < kKrBufs; ++i) {
+      mbar_init(bar(&misc->full_kr[i]), 1);
+      mbar_init(bar(&misc->empty_kr[i]), kQkIssuers);
     }
-    mbar_init(bar(&misc->p_full), 128);
-    mbar_init(bar(&misc->pv_done), 1);
-    mbar_init(bar(&misc->group_sync), 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(&misc->s_full[i]), kQkIssuers);
+      mbar_init(bar(&misc->s_empty[i]), 128);
+      mbar_init(bar(&misc->p_full[i]), 128);
+      mbar_init(bar(&misc->p_empty[i]), kPvIssuers);
+    }
+    mbar_init(bar(&misc->q_full), 1);
+    mbar_init(bar(&misc->q_empty), kQkIssuers);
     misc->abort_word = 0;
-    misc->flag[0] = 0;
-    misc->flag[1] = 0;
+    misc->last_flag = 0;
     mbar_fence_init();
     prefetch_tensormap(&cache_map);
+    prefetch_tensormap(&q_map);
   }
   if (warp == 1) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
   tc_fence_before_sync();
@@ -139,44 +185,43 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map, AttnTcArgs 
   tc_fence_after_sync();
   const uint32_t tmem_base = misc->tmem_base;
 
-  const int b = blockIdx.y, split = blockIdx.x;
-  const int slot0 = split * a.slots_per_split;
-  const int slot1 = min(a.n_slots, slot0 + a.slots_per_split);
-  const int n_tiles = (slot1 - slot0 + kTile - 1) / kTile;
-  const long long unit = (long long)b * a.n_split + split;
-  const int W = a.r + a.dr;
-
-  // q~ as the K-major, un-swizzled B operand: 8 x 16-byte core matrices, K-adjacent cores
-  // 128 B apart, 8-head groups SBOQ apart.  Heads >= n_h and columns >= r + d_R are zero.
-  {
-    const bf16* q = a.qt + (long long)b * a.n_heads * W;
-    for (int v = threadIdx.x; v < NHP * (WP / 8); v += 256) {
-      const int n = v / (WP / 8), kc = v % (WP / 8);
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (n < a.n_heads && kc * 8 < W) val = *reinterpret_cast<const uint4*>(q + n * W + kc * 8);
-      *reinterpret_cast<uint4*>(sm + kOffQ + (n >> 3) * SBOQ + kc * 128 + (n & 7) * 16) = val;
-    }
-    if (threadIdx.x >= 128 && threadIdx.x < 160) misc->m_cur[threadIdx.x - 128] = -INFINITY;
-  }
-  fence_proxy_async_smem();
-  __syncthreads();
+  // This CTA's share of the tile list.
+  const long long tps = a.tiles_per_seq, total = (long long)a.batch * tps, G = gridDim.x;
+  const long long g0 = share_begin(blockIdx.x, total, G), g1 = share_begin(blockIdx.x + 1, total, G);
+  const int n_tiles = (int)(g1 - g0);
 
   const uint32_t pairs_u32 = base + kOffPairs, kr_u32 = base + kOffKr;
   const uint32_t q_u32 = base + kOffQ, p_u32 = base + kOffP;
 
+  if (warp < 8) {
+  // Register budget: the producer / issuer warpgroups keep 56 registers, the softmax one gets 240.
+  reg_dealloc<56>();
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
-    int pc = 0;
-    for (int t = 0; t < n_tiles && ok; ++t) {
-      const int slot = slot0 + t * kTile;
-      ok = mbar_wait(bar(&misc->empty_kr), (t & 1) ^ 1, abort_word, a.error_word, 1);
+    int pc = 0, seg = 0;
+    for (int n = 0; n < n_tiles && ok; ++n) {
+      const long long g = g0 + n;
+      const int b = (int)(g / tps), t = (int)(g - (long long)b * tps);
+      if (n == 0 || t == 0) {
+        // A segment starts: q~ of sequence b, once the previous segment's score MMAs are done.
+        ok = mbar_wait(bar(&misc->q_empty), (seg & 1) ^ 1, abort_word, a.error_word, 1);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar(&misc->q_full), NCH * QCHUNK);
+        for (int ch = 0; ch < NCH; ++ch)
+          tma_load_3d(q_u32 + ch * QCHUNK, &q_map, bar(&misc->q_full), ch * 64, 0, b);
+        ++seg;
+      }
+      const int slot = t * kTile;
+      const int kb = n % kKrBufs;
+      ok = mbar_wait(bar(&misc->empty_kr[kb]), ((n / kKrBufs) & 1) ^ 1, abort_word, a.error_word, 2);
       if (!ok) break;
-      mbar_arrive_expect_tx(bar(&misc->full_kr), kSubBytes);
-      tma_load_3d(kr_u32, &cache_map, bar(&misc->full_kr), a.r, slot, b);
+      mbar_arrive_expect_tx(bar(&misc->full_kr[kb]), kSubBytes);
+      tma_load_3d(kr_u32 + kb * kSubBytes, &cache_map, bar(&misc->full_kr[kb]), a.r, slot, b);
       for (int c = 0; c < RP && ok; ++c, ++pc) {
-        const int buf = pc % kPairs, use = pc / kPairs;
-        ok = mbar_wait(bar(&misc->empty_pair[buf]), (use & 1) ^ 1, abort_word, a.error_word, 2);
+        const int buf = pc % kPairs;
+        ok = mbar_wait(bar(&misc->empty_pair[buf]), ((pc / kPairs) & 1) ^ 1, abort_word,
+                       a.error_word, 3);
         if (!ok) break;
         const uint32_t dst = pairs_u32 + buf * kPairBytes;
         mbar_arrive_expect_tx(bar(&misc->full_pair[buf]), kPairBytes);
@@ -184,122 +229,175 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map, AttnTcArgs 
         tma_load_3d(dst + kSubBytes, &cache_map, bar(&misc->full_pair[buf]), c * 128 + 64, slot, b);
       }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp >= 1 && warp <= kQkIssuers && lane == 0) {
+    // ------------------------------------------------------------------ score issuer k
+    // Issuer k multiplies k-step k (16 columns) of every 64-column chunk into partial k.
+    const int k = warp - 1;
     bool ok = true;
-    // Score MMAs of one 64-column chunk held at `a_smem`; chunk index selects q~'s columns.
-    auto qk_chunk = [&](uint32_t a_smem, int chunk, uint32_t d_tmem, bool first) {
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
-        const uint64_t ad = make_smem_desc(a_smem + ks * 32, 16, 1024, kSwizzle128B);
-        const uint64_t bd = make_smem_desc(q_u32 + (chunk * 8 + ks * 2) * 128, 128, SBOQ, kSwizzleNone);
-        mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, (first && ks == 0) ? 0u : 1u);
-      }
-    };
-    // Score phase for tile t, pairs [c_begin, c_end); the RoPE-key chunk goes first.
-    auto qk_phase = [&](int t, int c_begin, int c_end) {
-      const uint32_t d_tmem = tmem_base + kColS + (t & 1) * 32;
-      if (c_begin == 0) {
-        ok = mbar_wait(bar(&misc->s_empty[t & 1]), ((t >> 1) & 1) ^ 1, abort_word, a.error_word, 3);
-        if (!ok) return;
-        ok = mbar_wait(bar(&misc->full_kr), t & 1, abort_word, a.error_word, 4);
-        if (!ok) return;
-        tc_fence_after_sync();
-        qk_chunk(kr_u32, 2 * RP, d_tmem, true);
-        mma_commit(bar(&misc->empty_kr));
-      }
-      for (int c = c_begin; c < c_end; ++c) {
-        const int pcn = t * RP + c, buf = pcn % kPairs, use = pcn / kPairs;
-        ok = mbar_wait(bar(&misc->full_pair[buf]), use & 1, abort_word, a.error_word, 5);
-        if (!ok) return;
-        const uint32_t src = pairs_u32 + buf * kPairBytes;
-        qk_chunk(src, 2 * c, d_tmem, false);
-        qk_chunk(src + kSubBytes, 2 * c + 1, d_tmem, false);
-      }
-      if (c_end == RP) mma_commit(bar(&misc->s_full[t & 1]));
-    };
-    qk_phase(0, 0, RP);
-    for (int t = 0; t < n_tiles && ok; ++t) {
-      if (t + 1 < n_tiles) {
-        qk_phase(t + 1, 0, 1);   // the spare pair: overlaps this tile's softmax
+    int seg = 0;
+    for (int n = 0; n < n_tiles && ok; ++n) {
+      const long long g = g0 + n;
+      const int t = (int)(g % tps);
+      const uint32_t d_tmem = tmem_base + kColS + (n & 1) * (kSParts * 32) + k * 32;
+      auto qk = [&](uint32_t a_smem, int chunk, uint32_t accumulate) {
+        const uint64_t ad = make_smem_desc(a_smem + k * 32, 16, 1024, kSwizzle128B);
+        const uint64_t bd = make_smem_desc(q_u32 + chunk * QCHUNK + k * 32, 16, 1024, kSwizzle128B);
+        mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, accumulate);
+      };
+      if (n == 0 || t == 0) {
+        ok = mbar_wait(bar(&misc->q_full), seg & 1, abort_word, a.error_word, 4);
         if (!ok) break;
+        ++seg;
       }
-      ok = mbar_wait(bar(&misc->p_full), t & 1, abort_word, a.error_word, 6);
+      const int kb = n % kKrBufs;
+      ok = mbar_wait(bar(&misc->s_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 9) &&
+           mbar_wait(bar(&misc->full_kr[kb]), (n / kKrBufs) & 1, abort_word, a.error_word, 10);
       if (!ok) break;
       tc_fence_after_sync();
-      for (int mb = 0; mb < RP; ++mb) {
-        const int pcn = t * RP + mb, buf = pcn % kPairs;
+      qk(kr_u32 + kb * kSubBytes, 2 * RP, 0u);
+      mma_commit(bar(&misc->empty_kr[kb]));
+      for (int c = 0; c < RP && ok; ++c) {
+        const int pcn = n * RP + c, buf = pcn % kPairs;
+        ok = mbar_wait(bar(&misc->full_pair[buf]), (pcn / kPairs) & 1, abort_word, a.error_word, 11);
+        if (!ok) break;
+        tc_fence_after_sync();
         const uint32_t src = pairs_u32 + buf * kPairBytes;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t ad = make_smem_desc(src + ks * 2048, kSubBytes, 1024, kSwizzle128B);
-          const uint64_t bd = make_smem_desc(p_u32 + ks * 256, 128, 2048, kSwizzleNone);
-          mma_bf16_ss(tmem_base + kColO + mb * 32, ad, bd, IDESC_PV, (t == 0 && ks == 0) ? 0u : 1u);
-        }
-        mma_commit(bar(&misc->empty_pair[buf]));
+        qk(src, 2 * c, 1u);
+        qk(src + kSubBytes, 2 * c + 1, 1u);
       }
-      mma_commit(bar(&misc->pv_done));
-      if (RP > 1 && t + 1 < n_tiles) qk_phase(t + 1, 1, RP);
+      if (!ok) break;
+      mma_commit(bar(&misc->s_full[n & 1]));
+      if (n + 1 == n_tiles || t + 1 == tps) mma_commit(bar(&misc->q_empty));   // segment's last tile
     }
-  } else if (warp >= 4) {
-    // ------------------------------------------------------------------ softmax warps
-    const int q = warp - 4, row = q * 32 + lane, sidx = threadIdx.x - 128;
+  } else if (warp > kQkIssuers && warp <= kQkIssuers + kPvIssuers && lane == 0) {
+    // ------------------------------------------------------------------ value issuer j
+    // Issuer j accumulates the output blocks mb = j, j + 2, ... once a tile's probabilities
+    // are published, and hands the pairs it read back to the producer.
+    const int j = warp - 1 - kQkIssuers;
+    bool ok = true;
+    for (int n = 0; n < n_tiles && ok; ++n) {
+      ok = mbar_wait(bar(&misc->p_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 12);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const long long g = g0 + n;
+      const bool seg_first = n == 0 || (g % tps) == 0;
+#pragma unroll
+      for (int ks = 0; ks < kTile / 16; ++ks) {
+        const uint64_t bd = make_smem_desc(p_u32 + (n & 1) * kPBytes + ks * 256, 128, PSBO, kSwizzleNone);
+        for (int mb = j; mb < RP; mb += kPvIssuers) {
+          const uint32_t src = pairs_u32 + ((n * RP + mb) % kPairs) * kPairBytes;
+          const uint64_t ad = make_smem_desc(src + ks * 2048, kSubBytes, 1024, kSwizzle128B);
+          mma_bf16_ss(tmem_base + kColO + mb * 32, ad, bd, IDESC_PV, (seg_first && ks == 0) ? 0u : 1u);
+        }
+      }
+      for (int mb = j; mb < RP; mb += kPvIssuers) mma_commit(bar(&misc->empty_pair[(n * RP + mb) % kPairs]));
+      mma_commit(bar(&misc->p_empty[n & 1]));
+    }
+  }
+  } else {
+    // ------------------------------------------------------------------ softmax / epilogue warps
+    reg_alloc<240>();
+    const int q = warp & 3, sidx = q * 32 + lane;          // TMEM quarter; index among the 128
+    const bool active = lane < 16;                          // lanes that own a slot (M = 64 layout)
+    const int row = q * 16 + lane;                          // slot within the tile (active lanes)
     const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
     bool ok = true;
-    // Rendezvous of the 128 softmax threads on an mbarrier, so that it is bounded like
-    // every other wait (a plain named barrier could not give up).
-    int sync_phase = 0;
-    auto group_sync = [&]() {
-      mbar_arrive(bar(&misc->group_sync));
-      ok = mbar_wait(bar(&misc->group_sync), sync_phase & 1, abort_word, a.error_word, 10);
-      ++sync_phase;
-      return ok;
-    };
     float m_used[32], l_acc[32];
 #pragma unroll
     for (int h = 0; h < 32; ++h) {
       m_used[h] = -INFINITY;
       l_acc[h] = 0.f;
     }
-    for (int t = 0; t < n_tiles && ok; ++t) {
-      ok = mbar_wait(bar(&misc->s_full[t & 1]), (t >> 1) & 1, abort_word, a.error_word, 7);
-      if (!ok) break;
-      tc_fence_after_sync();
-      uint32_t sv[32];
-      if (NHP == 32) tmem_ld_x32(lane_base + kColS + (t & 1) * 32, sv);
-      else tmem_ld_x16(lane_base + kColS + (t & 1) * 32, sv);
-      tmem_wait_ld();
-      tc_fence_before_sync();
-      mbar_arrive(bar(&misc->s_empty[t & 1]));
-
-      const bool valid = slot0 + t * kTile + row < slot1;
-      float s[32], red[32];
-#pragma unroll
-      for (int h = 0; h < 32; ++h) {
-        s[h] = (valid && h < NHP) ? __uint_as_float(sv[h]) : -INFINITY;
-        red[h] = s[h];
-      }
-      misc->wmax[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return fmaxf(x, y); });
-      if (!group_sync()) break;
-      if (sidx < 32) {
-        const float mt = fmaxf(fmaxf(misc->wmax[0][sidx], misc->wmax[1][sidx]),
-                               fmaxf(misc->wmax[2][sidx], misc->wmax[3][sidx]));
-        const float m_old = misc->m_cur[sidx];
-        const float m_new = fmaxf(m_old, mt);
-        misc->cand_m[sidx] = m_new;
-        misc->fac[sidx] = (m_new == -INFINITY) ? 1.f : exp2f(m_old - m_new);
-        if (mt > m_old + kRescaleThreshold) misc->flag[t & 1] = 1;
-        if (sidx == 0) misc->flag[(t + 1) & 1] = 0;
-      }
-      if (!group_sync()) break;
-      const bool rescale = misc->flag[t & 1] != 0;
-      if (rescale) {
+    for (int n = 0; n < n_tiles; ++n) {
+      const long long g = g0 + n;
+      const int b = (int)(g / tps), t = (int)(g - (long long)b * tps);
+      const bool seg_first = n == 0 || t == 0;
+      const bool seg_last = n + 1 == n_tiles || t + 1 == (int)tps;
+      if (seg_first) {
 #pragma unroll
         for (int h = 0; h < 32; ++h) {
-          m_used[h] = misc->cand_m[h];
+          m_used[h] = -INFINITY;
+          l_acc[h] = 0.f;
+        }
+      }
+      float s[32];
+#pragma unroll
+      for (int h = 0; h < 32; ++h) s[h] = 0.f;
+      if (ok) ok = mbar_wait(bar(&misc->s_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 5);
+      ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are whole-warp operations
+      if (ok) {
+        tc_fence_after_sync();
+        const uint32_t s_addr = lane_base + kColS + (n & 1) * (kSParts * 32);
+#pragma unroll
+        for (int k2 = 0; k2 < kSParts; k2 += 2) {   // the score is the sum of the partials
+          uint32_t sa[32], sb[32];
+          if (NHP == 32) {
+            tmem_ld_x32(s_addr + k2 * 32, sa);
+            tmem_ld_x32(s_addr + (k2 + 1) * 32, sb);
+          } else {
+            tmem_ld_x16(s_addr + k2 * 32, sa);
+            tmem_ld_x16(s_addr + (k2 + 1) * 32, sb);
+          }
+          tmem_wait_ld();
+#pragma unroll
+          for (int h = 0; h < NHP; ++h) s[h] += __uint_as_float(sa[h]) + __uint_as_float(sb[h]);
+        }
+        tc_fence_before_sync();
+        mbar_arrive(bar(&misc->s_empty[n & 1]));
+      }
+      const bool valid = ok && active && t * kTile + row < a.n_slots;
+      bool exceed = false;
+#pragma unroll
+      for (int h = 0; h < 32; ++h) {
+        s[h] = (valid && h < NHP) ? s[h] : -INFINITY;
+        exceed |= s[h] > m_used[h] + kRescaleThreshold;
+      }
+      // One barrier tells everyone whether any head must raise its reference (or the CTA gave up).
+      if (named_barrier1_or_128(exceed || !ok || *abort_word)) {
+        if (named_barrier1_or_128(!ok || *abort_word)) break;   // collective result: all leave together
+        float red[32];
+#pragma unroll
+        for (int h = 0; h < 32; ++h) red[h] = s[h];
+        misc->wmax[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return fmaxf(x, y); });
+        named_barrier_sync(1, 128);
+        if (sidx < 32) {
+          const float mt = fmaxf(fmaxf(misc->wmax[0][sidx], misc->wmax[1][sidx]),
+                                 fmaxf(misc->wmax[2][sidx], misc->wmax[3][sidx]));
+          // Each thread's m_used[sidx] is the CTA-wide value: all threads apply the same updates.
+          float m_old = -INFINITY;
+#pragma unroll
+          for (int h = 0; h < 32; ++h) m_old = (h == sidx) ? m_used[h] : m_old;
+          const bool raise = mt > m_old + kRescaleThreshold;
+          const float m_nw = raise ? mt : m_old;
+          misc->m_new[sidx] = m_nw;
+          misc->fac[sidx] = (m_nw == m_old) ? 1.f : exp2f(m_old - m_nw);   // 0 from -inf
+        }
+        named_barrier_sync(1, 128);
+#pragma unroll
+        for (int h = 0; h < 32; ++h) {
+          m_used[h] = misc->m_new[h];
           l_acc[h] *= misc->fac[h];
         }
-        if (sidx < 32) misc->m_cur[sidx] = misc->cand_m[sidx];
+        if (!seg_first) {
+          // O holds contributions scaled to the old references: wait for the previous tile's
+          // value MMAs, then rescale the accumulator columns in TMEM.
+          ok = mbar_wait(bar(&misc->p_empty[(n - 1) & 1]), ((n - 1) >> 1) & 1, abort_word,
+                         a.error_word, 6);
+          ok = __all_sync(0xffffffffu, ok);
+          if (ok) {
+            tc_fence_after_sync();
+            for (int mb = 0; mb < RP; ++mb) {
+              uint32_t ov[32];
+              const uint32_t addr = lane_base + kColO + mb * 32;
+              if (NHP == 32) tmem_ld_x32(addr, ov); else tmem_ld_x16(addr, ov);
+              tmem_wait_ld();
+#pragma unroll
+              for (int h = 0; h < NHP; ++h) ov[h] = __float_as_uint(__uint_as_float(ov[h]) * misc->fac[h]);
+              if (NHP == 32) tmem_st_x32(addr, ov); else tmem_st_x16(addr, ov);
+            }
+            tmem_wait_st();
+          }
+        }
       }
       uint32_t pb[16];
 #pragma unroll
@@ -310,58 +408,118 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map, AttnTcArgs 
         l_acc[h + 1] += __high2float(pk);
         pb[h / 2] = *reinterpret_cast<const uint32_t*>(&pk);
       }
-      if (t > 0) {
-        ok = mbar_wait(bar(&misc->pv_done), (t - 1) & 1, abort_word, a.error_word, 8);
-        if (!ok) break;
-        tc_fence_after_sync();
-        if (rescale) {
-          for (int mb = 0; mb < RP; ++mb) {
-            uint32_t ov[32];
-            const uint32_t addr = lane_base + kColO + mb * 32;
-            if (NHP == 32) tmem_ld_x32(addr, ov); else tmem_ld_x16(addr, ov);
-            tmem_wait_ld();
+      // The probability buffer is free once the value MMAs of tile n - 2 have completed.
+      if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 7);
+      if (ok) {
+        if (active) {
+          // P^T as the K-major, un-swizzled B operand of the value MMA: element (head h, slot k)
+          // at (h/8)*PSBO + (k/8)*128 + (h%8)*16 + (k%8)*2.
+          uint8_t* prow = sm + kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
 #pragma unroll
-            for (int h = 0; h < NHP; ++h) ov[h] = __float_as_uint(__uint_as_float(ov[h]) * misc->fac[h]);
-            if (NHP == 32) tmem_st_x32(addr, ov); else tmem_st_x16(addr, ov);
+          for (int h = 0; h < NHP; ++h) {
+            const uint16_t bits = (h & 1) ? (uint16_t)(pb[h / 2] >> 16) : (uint16_t)(pb[h / 2] & 0xffffu);
+            *reinterpret_cast<uint16_t*>(prow + (h >> 3) * PSBO + (h & 7) * 16) = bits;
           }
-          tmem_wait_st();
         }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(bar(&misc->p_full[n & 1]));
       }
-      // P^T as the K-major, un-swizzled B operand of the value MMA: element (head n, slot k)
-      // at (n/8)*2048 + (k/8)*128 + (n%8)*16 + (k%8)*2.
-      uint8_t* prow = sm + kOffP + (row >> 3) * 128 + (row & 7) * 2;
+
+      if (!seg_last) continue;
+      // ---------------------------------------------------------------- end of a segment
+      // Partial of sequence b: wait for the last value MMAs, read O^T from TMEM.
+      const long long part = blockIdx.x + b;      // unique per (CTA, sequence), increasing
+      if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 8);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after_sync();
+        float* o_part = a.o_part + part * a.n_heads * a.r;
+        for (int mb = 0; mb < RP; ++mb) {
+          uint32_t ov[32];
+          const uint32_t addr = lane_base + kColO + mb * 32;
+          if (NHP == 32) tmem_ld_x32(addr, ov); else tmem_ld_x16(addr, ov);
+          tmem_wait_ld();
 #pragma unroll
-      for (int h = 0; h < NHP; ++h) {
-        const uint16_t bits = (h & 1) ? (uint16_t)(pb[h / 2] >> 16) : (uint16_t)(pb[h / 2] & 0xffffu);
-        *reinterpret_cast<uint16_t*>(prow + (h >> 3) * 2048 + (h & 7) * 16) = bits;
+          for (int h = 0; h < NHP; ++h)
+            if (h < a.n_heads) o_part[h * a.r + mb * 128 + sidx] = __uint_as_float(ov[h]);
+        }
+        tc_fence_before_sync();
       }
-      fence_proxy_async_smem();
-      tc_fence_before_sync();
-      mbar_arrive(bar(&misc->p_full));
-    }
-    if (ok && n_tiles > 0) {
-      ok = mbar_wait(bar(&misc->pv_done), (n_tiles - 1) & 1, abort_word, a.error_word, 9);
-    }
-    if (ok && n_tiles > 0) {
-      tc_fence_after_sync();
-      float* o_part = a.o_part + unit * a.n_heads * a.r;
-      for (int mb = 0; mb < RP; ++mb) {
-        uint32_t ov[32];
-        const uint32_t addr = lane_base + kColO + mb * 32;
-        if (NHP == 32) tmem_ld_x32(addr, ov); else tmem_ld_x16(addr, ov);
-        tmem_wait_ld();
+      float red[32];
 #pragma unroll
-        for (int h = 0; h < NHP; ++h)
-          if (h < a.n_heads) o_part[h * a.r + mb * 128 + row] = __uint_as_float(ov[h]);
+      for (int h = 0; h < 32; ++h) red[h] = l_acc[h];
+      misc->lsum[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return x + y; });
+      __threadfence();
+      if (named_barrier1_or_128(!ok || *abort_word)) break;   // collective result
+      if (sidx < a.n_heads) {
+        float m_mine = -INFINITY;
+#pragma unroll
+        for (int h = 0; h < 32; ++h) m_mine = (h == sidx) ? m_used[h] : m_mine;
+        a.ml_part[(part * a.n_heads + sidx) * 2] = m_mine;
+        a.ml_part[(part * a.n_heads + sidx) * 2 + 1] =
+            misc->lsum[0][sidx] + misc->lsum[1][sidx] + misc->lsum[2][sidx] + misc->lsum[3][sidx];
+        __threadfence();
       }
-      misc->lsum[q][lane] = transposed_reduce(l_acc, lane, [](float x, float y) { return x + y; });
-      if (group_sync() && sidx < a.n_heads) {
-        const float l = misc->lsum[0][sidx] + misc->lsum[1][sidx] + misc->lsum[2][sidx] +
-                        misc->lsum[3][sidx];
-        a.ml_part[(unit * a.n_heads + sidx) * 2] = misc->m_cur[sidx];
-        a.ml_part[(unit * a.n_heads + sidx) * 2 + 1] = l;
+      // Ticket: the CTA that delivers the sequence's last partial combines them.
+      const long long c_first = share_owner((long long)b * tps, total, G);
+      const int n_parts = (int)(share_owner((long long)(b + 1) * tps - 1, total, G) - c_first) + 1;
+      named_barrier_sync(1, 128);
+      if (sidx == 0) {
+        const int old = atomicAdd(a.tickets + b, 1);
+        const int last = old == n_parts - 1;
+        if (last) a.tickets[b] = 0;
+        misc->last_flag = last;
       }
-      tc_fence_before_sync();
+      named_barrier_sync(1, 128);
+      if (misc->last_flag) {
+        __threadfence();
+        const long long part0 = c_first + b;
+        // Per head: global reference, each part's weight 2^(m_p - m) and the denominator.
+        if (sidx < a.n_heads) {
+          float m = -INFINITY;
+          for (int pt = 0; pt < n_parts; ++pt)
+            m = fmaxf(m, __ldcg(a.ml_part + ((part0 + pt) * a.n_heads + sidx) * 2));
+          float denom = 0.f;
+          for (int pt = 0; pt < n_parts; ++pt) {
+            const float* ml = a.ml_part + ((part0 + pt) * a.n_heads + sidx) * 2;
+            const float wgt = exp2f(__ldcg(ml) - m);
+            denom += wgt * __ldcg(ml + 1);
+            if (pt < 8) misc->comb_w[pt][sidx] = wgt;
+          }
+          misc->fac[sidx] = 1.f / denom;
+          misc->m_new[sidx] = m;
+        }
+        named_barrier_sync(1, 128);
+        // Thread sidx owns latent columns 4*sidx .. 4*sidx+3 (r/4 <= 128 threads are busy).
+        if (4 * sidx < a.r) {
+          bf16* o_hi = a.o16 + (long long)b * 2 * a.n_heads * a.r + 4 * sidx;
+          bf16* o_lo = o_hi + (long long)a.n_heads * a.r;
+          for (int h = 0; h < a.n_heads; ++h) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int pt = 0; pt < n_parts; ++pt) {
+              const float wgt = pt < 8 ? misc->comb_w[pt][h]
+                                       : exp2f(__ldcg(a.ml_part + ((part0 + pt) * a.n_heads + h) * 2) -
+                                               misc->m_new[h]);
+              const float4 v = __ldcg(reinterpret_cast<const float4*>(
+                  a.o_part + ((part0 + pt) * a.n_heads + h) * a.r + 4 * sidx));
+              acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
+              acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+            }
+            const float inv = misc->fac[h];
+            const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(val[0], val[1]);
+            const __nv_bfloat162 h1 = __floats2bfloat162_rn(val[2], val[3]);
+            const __nv_bfloat162 l0 = __floats2bfloat162_rn(val[0] - __low2float(h0), val[1] - __high2float(h0));
+            const __nv_bfloat162 l1 = __floats2bfloat162_rn(val[2] - __low2float(h1), val[3] - __high2float(h1));
+            *reinterpret_cast<uint2*>(o_hi + (long long)h * a.r) =
+                make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+            *reinterpret_cast<uint2*>(o_lo + (long long)h * a.r) =
+                make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+          }
+        }
+        named_barrier_sync(1, 128);   // comb_w / fac are reused by the next segment
+      }
     }
   }
 

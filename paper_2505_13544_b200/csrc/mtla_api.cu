@@ -38,7 +38,7 @@ struct ArenaPlan {
   size_t wcat_t, w_k, w_kv_t, w_o_t;
   size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
   size_t cache, open_acc, err_flag;
-  size_t p1, q16, qt, o_part, ml_part, o, v, x_stage, y_stage, gemm_part, gemm_tickets;
+  size_t p1, q16, qt, o_part, ml_part, o, v, x_stage, y_stage, gemm_part, gemm_tickets, attn_tickets;
   size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
   size_t total;
 };
@@ -120,6 +120,7 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->gemm_part = take(c.dtype == MTLA_DTYPE_BF16
                           ? (size_t)kGemmSlots * gtc::kBM * act_box_rows(c.max_batch) * 4 : 0);
   p->gemm_tickets = take((size_t)kGemmSlots * 4 * sizeof(int));
+  p->attn_tickets = take(B * sizeof(int));
   const size_t rows = B * (size_t)c.max_prefill_tokens;
   p->pf_p1 = take(rows * dm.ntot * 4);
   p->pf_qcat = take(rows * dm.nh * (dm.dh + dm.dr) * 4);
@@ -145,14 +146,14 @@ struct mtla_handle {
   bool attn_smem_ready, pf_smem_ready;
   // Tensor-core decode attention (bf16, r a multiple of 128): TMA view of the cache.
   bool use_tc;
-  CUtensorMap cache_map;
+  CUtensorMap cache_map, q_map;
   // Tensor-core projections (bf16): weight panels as 128-row boxes, serving as the MMA's M side
   // in the decode step and as its N side in the prefill; decode activations as act_bn-row boxes.
   CUtensorMap map_wcat, map_wk, map_wkvt, map_wvt, map_wot;
   CUtensorMap map_q16, map_o16, map_v16;
   int act_bn;               // box rows the three activation maps were encoded with (0: none yet)
   unsigned gemm_attr_mask;  // kernel instances whose shared-memory limit has been raised
-  // Optional timing of the decode-attention kernel: one event pair per profiled step.
+  // Optional timing of the decode step's kernels: MTLA_DECODE_STAGES + 1 events per profiled step.
   std::vector<cudaEvent_t> prof_events;
   int prof_used;
 
@@ -217,20 +218,28 @@ EncodeTiledFn encode_tiled_fn() {
   return cached;
 }
 
-// TMA view of the bf16 cache [max_batch][max_slots][r + d_R]: boxes of 128 slots x 64
-// columns (128 bytes, the swizzle span), zero fill outside the tensor.
+// TMA views for the decode attention: the bf16 cache [max_batch][max_slots][r + d_R] in boxes of
+// 64 slots x 64 columns (128 bytes, the swizzle span), and the absorbed queries
+// [max_batch][n_h][r + d_R] in boxes of `heads_padded` heads x 64 columns; zero fill outside.
 int make_cache_map(mtla_handle* h) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return MTLA_ERR_CUDA;
   const Dims& dm = h->dm;
   const cuuint64_t dims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.max_slots, (cuuint64_t)h->cfg.max_batch};
   const cuuint64_t strides[2] = {(cuuint64_t)dm.W * 2, (cuuint64_t)dm.max_slots * dm.W * 2};
-  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t box[3] = {64, (cuuint32_t)tc::kTile, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult rc = fn(
+  CUresult rc = fn(
       &h->cache_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->at<void>(h->plan.cache), dims, strides,
       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) return MTLA_ERR_CUDA;
+  const cuuint64_t qdims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.nh, (cuuint64_t)h->cfg.max_batch};
+  const cuuint64_t qstrides[2] = {(cuuint64_t)dm.W * 2, (cuuint64_t)dm.nh * dm.W * 2};
+  const cuuint32_t qbox[3] = {64, (cuuint32_t)(dm.nh <= 16 ? 16 : 32), 1};
+  rc = fn(&h->q_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->at<void>(h->plan.qt), qdims, qstrides,
+          qbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
@@ -311,14 +320,14 @@ GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, i
 }
 
 template <int NHP>
-int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int B, cudaStream_t st) {
-  dim3 grid(a.n_split, B);
+int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_t st) {
 #define MTLA_TC_CASE(RP)                                                                       \
   case RP:                                                                                     \
     if (!h->attn_smem_ready)                                                                   \
       MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP>,                           \
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes)); \
-    decode_attn_tc_kernel<NHP, RP><<<grid, 256, tc::kSmemBytes, st>>>(h->cache_map, a);         \
+    decode_attn_tc_kernel<NHP, RP><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(h->cache_map,   \
+                                                                               h->q_map, a);   \
     break;
   switch (a.r / 128) {
     MTLA_TC_CASE(1)
@@ -375,6 +384,7 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.cache), 0,
                             (size_t)h->cfg.max_batch * dm.max_slots * dm.W * dm.elem, st));
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.gemm_tickets), 0, (size_t)kGemmSlots * 4 * sizeof(int), st));
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.attn_tickets), 0, (size_t)h->cfg.max_batch * sizeof(int), st));
   if (h->use_tc) {
     MTLA_TRY(make_cache_map(h));
     MTLA_TRY(make_map_2d(&h->map_wcat, h->at<void>(p.wcat_t), dm.ntot, dm.d, dm.d, gtc::kBM));
@@ -431,6 +441,13 @@ int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
   return launch_attn_fma_rpt<T, TQ, 32>(h, a, B, st);
 }
 
+// Records the event that closes stage `stage - 1` / opens stage `stage` of a profiled step.
+int prof_mark(mtla_handle* h, bool prof, int stage, cudaStream_t st) {
+  if (!prof) return MTLA_OK;
+  MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used + stage], st));
+  return MTLA_OK;
+}
+
 // The decode step (Section 4.1): a1 fused projection, a2-a5 post kernel, a6 absorption,
 // a7 split-K attention + combine, a8 value and output projections.
 template <typename T>
@@ -442,6 +459,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   const int slot = i0 / dm.s;
   const int n_slots = slot + 1;
 
+  const bool prof = h->prof_used + MTLA_DECODE_STAGES + 1 <= (int)h->prof_events.size();
+  MTLA_TRY(prof_mark(h, prof, 0, st));
   const int bn = act_box_rows(B);
   if (h->use_tc) {
     // a1 on the tensor cores: weights stream through the MMA's M side, the batch sits in N.
@@ -456,6 +475,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
                                 dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
   }
 
+  MTLA_TRY(prof_mark(h, prof, 1, st));
   PostArgs pa;
   pa.p1 = h->at<float>(p.p1);
   pa.proj = dm.proj;
@@ -481,6 +501,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
 
+  MTLA_TRY(prof_mark(h, prof, 2, st));
   // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection
   // (bf16 output where the tensor-core attention consumes it).
   if (h->use_tc) {
@@ -492,6 +513,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
                                     h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
                                     pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
 
+  MTLA_TRY(prof_mark(h, prof, 3, st));
   AttnArgs aa;
   aa.qt = h->at<void>(p.qt);
   aa.cache = h->at<void>(p.cache);
@@ -499,58 +521,60 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   aa.ml_part = h->at<float>(p.ml_part);
   aa.n_heads = dm.nh; aa.r = dm.r; aa.dr = dm.dr; aa.max_slots = dm.max_slots;
   aa.n_slots = n_slots;
-  const bool prof = h->prof_used + 2 <= (int)h->prof_events.size();
   if (h->use_tc) {
-    // One CTA per SM: as many splits per sequence as keep B * n_split within the SM count.
-    int n_split = min(max(1, kSmCount / B), ceil_div(n_slots, tc::kTile));
-    aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), tc::kTile) * tc::kTile;
-    aa.n_split = ceil_div(n_slots, aa.slots_per_split);
+    // One persistent CTA per SM; the step's 64-slot tiles are dealt out in equal shares, and
+    // the kernel combines the partials itself (no separate combine launch).
     AttnTcArgs ta;
-    ta.qt = h->at<bf16>(p.qt);
     ta.o_part = aa.o_part; ta.ml_part = aa.ml_part;
+    ta.o16 = h->at<bf16>(p.o);
+    ta.tickets = h->at<int>(p.attn_tickets);
     ta.error_word = h->at<int>(p.err_flag);
-    ta.n_heads = dm.nh; ta.r = dm.r; ta.dr = dm.dr; ta.n_slots = n_slots;
-    ta.slots_per_split = aa.slots_per_split; ta.n_split = aa.n_split;
-    if (prof) MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used], st));
-    if (dm.nh <= 16) MTLA_TRY(launch_attn_tc_rp<16>(h, ta, B, st));
-    else MTLA_TRY(launch_attn_tc_rp<32>(h, ta, B, st));
+    ta.n_heads = dm.nh; ta.r = dm.r; ta.dr = dm.dr; ta.n_slots = n_slots; ta.batch = B;
+    ta.tiles_per_seq = ceil_div(n_slots, tc::kTile);
+    const long long total = (long long)B * ta.tiles_per_seq;
+    const int grid = (int)(total < kSmCount ? total : kSmCount);
+    aa.n_split = 0;
+    if (dm.nh <= 16) MTLA_TRY(launch_attn_tc_rp<16>(h, ta, grid, st));
+    else MTLA_TRY(launch_attn_tc_rp<32>(h, ta, grid, st));
   } else {
     int want = ceil_div(kTargetCtas, B);
     int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
     if (n_split < 1) n_split = 1;
     aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
     aa.n_split = ceil_div(n_slots, aa.slots_per_split);
-    if (prof) MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used], st));
     MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st)));
   }
-  if (prof) {
-    MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used + 1], st));
-    h->prof_used += 2;
-  }
+  MTLA_TRY(prof_mark(h, prof, 4, st));
 
   CombineArgs ca;
   ca.o_part = aa.o_part; ca.ml_part = aa.ml_part; ca.o = h->at<void>(p.o);
   ca.n_heads = dm.nh; ca.r = dm.r; ca.n_split = aa.n_split;
-  if (h->use_tc) decode_combine_kernel<bf16><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
-  else decode_combine_kernel<float><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
-  h->launches++;
-  MTLA_CUDA(cudaGetLastError());
+  if (!h->use_tc) {
+    decode_combine_kernel<float><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
 
   // a8: v_h = o_h W_{V,h} per head, then y = concat_h(v_h) W_O.
+  MTLA_TRY(prof_mark(h, prof, 5, st));
   if (h->use_tc) {
     GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.v), 1, 2 * hd, dm.dh, B, dm.r, 1.f);
     g.c_sz = dm.dh; g.a_row_z = dm.dh; g.b_col_z = dm.r; g.b_lo_col = dm.nh * dm.r; g.c_lo_off = hd;
     MTLA_TRY(gemm_tc<bf16>(h, h->map_wvt, h->map_o16, g, bn, dm.nh, true, st));
+    MTLA_TRY(prof_mark(h, prof, 6, st));
     g = gemm_tc_args(y, 1, dm.d, dm.d, B, hd, 1.f);
     g.b_lo_col = hd;
     MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, h->map_v16, g, bn, 1, true, st));
-    return MTLA_OK;
+  } else {
+    MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r,
+                                    h->at<float>(p.v), B, dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f,
+                                    dm.nh, dm.r, (long long)dm.dh * dm.r, dm.dh, st)));
+    MTLA_TRY(prof_mark(h, prof, 6, st));
+    MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.v), h->at<T>(p.w_o_t), y, B, dm.d, hd, hd, hd,
+                                dm.d, 1.f, 1, 0, 0, 0, st)));
   }
-  MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r,
-                                  h->at<float>(p.v), B, dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f,
-                                  dm.nh, dm.r, (long long)dm.dh * dm.r, dm.dh, st)));
-  MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.v), h->at<T>(p.w_o_t), y, B, dm.d, hd, hd, hd,
-                              dm.d, 1.f, 1, 0, 0, 0, st)));
+  MTLA_TRY(prof_mark(h, prof, 7, st));
+  if (prof) h->prof_used += MTLA_DECODE_STAGES + 1;
   return MTLA_OK;
 }
 
@@ -830,7 +854,7 @@ int mtla_profile_begin(mtla_handle* h, int32_t max_steps) {
   for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
   h->prof_events.clear();
   h->prof_used = 0;
-  for (int i = 0; i < 2 * max_steps; ++i) {
+  for (int i = 0; i < (MTLA_DECODE_STAGES + 1) * max_steps; ++i) {
     cudaEvent_t e;
     MTLA_CUDA(cudaEventCreate(&e));
     h->prof_events.push_back(e);
@@ -838,21 +862,31 @@ int mtla_profile_begin(mtla_handle* h, int32_t max_steps) {
   return MTLA_OK;
 }
 
-int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps) {
-  if (!h || !attention_ms || !steps) return MTLA_ERR_INVALID_ARG;
-  double total = 0.0;
-  for (int i = 0; i + 1 < h->prof_used; i += 2) {
-    MTLA_CUDA(cudaEventSynchronize(h->prof_events[i + 1]));
-    float ms = 0.f;
-    MTLA_CUDA(cudaEventElapsedTime(&ms, h->prof_events[i], h->prof_events[i + 1]));
-    total += ms;
+int mtla_profile_end_stages(mtla_handle* h, double* stage_ms, int32_t* steps) {
+  if (!h || !stage_ms || !steps) return MTLA_ERR_INVALID_ARG;
+  constexpr int per_step = MTLA_DECODE_STAGES + 1;
+  for (int s = 0; s < MTLA_DECODE_STAGES; ++s) stage_ms[s] = 0.0;
+  for (int i = 0; i + per_step <= h->prof_used; i += per_step) {
+    MTLA_CUDA(cudaEventSynchronize(h->prof_events[i + MTLA_DECODE_STAGES]));
+    for (int s = 0; s < MTLA_DECODE_STAGES; ++s) {
+      float ms = 0.f;
+      MTLA_CUDA(cudaEventElapsedTime(&ms, h->prof_events[i + s], h->prof_events[i + s + 1]));
+      stage_ms[s] += ms;
+    }
   }
-  *attention_ms = total;
-  *steps = h->prof_used / 2;
+  *steps = h->prof_used / per_step;
   for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
   h->prof_events.clear();
   h->prof_used = 0;
   return MTLA_OK;
+}
+
+int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps) {
+  if (!attention_ms) return MTLA_ERR_INVALID_ARG;
+  double stage_ms[MTLA_DECODE_STAGES];
+  const int rc = mtla_profile_end_stages(h, stage_ms, steps);
+  if (rc == MTLA_OK) *attention_ms = stage_ms[MTLA_STAGE_ATTENTION];
+  return rc;
 }
 
 const char* mtla_attention_variant(const mtla_handle* h) {
