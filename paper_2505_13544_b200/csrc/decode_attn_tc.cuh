@@ -31,9 +31,13 @@
 // tile whose probabilities are ready" can go, so loads stay in flight through every phase.
 //
 // The online softmax raises a head's reference maximum only when a tile exceeds it by more
-// than 2^8: the common tile needs one barrier-with-OR and no cross-thread reduction, and the
-// TMEM read-modify-write of O is rare.  Results are exact either way because the same
-// reference enters numerator and denominator.
+// than 2^8.  The common tile therefore needs no cross-thread reduction: each thread compares
+// its scores with the shared references, raises a flag if one is outgrown, and forms its
+// probabilities at once; the flag is collected through a split mbarrier arrive / wait that
+// overlaps that work, and only a raised flag (always at a sequence's first tile, otherwise
+// rare) sends the 128 threads through the reduction, the TMEM rescale of O and a second
+// exponentiation.  Results are exact either way because the same reference enters numerator
+// and denominator.
 //
 // One thread can issue a tcgen05.mma only about every hundred cycles, far slower than these
 // small-N MMAs execute, so issue is spread over six single-thread issuers in six warps: four
@@ -42,10 +46,9 @@
 // warps 5-6 = value issuers, warp 7 idle, warps 8-11 = softmax and epilogue.  The first two
 // warpgroups give most of their registers to the third (setmaxnreg).
 //
-// Every mbarrier wait is bounded (see sm100_ptx.cuh); on a timeout the CTA raises its abort
-// word, all roles unwind, and the host sees MTLA_ERR_DEVICE_TIMEOUT from mtla_check.  The
-// named barrier among the softmax warps is reached by all of them in every iteration, and
-// carries the abort state in its OR.
+// Every wait is a bounded mbarrier wait (see sm100_ptx.cuh), the rendezvous of the softmax
+// threads included; on a timeout the CTA raises its abort word, all roles unwind, and the host
+// sees MTLA_ERR_DEVICE_TIMEOUT from mtla_check.
 #pragma once
 
 #include <math.h>
@@ -95,12 +98,16 @@ struct Misc {
   unsigned long long full_pair[kPairs], empty_pair[kPairs];
   unsigned long long full_kr[kKrBufs], empty_kr[kKrBufs];
   unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], q_full, q_empty;
+  unsigned long long flag_bar[2], group_sync;
   uint32_t tmem_base;
   int abort_word;
   int last_flag;
+  int exceed_flag[2];      // raised by any softmax thread whose tile outgrew a reference
+  float m_used[32];        // per-head reference maximum of the running segment (log2 units)
   float wmax[4][32];
-  float m_new[32], fac[32];
+  float fac[32];
   float lsum[4][32];
+  float comb_m[32];
   float comb_w[8][32];     // combine: weight of part p for head h (first 8 parts cached)
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
@@ -173,8 +180,13 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     }
     mbar_init(bar(&misc->q_full), 1);
     mbar_init(bar(&misc->q_empty), kQkIssuers);
+    mbar_init(bar(&misc->flag_bar[0]), 128);
+    mbar_init(bar(&misc->flag_bar[1]), 128);
+    mbar_init(bar(&misc->group_sync), 128);
     misc->abort_word = 0;
     misc->last_flag = 0;
+    misc->exceed_flag[0] = 0;
+    misc->exceed_flag[1] = 0;
     mbar_fence_init();
     prefetch_tensormap(&cache_map);
     prefetch_tensormap(&q_map);
@@ -200,9 +212,12 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
     int pc = 0, seg = 0;
-    for (int n = 0; n < n_tiles && ok; ++n) {
-      const long long g = g0 + n;
-      const int b = (int)(g / tps), t = (int)(g - (long long)b * tps);
+    int b = (int)(g0 / tps), t = (int)(g0 - (long long)b * tps);
+    for (int n = 0; n < n_tiles && ok; ++n, ++t) {
+      if (t == (int)tps) {
+        t = 0;
+        ++b;
+      }
       if (n == 0 || t == 0) {
         // A segment starts: q~ of sequence b, once the previous segment's score MMAs are done.
         ok = mbar_wait(bar(&misc->q_empty), (seg & 1) ^ 1, abort_word, a.error_word, 1);
@@ -235,9 +250,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     const int k = warp - 1;
     bool ok = true;
     int seg = 0;
-    for (int n = 0; n < n_tiles && ok; ++n) {
-      const long long g = g0 + n;
-      const int t = (int)(g % tps);
+    int t = (int)(g0 % tps);
+    for (int n = 0; n < n_tiles && ok; ++n, ++t) {
+      if (t == (int)tps) t = 0;
       const uint32_t d_tmem = tmem_base + kColS + (n & 1) * (kSParts * 32) + k * 32;
       auto qk = [&](uint32_t a_smem, int chunk, uint32_t accumulate) {
         const uint64_t ad = make_smem_desc(a_smem + k * 32, 16, 1024, kSwizzle128B);
@@ -275,12 +290,13 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     // are published, and hands the pairs it read back to the producer.
     const int j = warp - 1 - kQkIssuers;
     bool ok = true;
-    for (int n = 0; n < n_tiles && ok; ++n) {
+    int t = (int)(g0 % tps);
+    for (int n = 0; n < n_tiles && ok; ++n, ++t) {
+      if (t == (int)tps) t = 0;
       ok = mbar_wait(bar(&misc->p_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 12);
       if (!ok) break;
       tc_fence_after_sync();
-      const long long g = g0 + n;
-      const bool seg_first = n == 0 || (g % tps) == 0;
+      const bool seg_first = n == 0 || t == 0;
 #pragma unroll
       for (int ks = 0; ks < kTile / 16; ++ks) {
         const uint64_t bd = make_smem_desc(p_u32 + (n & 1) * kPBytes + ks * 256, 128, PSBO, kSwizzleNone);
@@ -302,23 +318,28 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     const int row = q * 16 + lane;                          // slot within the tile (active lanes)
     const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
     bool ok = true;
-    float m_used[32], l_acc[32];
-#pragma unroll
-    for (int h = 0; h < 32; ++h) {
-      m_used[h] = -INFINITY;
-      l_acc[h] = 0.f;
-    }
-    for (int n = 0; n < n_tiles; ++n) {
-      const long long g = g0 + n;
-      const int b = (int)(g / tps), t = (int)(g - (long long)b * tps);
+    // Rendezvous of the 128 threads on an mbarrier, so that it is bounded like every other wait.
+    int sync_phase = 0;
+    auto group_sync = [&]() {
+      mbar_arrive(bar(&misc->group_sync));
+      if (ok) ok = mbar_wait(bar(&misc->group_sync), sync_phase & 1, abort_word, a.error_word, 13);
+      ++sync_phase;
+    };
+    float l_acc[32];
+    int b = (int)(g0 / tps), t = (int)(g0 - (long long)b * tps);
+    for (int n = 0; n < n_tiles; ++n, ++t) {
+      if (t == (int)tps) {
+        t = 0;
+        ++b;
+      }
       const bool seg_first = n == 0 || t == 0;
       const bool seg_last = n + 1 == n_tiles || t + 1 == (int)tps;
       if (seg_first) {
+        // New sequence: empty references (shared by the 128 threads) and denominators.
+        if (sidx < 32) misc->m_used[sidx] = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < 32; ++h) {
-          m_used[h] = -INFINITY;
-          l_acc[h] = 0.f;
-        }
+        for (int h = 0; h < 32; ++h) l_acc[h] = 0.f;
+        group_sync();
       }
       float s[32];
 #pragma unroll
@@ -343,46 +364,76 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
           for (int h = 0; h < NHP; ++h) s[h] += __uint_as_float(sa[h]) + __uint_as_float(sb[h]);
         }
         tc_fence_before_sync();
-        mbar_arrive(bar(&misc->s_empty[n & 1]));
       }
       const bool valid = ok && active && t * kTile + row < a.n_slots;
+      float m_ref[32];
       bool exceed = false;
 #pragma unroll
-      for (int h = 0; h < 32; ++h) {
-        s[h] = (valid && h < NHP) ? s[h] : -INFINITY;
-        exceed |= s[h] > m_used[h] + kRescaleThreshold;
+      for (int h = 0; h < NHP; ++h) {
+        m_ref[h] = misc->m_used[h];
+        s[h] = valid ? s[h] : -INFINITY;
+        exceed |= s[h] > m_ref[h] + kRescaleThreshold;
       }
-      // One barrier tells everyone whether any head must raise its reference (or the CTA gave up).
-      if (named_barrier1_or_128(exceed || !ok || *abort_word)) {
-        if (named_barrier1_or_128(!ok || *abort_word)) break;   // collective result: all leave together
+      // Tell the others (rarely) that a reference must rise; the answer is collected further
+      // down, after the probabilities have been formed with the current references.
+      if (exceed) misc->exceed_flag[n & 1] = 1;
+      mbar_arrive(bar(&misc->flag_bar[n & 1]));
+      if (ok) mbar_arrive(bar(&misc->s_empty[n & 1]));
+
+      uint32_t pb[16];
+      auto probabilities = [&]() {
+#pragma unroll
+        for (int h = 0; h < NHP; h += 2) {
+          const __nv_bfloat162 pk = __floats2bfloat162_rn(ex2_approx(s[h] - m_ref[h]),
+                                                          ex2_approx(s[h + 1] - m_ref[h + 1]));
+          pb[h / 2] = *reinterpret_cast<const uint32_t*>(&pk);
+        }
+      };
+      // P^T as the K-major, un-swizzled B operand of the value MMA: element (head h, slot k)
+      // at (h/8)*PSBO + (k/8)*128 + (h%8)*16 + (k%8)*2.
+      auto store_probabilities = [&]() {
+        if (!active) return;
+        uint8_t* prow = sm + kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
+#pragma unroll
+        for (int h = 0; h < NHP; ++h) {
+          const uint16_t bits = (h & 1) ? (uint16_t)(pb[h / 2] >> 16) : (uint16_t)(pb[h / 2] & 0xffffu);
+          *reinterpret_cast<uint16_t*>(prow + (h >> 3) * PSBO + (h & 7) * 16) = bits;
+        }
+      };
+      probabilities();
+      // The probability buffer is free once the value MMAs of tile n - 2 have completed.
+      if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 7);
+      if (ok) store_probabilities();
+      if (ok) ok = mbar_wait(bar(&misc->flag_bar[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 14);
+      if (ok && misc->exceed_flag[n & 1]) {
+        // ---- rare: some head's scores rose more than 2^8 above its reference (always at
+        // a sequence's first tile).  Everybody takes this branch: the flag is read after all
+        // 128 arrivals.  New references, rescaled denominators and accumulators, new P.
         float red[32];
 #pragma unroll
-        for (int h = 0; h < 32; ++h) red[h] = s[h];
+        for (int h = 0; h < 32; ++h) red[h] = h < NHP ? s[h] : -INFINITY;
         misc->wmax[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return fmaxf(x, y); });
-        named_barrier_sync(1, 128);
+        group_sync();
+        if (sidx == 0) misc->exceed_flag[n & 1] = 0;
         if (sidx < 32) {
           const float mt = fmaxf(fmaxf(misc->wmax[0][sidx], misc->wmax[1][sidx]),
                                  fmaxf(misc->wmax[2][sidx], misc->wmax[3][sidx]));
-          // Each thread's m_used[sidx] is the CTA-wide value: all threads apply the same updates.
-          float m_old = -INFINITY;
-#pragma unroll
-          for (int h = 0; h < 32; ++h) m_old = (h == sidx) ? m_used[h] : m_old;
-          const bool raise = mt > m_old + kRescaleThreshold;
-          const float m_nw = raise ? mt : m_old;
-          misc->m_new[sidx] = m_nw;
+          const float m_old = misc->m_used[sidx];
+          const float m_nw = mt > m_old + kRescaleThreshold ? mt : m_old;
+          misc->m_used[sidx] = m_nw;
           misc->fac[sidx] = (m_nw == m_old) ? 1.f : exp2f(m_old - m_nw);   // 0 from -inf
         }
-        named_barrier_sync(1, 128);
+        group_sync();
 #pragma unroll
-        for (int h = 0; h < 32; ++h) {
-          m_used[h] = misc->m_new[h];
+        for (int h = 0; h < NHP; ++h) {
+          m_ref[h] = misc->m_used[h];
           l_acc[h] *= misc->fac[h];
         }
         if (!seg_first) {
           // O holds contributions scaled to the old references: wait for the previous tile's
           // value MMAs, then rescale the accumulator columns in TMEM.
-          ok = mbar_wait(bar(&misc->p_empty[(n - 1) & 1]), ((n - 1) >> 1) & 1, abort_word,
-                         a.error_word, 6);
+          if (ok) ok = mbar_wait(bar(&misc->p_empty[(n - 1) & 1]), ((n - 1) >> 1) & 1, abort_word,
+                                 a.error_word, 6);
           ok = __all_sync(0xffffffffu, ok);
           if (ok) {
             tc_fence_after_sync();
@@ -398,29 +449,17 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
             tmem_wait_st();
           }
         }
+        probabilities();
+        if (ok) store_probabilities();
+        group_sync();                         // fac / wmax may be rewritten by the next rare tile
       }
-      uint32_t pb[16];
 #pragma unroll
       for (int h = 0; h < NHP; h += 2) {
-        const float p0 = exp2f(s[h] - m_used[h]), p1 = exp2f(s[h + 1] - m_used[h + 1]);
-        const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+        const __nv_bfloat162 pk = *reinterpret_cast<const __nv_bfloat162*>(&pb[h / 2]);
         l_acc[h] += __low2float(pk);
         l_acc[h + 1] += __high2float(pk);
-        pb[h / 2] = *reinterpret_cast<const uint32_t*>(&pk);
       }
-      // The probability buffer is free once the value MMAs of tile n - 2 have completed.
-      if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 7);
       if (ok) {
-        if (active) {
-          // P^T as the K-major, un-swizzled B operand of the value MMA: element (head h, slot k)
-          // at (h/8)*PSBO + (k/8)*128 + (h%8)*16 + (k%8)*2.
-          uint8_t* prow = sm + kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
-#pragma unroll
-          for (int h = 0; h < NHP; ++h) {
-            const uint16_t bits = (h & 1) ? (uint16_t)(pb[h / 2] >> 16) : (uint16_t)(pb[h / 2] & 0xffffu);
-            *reinterpret_cast<uint16_t*>(prow + (h >> 3) * PSBO + (h & 7) * 16) = bits;
-          }
-        }
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(bar(&misc->p_full[n & 1]));
@@ -448,15 +487,12 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       }
       float red[32];
 #pragma unroll
-      for (int h = 0; h < 32; ++h) red[h] = l_acc[h];
+      for (int h = 0; h < 32; ++h) red[h] = h < NHP ? l_acc[h] : 0.f;
       misc->lsum[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return x + y; });
       __threadfence();
-      if (named_barrier1_or_128(!ok || *abort_word)) break;   // collective result
-      if (sidx < a.n_heads) {
-        float m_mine = -INFINITY;
-#pragma unroll
-        for (int h = 0; h < 32; ++h) m_mine = (h == sidx) ? m_used[h] : m_mine;
-        a.ml_part[(part * a.n_heads + sidx) * 2] = m_mine;
+      group_sync();
+      if (ok && sidx < a.n_heads) {
+        a.ml_part[(part * a.n_heads + sidx) * 2] = misc->m_used[sidx];
         a.ml_part[(part * a.n_heads + sidx) * 2 + 1] =
             misc->lsum[0][sidx] + misc->lsum[1][sidx] + misc->lsum[2][sidx] + misc->lsum[3][sidx];
         __threadfence();
@@ -464,15 +500,18 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       // Ticket: the CTA that delivers the sequence's last partial combines them.
       const long long c_first = share_owner((long long)b * tps, total, G);
       const int n_parts = (int)(share_owner((long long)(b + 1) * tps - 1, total, G) - c_first) + 1;
-      named_barrier_sync(1, 128);
+      group_sync();
       if (sidx == 0) {
-        const int old = atomicAdd(a.tickets + b, 1);
-        const int last = old == n_parts - 1;
-        if (last) a.tickets[b] = 0;
+        int last = 0;
+        if (ok) {
+          const int old = atomicAdd(a.tickets + b, 1);
+          last = old == n_parts - 1;
+          if (last) a.tickets[b] = 0;
+        }
         misc->last_flag = last;
       }
-      named_barrier_sync(1, 128);
-      if (misc->last_flag) {
+      group_sync();
+      if (ok && misc->last_flag) {
         __threadfence();
         const long long part0 = c_first + b;
         // Per head: global reference, each part's weight 2^(m_p - m) and the denominator.
@@ -488,11 +527,11 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
             if (pt < 8) misc->comb_w[pt][sidx] = wgt;
           }
           misc->fac[sidx] = 1.f / denom;
-          misc->m_new[sidx] = m;
+          misc->comb_m[sidx] = m;
         }
-        named_barrier_sync(1, 128);
+        group_sync();
         // Thread sidx owns latent columns 4*sidx .. 4*sidx+3 (r/4 <= 128 threads are busy).
-        if (4 * sidx < a.r) {
+        if (ok && 4 * sidx < a.r) {
           bf16* o_hi = a.o16 + (long long)b * 2 * a.n_heads * a.r + 4 * sidx;
           bf16* o_lo = o_hi + (long long)a.n_heads * a.r;
           for (int h = 0; h < a.n_heads; ++h) {
@@ -500,7 +539,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
             for (int pt = 0; pt < n_parts; ++pt) {
               const float wgt = pt < 8 ? misc->comb_w[pt][h]
                                        : exp2f(__ldcg(a.ml_part + ((part0 + pt) * a.n_heads + h) * 2) -
-                                               misc->m_new[h]);
+                                               misc->comb_m[h]);
               const float4 v = __ldcg(reinterpret_cast<const float4*>(
                   a.o_part + ((part0 + pt) * a.n_heads + h) * a.r + 4 * sidx));
               acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
@@ -518,7 +557,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
                 make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
           }
         }
-        named_barrier_sync(1, 128);   // comb_w / fac are reused by the next segment
+        group_sync();   // comb_w / fac are reused by the next segment
       }
     }
   }
