@@ -13,6 +13,7 @@ slowest rank's device time.  `--impl reference` times the CPU oracle instead.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import sys
@@ -344,11 +345,16 @@ def main() -> None:
     step_s = local_ms * 1e-3 / K
     hbm_time = (work["weight_bytes"] + work["cache_bytes"]) / (peaks["hbm_gbs"] * 1e9)
     tensor_time = (work["attn_flop"] + work["proj_flop"]) / (peaks["bf16_tflops_sustained"] * 1e12)
+    # DRAM traffic of the attention kernel from the committed ncu capture, scaled by the cache
+    # bytes of this launch; dropped once the kernel's source differs from the captured one.
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
         t = json.load(open(tpath)).get(M.mtla_attention_variant(h), {})
-        if t.get("dram_bytes_per_cache_byte") is not None:
+        csrc = os.path.join(ROOT, "paper_2505_13544_b200", "csrc")
+        sha = hashlib.sha256(open(os.path.join(csrc, "decode_attn_tc.cuh"), "rb").read()
+                             + open(os.path.join(csrc, "sm100_ptx.cuh"), "rb").read()).hexdigest()
+        if t.get("dram_bytes_per_cache_byte") is not None and t.get("kernel_source_sha256") == sha:
             traffic = t["dram_bytes_per_cache_byte"] * work["cache_bytes"]
 
     line = {
