@@ -41,7 +41,8 @@ typedef enum {
   MTLA_ERR_BATCH_MISMATCH = -5,   /* B differs from the batch the cache currently holds */
   MTLA_ERR_CUDA = -6,             /* a CUDA runtime call or launch failed */
   MTLA_ERR_STATE = -7,            /* call not valid in the handle's current state */
-  MTLA_ERR_DEVICE_TIMEOUT = -8    /* a bounded device-side wait gave up (reported by mtla_check) */
+  MTLA_ERR_DEVICE_TIMEOUT = -8,   /* a bounded device-side wait gave up (reported by mtla_check) */
+  MTLA_ERR_SCRATCH_LIMIT = -9     /* mtla_decode_step_static: split workspace exceeds the static array */
 } mtla_status;
 
 enum { MTLA_DTYPE_FP32 = 0, MTLA_DTYPE_BF16 = 1 };
@@ -113,6 +114,31 @@ int mtla_decode_step(mtla_handle* h, const void* x, int32_t B, void* y, void* st
  * y back to y_host [B][d], all enqueued on `stream` (pinned host memory keeps it async). */
 int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y_host,
                           void* stream);
+
+/* The same decode step as mtla_decode_step, for callers that must not depend on allocated
+ * scratch.  (The paper has no counterpart to this call; it exists for integration reasons only.)
+ * Who needs it: a host program that has handed all device memory to its own pool and sizes the
+ * arena to the byte, an embedding that runs under a "no allocation after start-up" rule, or a
+ * caller that wants to shrink the arena by leaving the attention split workspace out of it.  The
+ * attention kernel's scratch - the per-split partial outputs, their (maximum, denominator) pairs
+ * and the combine tickets - is taken from an array of MTLA_STATIC_SCRATCH_BYTES that is built
+ * into the library image, so each GPU that loads the library carries it until the process
+ * exits.  The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating library
+ * routine.  x, y, B and stream mean what they mean for mtla_decode_step, and the result is the
+ * same within rounding (the partials are summed in the same order).
+ *   - Limit: (B + 148) * n_h * (r + 2) * 4 bytes (B + 296 units on the CUDA-core path) plus
+ *     the tickets must fit the array; otherwise MTLA_ERR_SCRATCH_LIMIT is returned and nothing
+ *     is enqueued.  The paper's layer (8 heads, r 256) fits up to B = 350.
+ *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress,
+ *     checked); make that first call with the handle's device current and before starting
+ *     any stream capture.
+ *   - All handles and all calls on a device share the one array, and it keeps the previous
+ *     call's contents.  The tickets are cleared on `stream` at the start of every call; the
+ *     partials are fully rewritten before they are read.  Two calls whose kernels may overlap
+ *     on the GPU (different streams, or different handles without ordering) race on it: keep
+ *     calls of this entry point ordered on one stream per device. */
+#define MTLA_STATIC_SCRATCH_BYTES (4u << 20)
+int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, void* stream);
 
 /* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3). */
 size_t mtla_cache_bytes(const mtla_handle* h);

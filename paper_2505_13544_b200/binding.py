@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
     "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
     "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
-    "mtla_profile_end_stages")
+    "mtla_profile_end_stages", "mtla_decode_step_static")
 
 DECODE_STAGES = ("input_proj", "norm_gate_update", "absorb", "attention", "combine", "value_proj",
                  "output_proj")
@@ -68,6 +68,7 @@ def load_library() -> ctypes.CDLL:
         "mtla_prefill": (ctypes.c_int, [vp, vp, i32, i32, vp, vp]),
         "mtla_decode_step": (ctypes.c_int, [vp, vp, i32, vp, vp]),
         "mtla_decode_step_host": (ctypes.c_int, [vp, vp, i32, vp, vp]),
+        "mtla_decode_step_static": (ctypes.c_int, [vp, vp, i32, vp, vp]),
         "mtla_cache_bytes": (sz, [vp]),
         "mtla_destroy": (ctypes.c_int, [vp]),
         "mtla_reset": (ctypes.c_int, [vp]),
@@ -190,6 +191,20 @@ def mtla_decode_step(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, 
     _expect(y, h, x.shape, "y")
     _check(load_library().mtla_decode_step(h.ptr, x.data_ptr(), b, y.data_ptr(),
                                            _stream_ptr(stream)), "mtla_decode_step")
+    return y
+
+
+def mtla_decode_step_static(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, stream=None):
+    """mtla_decode_step with the attention split workspace taken from the library's built-in
+    static array instead of allocated memory; x, y [B][d] on the device.  Raises MTLAError(-9)
+    when the batch and layer shape need more than that array holds."""
+    b = x.shape[0]
+    _expect(x, h, (b, h.config.d_model), "x")
+    if y is None:
+        y = torch.empty_like(x)
+    _expect(y, h, x.shape, "y")
+    _check(load_library().mtla_decode_step_static(h.ptr, x.data_ptr(), b, y.data_ptr(),
+                                                  _stream_ptr(stream)), "mtla_decode_step_static")
     return y
 
 

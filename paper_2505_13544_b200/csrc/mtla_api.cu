@@ -135,6 +135,13 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 
 }  // namespace
 
+// Split workspace of mtla_decode_step_static: lives in every GPU that loads the library, for
+// the life of the process.  In host code this name is only a handle for cudaGetSymbolAddress;
+// the device address is looked up once per device and kept here.
+static __device__ __align__(256) unsigned char g_static_scratch[MTLA_STATIC_SCRATCH_BYTES];
+constexpr int kMaxDevices = 64;
+static unsigned char* g_static_scratch_addr[kMaxDevices];
+
 struct mtla_handle {
   mtla_config cfg;
   Dims dm;
@@ -441,6 +448,13 @@ int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
   return launch_attn_fma_rpt<T, TQ, 32>(h, a, B, st);
 }
 
+// Where the attention kernels keep their split partials; nullptr members select the arena.
+struct AttnScratch {
+  float* o_part;
+  float* ml_part;
+  int* tickets;
+};
+
 // Records the event that closes stage `stage - 1` / opens stage `stage` of a profiled step.
 int prof_mark(mtla_handle* h, bool prof, int stage, cudaStream_t st) {
   if (!prof) return MTLA_OK;
@@ -451,7 +465,8 @@ int prof_mark(mtla_handle* h, bool prof, int stage, cudaStream_t st) {
 // The decode step (Section 4.1): a1 fused projection, a2-a5 post kernel, a6 absorption,
 // a7 split-K attention + combine, a8 value and output projections.
 template <typename T>
-int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) {
+int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
+                const AttnScratch* scratch = nullptr) {
   const Dims& dm = h->dm;
   const ArenaPlan& p = h->plan;
   const int hd = dm.nh * dm.dh;
@@ -517,8 +532,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
   AttnArgs aa;
   aa.qt = h->at<void>(p.qt);
   aa.cache = h->at<void>(p.cache);
-  aa.o_part = h->at<float>(p.o_part);
-  aa.ml_part = h->at<float>(p.ml_part);
+  aa.o_part = scratch ? scratch->o_part : h->at<float>(p.o_part);
+  aa.ml_part = scratch ? scratch->ml_part : h->at<float>(p.ml_part);
   aa.n_heads = dm.nh; aa.r = dm.r; aa.dr = dm.dr; aa.max_slots = dm.max_slots;
   aa.n_slots = n_slots;
   if (h->use_tc) {
@@ -527,7 +542,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) 
     AttnTcArgs ta;
     ta.o_part = aa.o_part; ta.ml_part = aa.ml_part;
     ta.o16 = h->at<bf16>(p.o);
-    ta.tickets = h->at<int>(p.attn_tickets);
+    ta.tickets = scratch ? scratch->tickets : h->at<int>(p.attn_tickets);
     ta.error_word = h->at<int>(p.err_flag);
     ta.n_heads = dm.nh; ta.r = dm.r; ta.dr = dm.dr; ta.n_slots = n_slots; ta.batch = B;
     ta.tiles_per_seq = ceil_div(n_slots, tc::kTile);
@@ -774,6 +789,42 @@ int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y
   return MTLA_OK;
 }
 
+int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, void* stream) {
+  const int chk = check_step_args(h, x, B, y);
+  if (chk != MTLA_OK) return chk;
+  if (!aligned16(x) || !aligned16(y)) return MTLA_ERR_INVALID_ARG;
+  // Same sizing as the arena's split workspace, for this call's batch.
+  const Dims& dm = h->dm;
+  const size_t units = (size_t)(h->use_tc ? kSmCount : kTargetCtas) + (size_t)B;
+  const size_t tickets_bytes = align_up((size_t)B * sizeof(int), 256);
+  const size_t ml_bytes = align_up(units * dm.nh * 2 * sizeof(float), 256);
+  const size_t o_bytes = units * dm.nh * dm.r * sizeof(float);
+  if (tickets_bytes + ml_bytes + o_bytes > MTLA_STATIC_SCRATCH_BYTES) return MTLA_ERR_SCRATCH_LIMIT;
+  // First call on this device: turn the array's host-side name into its device address.
+  int dev = -1;
+  MTLA_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  if (!g_static_scratch_addr[dev]) {
+    void* addr = nullptr;
+    MTLA_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(addr);
+  }
+  unsigned char* base = g_static_scratch_addr[dev];
+  AttnScratch sc;
+  sc.tickets = reinterpret_cast<int*>(base);
+  sc.ml_part = reinterpret_cast<float*>(base + tickets_bytes);
+  sc.o_part = reinterpret_cast<float*>(base + tickets_bytes + ml_bytes);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left: the tickets must start at zero.
+  MTLA_CUDA(cudaMemsetAsync(sc.tickets, 0, (size_t)B * sizeof(int), st));
+  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? decode_impl<bf16>(h, x, B, y, st, &sc)
+                                                 : decode_impl<float>(h, x, B, y, st, &sc);
+  if (rc != MTLA_OK) return rc;
+  h->tokens += 1;
+  h->batch = B;
+  return MTLA_OK;
+}
+
 size_t mtla_cache_bytes(const mtla_handle* h) {
   if (!h) return 0;
   return (size_t)h->batch * ceil_div(h->tokens, h->dm.s) * h->dm.W * h->dm.elem;
@@ -904,6 +955,7 @@ const char* mtla_error_string(int status) {
     case MTLA_ERR_CUDA: return "CUDA error";
     case MTLA_ERR_STATE: return "call not valid in this state";
     case MTLA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case MTLA_ERR_SCRATCH_LIMIT: return "batch and layer shape need more than the built-in static scratch";
     default: return "unknown status";
   }
 }
