@@ -37,6 +37,60 @@ struct PostArgs {
   float q_scale;          // log2(e) / sqrt(d_h), folded into the absorbed query
 };
 
+// Merge weight of Eq. 13 for one token, by a CTA of 256 threads: h = c A + a over the d_w
+// hyper-network outputs, then sigmoid(<h, g>) with g = Linear(pe_j) from the table.  `c` is the
+// normalised latent in shared memory; `part` holds 512 floats, `red` 33.  A [r][d_w] is read
+// once per CTA: each thread owns two adjacent outputs and a slice of the r rows, with sixteen
+// independent 8-byte loads in flight to cover the L2 latency (d_w even; a scalar loop otherwise).
+// Every thread receives the weight.  Contains __syncthreads().
+__device__ inline float gate_weight(const float* c, const float* hyp_w, const float* hyp_b,
+                                    const float* gate_pe, int r, int dw, float* part, float* red) {
+  const int tid = threadIdx.x;
+  float prod = 0.f;
+  if ((dw & 1) == 0) {
+    const int pairs = dw >> 1, parts = 256 / pairs;      // pairs <= 128, so parts >= 2
+    float h0 = 0.f, h1 = 0.f;
+    if (tid < parts * pairs) {
+      const int n2 = tid % pairs, part_i = tid / pairs;
+      const int per = ceil_div(r, parts);
+      const int lo = part_i * per, hi = min(r, lo + per);
+      const float2* wp = reinterpret_cast<const float2*>(hyp_w) + n2;
+#pragma unroll 16
+      for (int i = lo; i < hi; ++i) {
+        const float2 wv = __ldg(wp + (long long)i * pairs);
+        h0 = fmaf(c[i], wv.x, h0);
+        h1 = fmaf(c[i], wv.y, h1);
+      }
+    }
+    part[2 * tid] = h0;
+    part[2 * tid + 1] = h1;
+    __syncthreads();
+    if (tid < dw) {
+      float hn = hyp_b[tid];
+      for (int p = 0; p < parts; ++p) hn += part[2 * (p * pairs + (tid >> 1)) + (tid & 1)];
+      prod = hn * gate_pe[tid];
+    }
+  } else {
+    const int parts = 256 / dw > 0 ? 256 / dw : 1;
+    float h = 0.f;
+    if (tid < parts * dw) {
+      const int n = tid % dw, part_i = tid / dw;
+      const int per = ceil_div(r, parts);
+      const int lo = part_i * per, hi = min(r, lo + per);
+      for (int i = lo; i < hi; ++i) h = fmaf(c[i], hyp_w[(long long)i * dw + n], h);
+    }
+    part[tid] = h;
+    __syncthreads();
+    if (tid < dw) {
+      float hn = hyp_b[tid];
+      for (int p = 0; p < parts; ++p) hn += part[p * dw + tid];
+      prod = hn * gate_pe[tid];
+    }
+  }
+  const float logit = block_sum(prod, red);
+  return 1.f / (1.f + expf(-logit));
+}
+
 // One CTA of 256 threads per sequence.  Section 4.1: c_i = LayerNorm(x_i W_r); Eq. 13 gate;
 // slot update (open: c_hat_j = w c, else c_hat_j += w c); Section 4.3: RoPE key replaces
 // the slot's key, RoPE queries are rotated and written behind the absorbed query.
@@ -44,7 +98,7 @@ struct PostArgs {
 template <typename T, typename TQ>
 __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   __shared__ float c_s[512];
-  __shared__ float part_s[256];
+  __shared__ float part_s[512];
   __shared__ float red_s[33];
   const int b = blockIdx.x, tid = threadIdx.x;
   const float* row = a.p1 + (long long)b * a.proj.width;
@@ -68,27 +122,8 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   __syncthreads();
 
   // Hyper-network gate: w = sigmoid(<c A + a, Linear(pe_j)>).
-  float w = 1.f;
-  if (a.use_gate) {
-    const int parts = 256 / a.dw > 0 ? 256 / a.dw : 1;
-    float h = 0.f;
-    if (tid < parts * a.dw) {
-      const int n = tid % a.dw, part = tid / a.dw;
-      const int per = ceil_div(a.r, parts);
-      const int lo = part * per, hi = min(a.r, lo + per);
-      for (int i = lo; i < hi; ++i) h = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], h);
-    }
-    part_s[tid] = h;
-    __syncthreads();
-    float prod = 0.f;
-    if (tid < a.dw) {
-      float hn = a.hyp_c_b[tid];
-      for (int p = 0; p < parts; ++p) hn += part_s[p * a.dw + tid];
-      prod = hn * a.gate_pe[tid];
-    }
-    const float logit = block_sum(prod, red_s);
-    w = 1.f / (1.f + expf(-logit));
-  }
+  const float w = a.use_gate ? gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, a.gate_pe, a.r, a.dw, part_s, red_s)
+                             : 1.f;
 
   // Slot update: fp32 running sum, stored to the cache in the storage type.
   const int W = a.r + a.dr;

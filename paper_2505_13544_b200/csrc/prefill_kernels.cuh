@@ -37,7 +37,7 @@ template <typename T, typename TQ>
 __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
   __shared__ float c_s[512];
   __shared__ float acc_s[512];
-  __shared__ float part_s[256];
+  __shared__ float part_s[512];
   __shared__ float red_s[33];
   const int chunk = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const int W = a.r + a.dr, DQ = a.head_dim + a.dr, half = a.dr / 2;
@@ -67,27 +67,8 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
       c_s[i] = (c_s[i] - mean) * rstd * a.gamma[i] + a.beta[i];
     __syncthreads();
 
-    float w = 1.f;
-    if (a.use_gate) {
-      const int parts = 256 / a.dw > 0 ? 256 / a.dw : 1;
-      float h = 0.f;
-      if (tid < parts * a.dw) {
-        const int n = tid % a.dw, part = tid / a.dw;
-        const int per = ceil_div(a.r, parts);
-        const int lo = part * per, hi = min(a.r, lo + per);
-        for (int i = lo; i < hi; ++i) h = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], h);
-      }
-      part_s[tid] = h;
-      __syncthreads();
-      float prod = 0.f;
-      if (tid < a.dw) {
-        float hn = a.hyp_c_b[tid];
-        for (int p = 0; p < parts; ++p) hn += part_s[p * a.dw + tid];
-        prod = hn * gate_pe[tid];
-      }
-      const float logit = block_sum(prod, red_s);
-      w = 1.f / (1.f + expf(-logit));
-    }
+    const float w = a.use_gate ? gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, gate_pe, a.r, a.dw, part_s, red_s)
+                               : 1.f;
 
     T* cp = static_cast<T*>(a.cprime) + rowi * a.r;
     for (int i = tid; i < a.r; i += 256) {
