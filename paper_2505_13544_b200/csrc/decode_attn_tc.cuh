@@ -42,9 +42,11 @@
 // One thread can issue a tcgen05.mma only about every hundred cycles, far slower than these
 // small-N MMAs execute, so issue is spread over six single-thread issuers in six warps: four
 // for the scores (issuer k owns partial accumulator k) and two for the values (output blocks
-// of even / odd index).  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
-// warps 5-6 = value issuers, warp 7 idle, warps 8-11 = softmax and epilogue.  The first two
-// warpgroups give most of their registers to the third (setmaxnreg).
+// of even / odd index).  The softmax is instruction-bound too, so it runs on eight warps: with
+// M = 64 only lanes 0-15 of a warp's TMEM quarter hold scores, and two warps per quarter split
+// the heads between them.  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
+// warps 5-6 = value issuers, warp 7 idle, warps 8-15 = softmax and epilogue.  The first two
+// warpgroups give most of their registers to the other two (setmaxnreg).
 //
 // Every wait is a bounded mbarrier wait (see sm100_ptx.cuh), the rendezvous of the softmax
 // threads included; on a timeout the CTA raises its abort word, all roles unwind, and the host
@@ -71,8 +73,9 @@ struct AttnTcArgs {
 namespace tc {
 
 constexpr int kTile = 64;                  // slots per tile
-constexpr int kThreads = 384;
+constexpr int kThreads = 512;
 constexpr int kQkIssuers = 4, kPvIssuers = 2;
+constexpr int kFirstSoftmaxWarp = 8, kSoftmaxThreads = 256;
 constexpr int kSubBytes = kTile * 128;     // one 64-column sub-tile
 constexpr int kPairBytes = 2 * kSubBytes;
 constexpr int kPairs = 9;
@@ -90,7 +93,7 @@ constexpr int kMaxQBytes = 9 * 32 * 128;   // (2 * 4 + 1) chunks x 32 heads x 12
 constexpr int kOffP = kOffQ + kMaxQBytes;
 constexpr int kPBytes = 32 * kTile * 2;    // one probability buffer
 constexpr int kOffMisc = kOffP + 2 * kPBytes;
-constexpr int kMiscBytes = 3072;
+constexpr int kMiscBytes = 4096;
 constexpr int kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + slack for 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
@@ -104,9 +107,8 @@ struct Misc {
   int last_flag;
   int exceed_flag[2];      // raised by any softmax thread whose tile outgrew a reference
   float m_used[32];        // per-head reference maximum of the running segment (log2 units)
-  float wmax[4][32];
+  float red[8][32];        // per-warp reductions (tile maxima / denominators) of the softmax warps
   float fac[32];
-  float lsum[4][32];
   float comb_m[32];
   float comb_w[8][32];     // combine: weight of part p for head h (first 8 parts cached)
 };
@@ -174,15 +176,15 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(&misc->s_full[i]), kQkIssuers);
-      mbar_init(bar(&misc->s_empty[i]), 128);
-      mbar_init(bar(&misc->p_full[i]), 128);
+      mbar_init(bar(&misc->s_empty[i]), kSoftmaxThreads);
+      mbar_init(bar(&misc->p_full[i]), kSoftmaxThreads);
       mbar_init(bar(&misc->p_empty[i]), kPvIssuers);
     }
     mbar_init(bar(&misc->q_full), 1);
     mbar_init(bar(&misc->q_empty), kQkIssuers);
-    mbar_init(bar(&misc->flag_bar[0]), 128);
-    mbar_init(bar(&misc->flag_bar[1]), 128);
-    mbar_init(bar(&misc->group_sync), 128);
+    mbar_init(bar(&misc->flag_bar[0]), kSoftmaxThreads);
+    mbar_init(bar(&misc->flag_bar[1]), kSoftmaxThreads);
+    mbar_init(bar(&misc->group_sync), kSoftmaxThreads);
     misc->abort_word = 0;
     misc->last_flag = 0;
     misc->exceed_flag[0] = 0;
@@ -206,8 +208,8 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   const uint32_t q_u32 = base + kOffQ, p_u32 = base + kOffP;
 
   if (warp < 8) {
-  // Register budget: the producer / issuer warpgroups keep 56 registers, the softmax one gets 240.
-  reg_dealloc<56>();
+  // Register budget: the producer / issuer warpgroups keep 48 registers, the softmax ones get 208.
+  reg_dealloc<48>();
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
@@ -312,20 +314,48 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   }
   } else {
     // ------------------------------------------------------------------ softmax / epilogue warps
-    reg_alloc<240>();
-    const int q = warp & 3, sidx = q * 32 + lane;          // TMEM quarter; index among the 128
+    // Two groups of four warps; group g owns heads [g * NHH, (g + 1) * NHH) of every slot, i.e.
+    // TMEM columns g * NHH .. of each score partial and of each output block.
+    reg_alloc<208>();
+    constexpr int NHH = NHP / 2;
+    const int sw = warp - kFirstSoftmaxWarp;                // 0..7
+    const int g = sw >> 2, q = warp & 3;                    // head group; TMEM lane quarter
+    const int HO = g * NHH;
+    const int sidx = sw * 32 + lane;                        // index among the 256
     const bool active = lane < 16;                          // lanes that own a slot (M = 64 layout)
     const int row = q * 16 + lane;                          // slot within the tile (active lanes)
-    const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+    const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16) + HO;
     bool ok = true;
-    // Rendezvous of the 128 threads on an mbarrier, so that it is bounded like every other wait.
+    auto ld_cols = [&](uint32_t addr, uint32_t (&v)[16]) {
+      if (NHH == 16) tmem_ld_x16(addr, v); else tmem_ld_x8(addr, v);
+    };
+    auto st_cols = [&](uint32_t addr, const uint32_t (&v)[16]) {
+      if (NHH == 16) tmem_st_x16(addr, v); else tmem_st_x8(addr, v);
+    };
+    // Rendezvous of the 256 threads on an mbarrier, so that it is bounded like every other wait.
     int sync_phase = 0;
     auto group_sync = [&]() {
       mbar_arrive(bar(&misc->group_sync));
       if (ok) ok = mbar_wait(bar(&misc->group_sync), sync_phase & 1, abort_word, a.error_word, 13);
       ++sync_phase;
     };
-    float l_acc[32];
+    // Per-warp reduction of one value per owned head over the warp's 32 lanes, left in
+    // misc->red[sw][i] for head HO + i.
+    auto reduce_heads = [&](const float (&v)[NHH], float fill, bool is_max) {
+      float red[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) red[i] = i < NHH ? v[i < NHH ? i : 0] : fill;
+      misc->red[sw][lane] = is_max
+          ? transposed_reduce(red, lane, [](float x, float y) { return fmaxf(x, y); })
+          : transposed_reduce(red, lane, [](float x, float y) { return x + y; });
+    };
+    // Head h's value combined over the four warps of the group that owns it.
+    auto reduced = [&](int h, bool is_max) {
+      const int gg = h / NHH, i = h % NHH;
+      const float* r0 = &misc->red[gg * 4][i];
+      return is_max ? fmaxf(fmaxf(r0[0], r0[32]), fmaxf(r0[64], r0[96])) : r0[0] + r0[32] + r0[64] + r0[96];
+    };
+    float l_acc[NHH];
     int b = (int)(g0 / tps), t = (int)(g0 - (long long)b * tps);
     for (int n = 0; n < n_tiles; ++n, ++t) {
       if (t == (int)tps) {
@@ -335,44 +365,38 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       const bool seg_first = n == 0 || t == 0;
       const bool seg_last = n + 1 == n_tiles || t + 1 == (int)tps;
       if (seg_first) {
-        // New sequence: empty references (shared by the 128 threads) and denominators.
+        // New sequence: empty references (shared by all threads) and denominators.
         if (sidx < 32) misc->m_used[sidx] = -INFINITY;
 #pragma unroll
-        for (int h = 0; h < 32; ++h) l_acc[h] = 0.f;
+        for (int i = 0; i < NHH; ++i) l_acc[i] = 0.f;
         group_sync();
       }
-      float s[32];
+      float s[NHH];
 #pragma unroll
-      for (int h = 0; h < 32; ++h) s[h] = 0.f;
+      for (int i = 0; i < NHH; ++i) s[i] = 0.f;
       if (ok) ok = mbar_wait(bar(&misc->s_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 5);
       ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are whole-warp operations
       if (ok) {
         tc_fence_after_sync();
         const uint32_t s_addr = lane_base + kColS + (n & 1) * (kSParts * 32);
+        uint32_t sp[kSParts][16];
 #pragma unroll
-        for (int k2 = 0; k2 < kSParts; k2 += 2) {   // the score is the sum of the partials
-          uint32_t sa[32], sb[32];
-          if (NHP == 32) {
-            tmem_ld_x32(s_addr + k2 * 32, sa);
-            tmem_ld_x32(s_addr + (k2 + 1) * 32, sb);
-          } else {
-            tmem_ld_x16(s_addr + k2 * 32, sa);
-            tmem_ld_x16(s_addr + (k2 + 1) * 32, sb);
-          }
-          tmem_wait_ld();
+        for (int k = 0; k < kSParts; ++k) ld_cols(s_addr + k * 32, sp[k]);
+        tmem_wait_ld();
 #pragma unroll
-          for (int h = 0; h < NHP; ++h) s[h] += __uint_as_float(sa[h]) + __uint_as_float(sb[h]);
-        }
+        for (int i = 0; i < NHH; ++i)               // the score is the sum of the partials
+          s[i] = (__uint_as_float(sp[0][i]) + __uint_as_float(sp[1][i])) +
+                 (__uint_as_float(sp[2][i]) + __uint_as_float(sp[3][i]));
         tc_fence_before_sync();
       }
       const bool valid = ok && active && t * kTile + row < a.n_slots;
-      float m_ref[32];
+      float m_ref[NHH];
       bool exceed = false;
 #pragma unroll
-      for (int h = 0; h < NHP; ++h) {
-        m_ref[h] = misc->m_used[h];
-        s[h] = valid ? s[h] : -INFINITY;
-        exceed |= s[h] > m_ref[h] + kRescaleThreshold;
+      for (int i = 0; i < NHH; ++i) {
+        m_ref[i] = misc->m_used[HO + i];
+        s[i] = valid ? s[i] : -INFINITY;
+        exceed |= s[i] > m_ref[i] + kRescaleThreshold;
       }
       // Tell the others (rarely) that a reference must rise; the answer is collected further
       // down, after the probabilities have been formed with the current references.
@@ -380,13 +404,13 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       mbar_arrive(bar(&misc->flag_bar[n & 1]));
       if (ok) mbar_arrive(bar(&misc->s_empty[n & 1]));
 
-      uint32_t pb[16];
+      uint32_t pb[NHH / 2];
       auto probabilities = [&]() {
 #pragma unroll
-        for (int h = 0; h < NHP; h += 2) {
-          const __nv_bfloat162 pk = __floats2bfloat162_rn(ex2_approx(s[h] - m_ref[h]),
-                                                          ex2_approx(s[h + 1] - m_ref[h + 1]));
-          pb[h / 2] = *reinterpret_cast<const uint32_t*>(&pk);
+        for (int i = 0; i < NHH; i += 2) {
+          const __nv_bfloat162 pk = __floats2bfloat162_rn(ex2_approx(s[i] - m_ref[i]),
+                                                          ex2_approx(s[i + 1] - m_ref[i + 1]));
+          pb[i / 2] = *reinterpret_cast<const uint32_t*>(&pk);
         }
       };
       // P^T as the K-major, un-swizzled B operand of the value MMA: element (head h, slot k)
@@ -395,8 +419,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         if (!active) return;
         uint8_t* prow = sm + kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
 #pragma unroll
-        for (int h = 0; h < NHP; ++h) {
-          const uint16_t bits = (h & 1) ? (uint16_t)(pb[h / 2] >> 16) : (uint16_t)(pb[h / 2] & 0xffffu);
+        for (int i = 0; i < NHH; ++i) {
+          const int h = HO + i;
+          const uint16_t bits = (i & 1) ? (uint16_t)(pb[i / 2] >> 16) : (uint16_t)(pb[i / 2] & 0xffffu);
           *reinterpret_cast<uint16_t*>(prow + (h >> 3) * PSBO + (h & 7) * 16) = bits;
         }
       };
@@ -408,16 +433,12 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (ok && misc->exceed_flag[n & 1]) {
         // ---- rare: some head's scores rose more than 2^8 above its reference (always at
         // a sequence's first tile).  Everybody takes this branch: the flag is read after all
-        // 128 arrivals.  New references, rescaled denominators and accumulators, new P.
-        float red[32];
-#pragma unroll
-        for (int h = 0; h < 32; ++h) red[h] = h < NHP ? s[h] : -INFINITY;
-        misc->wmax[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return fmaxf(x, y); });
+        // arrivals.  New references, rescaled denominators and accumulators, new P.
+        reduce_heads(s, -INFINITY, true);
         group_sync();
         if (sidx == 0) misc->exceed_flag[n & 1] = 0;
-        if (sidx < 32) {
-          const float mt = fmaxf(fmaxf(misc->wmax[0][sidx], misc->wmax[1][sidx]),
-                                 fmaxf(misc->wmax[2][sidx], misc->wmax[3][sidx]));
+        if (sidx < NHP) {
+          const float mt = reduced(sidx, true);
           const float m_old = misc->m_used[sidx];
           const float m_nw = mt > m_old + kRescaleThreshold ? mt : m_old;
           misc->m_used[sidx] = m_nw;
@@ -425,39 +446,40 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         }
         group_sync();
 #pragma unroll
-        for (int h = 0; h < NHP; ++h) {
-          m_ref[h] = misc->m_used[h];
-          l_acc[h] *= misc->fac[h];
+        for (int i = 0; i < NHH; ++i) {
+          m_ref[i] = misc->m_used[HO + i];
+          l_acc[i] *= misc->fac[HO + i];
         }
         if (!seg_first) {
           // O holds contributions scaled to the old references: wait for the previous tile's
-          // value MMAs, then rescale the accumulator columns in TMEM.
+          // value MMAs, then rescale this group's accumulator columns in TMEM.
           if (ok) ok = mbar_wait(bar(&misc->p_empty[(n - 1) & 1]), ((n - 1) >> 1) & 1, abort_word,
                                  a.error_word, 6);
           ok = __all_sync(0xffffffffu, ok);
           if (ok) {
             tc_fence_after_sync();
             for (int mb = 0; mb < RP; ++mb) {
-              uint32_t ov[32];
+              uint32_t ov[16];
               const uint32_t addr = lane_base + kColO + mb * 32;
-              if (NHP == 32) tmem_ld_x32(addr, ov); else tmem_ld_x16(addr, ov);
+              ld_cols(addr, ov);
               tmem_wait_ld();
 #pragma unroll
-              for (int h = 0; h < NHP; ++h) ov[h] = __float_as_uint(__uint_as_float(ov[h]) * misc->fac[h]);
-              if (NHP == 32) tmem_st_x32(addr, ov); else tmem_st_x16(addr, ov);
+              for (int i = 0; i < NHH; ++i)
+                ov[i] = __float_as_uint(__uint_as_float(ov[i]) * misc->fac[HO + i]);
+              st_cols(addr, ov);
             }
             tmem_wait_st();
           }
         }
         probabilities();
         if (ok) store_probabilities();
-        group_sync();                         // fac / wmax may be rewritten by the next rare tile
+        group_sync();                         // fac / red may be rewritten by the next rare tile
       }
 #pragma unroll
-      for (int h = 0; h < NHP; h += 2) {
-        const __nv_bfloat162 pk = *reinterpret_cast<const __nv_bfloat162*>(&pb[h / 2]);
-        l_acc[h] += __low2float(pk);
-        l_acc[h + 1] += __high2float(pk);
+      for (int i = 0; i < NHH; i += 2) {
+        const __nv_bfloat162 pk = *reinterpret_cast<const __nv_bfloat162*>(&pb[i / 2]);
+        l_acc[i] += __low2float(pk);
+        l_acc[i + 1] += __high2float(pk);
       }
       if (ok) {
         fence_proxy_async_smem();
@@ -475,26 +497,21 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         tc_fence_after_sync();
         float* o_part = a.o_part + part * a.n_heads * a.r;
         for (int mb = 0; mb < RP; ++mb) {
-          uint32_t ov[32];
-          const uint32_t addr = lane_base + kColO + mb * 32;
-          if (NHP == 32) tmem_ld_x32(addr, ov); else tmem_ld_x16(addr, ov);
+          uint32_t ov[16];
+          ld_cols(lane_base + kColO + mb * 32, ov);
           tmem_wait_ld();
 #pragma unroll
-          for (int h = 0; h < NHP; ++h)
-            if (h < a.n_heads) o_part[h * a.r + mb * 128 + sidx] = __uint_as_float(ov[h]);
+          for (int i = 0; i < NHH; ++i)
+            if (HO + i < a.n_heads) o_part[(HO + i) * a.r + mb * 128 + q * 32 + lane] = __uint_as_float(ov[i]);
         }
         tc_fence_before_sync();
       }
-      float red[32];
-#pragma unroll
-      for (int h = 0; h < 32; ++h) red[h] = h < NHP ? l_acc[h] : 0.f;
-      misc->lsum[q][lane] = transposed_reduce(red, lane, [](float x, float y) { return x + y; });
+      reduce_heads(l_acc, 0.f, false);
       __threadfence();
       group_sync();
       if (ok && sidx < a.n_heads) {
         a.ml_part[(part * a.n_heads + sidx) * 2] = misc->m_used[sidx];
-        a.ml_part[(part * a.n_heads + sidx) * 2 + 1] =
-            misc->lsum[0][sidx] + misc->lsum[1][sidx] + misc->lsum[2][sidx] + misc->lsum[3][sidx];
+        a.ml_part[(part * a.n_heads + sidx) * 2 + 1] = reduced(sidx, false);
         __threadfence();
       }
       // Ticket: the CTA that delivers the sequence's last partial combines them.
@@ -530,18 +547,19 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
           misc->comb_m[sidx] = m;
         }
         group_sync();
-        // Thread sidx owns latent columns 4*sidx .. 4*sidx+3 (r/4 <= 128 threads are busy).
-        if (ok && 4 * sidx < a.r) {
-          bf16* o_hi = a.o16 + (long long)b * 2 * a.n_heads * a.r + 4 * sidx;
+        // Thread (cg, hh): latent columns 4*cg .. 4*cg+3 of the heads of parity hh.
+        const int cg = sidx & 127, hh = sidx >> 7;
+        if (ok && 4 * cg < a.r) {
+          bf16* o_hi = a.o16 + (long long)b * 2 * a.n_heads * a.r + 4 * cg;
           bf16* o_lo = o_hi + (long long)a.n_heads * a.r;
-          for (int h = 0; h < a.n_heads; ++h) {
+          for (int h = hh; h < a.n_heads; h += 2) {
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int pt = 0; pt < n_parts; ++pt) {
               const float wgt = pt < 8 ? misc->comb_w[pt][h]
                                        : exp2f(__ldcg(a.ml_part + ((part0 + pt) * a.n_heads + h) * 2) -
                                                misc->comb_m[h]);
               const float4 v = __ldcg(reinterpret_cast<const float4*>(
-                  a.o_part + ((part0 + pt) * a.n_heads + h) * a.r + 4 * sidx));
+                  a.o_part + ((part0 + pt) * a.n_heads + h) * a.r + 4 * cg));
               acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
               acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
             }
