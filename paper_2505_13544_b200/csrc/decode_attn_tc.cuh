@@ -18,11 +18,9 @@
 // of slot i sits in TMEM lane 32*(i/16) + i%16, i.e. in the first 16 lanes of each warp's
 // quarter, so lanes 0-15 of each softmax warp own one slot each.
 //
-// An MMA that accumulates into the tile a previous MMA wrote cannot start before that one has
-// drained, and with N this small the drain latency dwarfs the arithmetic.  So consecutive MMAs
-// never share an accumulator: a score buffer is four partial accumulators (k-step ks of every
-// 64-column chunk goes to partial ks; the softmax threads add the four), and the value MMAs
-// rotate over the r/128 output blocks.
+// A score buffer is four partial accumulators: k-step ks (16 columns) of every 64-column chunk
+// goes to partial ks, each partial has its own issuing thread (see below), and the softmax
+// threads add the four when they read them.
 //
 // Shared memory: a ring of nine 16 KB "pairs" (two adjacent sub-tiles = a 128-row MN-major
 // operand block), three 8 KB sub-tiles for the RoPE-key columns, q~ as a K-major swizzled B
@@ -40,13 +38,13 @@
 // and denominator.
 //
 // One thread can issue a tcgen05.mma only about every hundred cycles, far slower than these
-// small-N MMAs execute, so issue is spread over six single-thread issuers in six warps: four
-// for the scores (issuer k owns partial accumulator k) and two for the values (output blocks
-// of even / odd index).  The softmax is instruction-bound too, so it runs on eight warps: with
+// small-N MMAs execute, so issue is spread over eight single-thread issuers in eight warps:
+// four for the scores (issuer k owns partial accumulator k) and four for the values (issuer j
+// owns output block j and returns its pair to the ring as soon as its four MMAs are in).  The softmax is instruction-bound too, so it runs on eight warps: with
 // M = 64 only lanes 0-15 of a warp's TMEM quarter hold scores, and two warps per quarter split
 // the heads between them.  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
-// warps 5-6 = value issuers, warp 7 idle, warps 8-15 = softmax and epilogue.  The first two
-// warpgroups give most of their registers to the other two (setmaxnreg).
+// warps 5-8 = value issuers, warps 9-11 idle, warps 12-19 = softmax and epilogue.  The first
+// three warpgroups give most of their registers to the other two (setmaxnreg).
 //
 // Every wait is a bounded mbarrier wait (see sm100_ptx.cuh), the rendezvous of the softmax
 // threads included; on a timeout the CTA raises its abort word, all roles unwind, and the host
@@ -73,9 +71,19 @@ struct AttnTcArgs {
 namespace tc {
 
 constexpr int kTile = 64;                  // slots per tile
-constexpr int kThreads = 512;
-constexpr int kQkIssuers = 4, kPvIssuers = 2;
-constexpr int kFirstSoftmaxWarp = 8, kSoftmaxThreads = 256;
+constexpr int kThreads = 640;
+constexpr int kQkIssuers = 4, kPvIssuers = 4;
+constexpr int kFirstSoftmaxWarp = 12, kSoftmaxThreads = 256;
+// setmaxnreg moves registers inside the pool the CTA was launched with (threads x the per-thread
+// count the compiler settles on, which is the launch-bound cap rounded down to 8).  An increase
+// that the pool cannot cover would block for ever, so the budget is checked here.
+constexpr int kRegsIssuer = 40, kRegsSoftmax = 176;
+constexpr int kRegsAtLaunch = 65536 / kThreads / 8 * 8;
+static_assert((kThreads - kSoftmaxThreads) * kRegsIssuer + kSoftmaxThreads * kRegsSoftmax <=
+                  kThreads * kRegsAtLaunch,
+              "register re-allocation exceeds the CTA's pool");
+static_assert(kFirstSoftmaxWarp % 4 == 0 && kThreads == kFirstSoftmaxWarp * 32 + kSoftmaxThreads,
+              "softmax warps must start at a warpgroup boundary");
 constexpr int kSubBytes = kTile * 128;     // one 64-column sub-tile
 constexpr int kPairBytes = 2 * kSubBytes;
 constexpr int kPairs = 9;
@@ -207,9 +215,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   const uint32_t pairs_u32 = base + kOffPairs, kr_u32 = base + kOffKr;
   const uint32_t q_u32 = base + kOffQ, p_u32 = base + kOffP;
 
-  if (warp < 8) {
-  // Register budget: the producer / issuer warpgroups keep 48 registers, the softmax ones get 208.
-  reg_dealloc<48>();
+  if (warp < kFirstSoftmaxWarp) {
+  // Register budget: the producer / issuer warpgroups keep 40 registers, the softmax ones get 176.
+  reg_dealloc<kRegsIssuer>();
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
@@ -299,16 +307,17 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (!ok) break;
       tc_fence_after_sync();
       const bool seg_first = n == 0 || t == 0;
+      for (int mb = j; mb < RP; mb += kPvIssuers) {
+        const int buf = (n * RP + mb) % kPairs;
+        const uint32_t src = pairs_u32 + buf * kPairBytes;
 #pragma unroll
-      for (int ks = 0; ks < kTile / 16; ++ks) {
-        const uint64_t bd = make_smem_desc(p_u32 + (n & 1) * kPBytes + ks * 256, 128, PSBO, kSwizzleNone);
-        for (int mb = j; mb < RP; mb += kPvIssuers) {
-          const uint32_t src = pairs_u32 + ((n * RP + mb) % kPairs) * kPairBytes;
+        for (int ks = 0; ks < kTile / 16; ++ks) {
+          const uint64_t bd = make_smem_desc(p_u32 + (n & 1) * kPBytes + ks * 256, 128, PSBO, kSwizzleNone);
           const uint64_t ad = make_smem_desc(src + ks * 2048, kSubBytes, 1024, kSwizzle128B);
           mma_bf16_ss(tmem_base + kColO + mb * 32, ad, bd, IDESC_PV, (seg_first && ks == 0) ? 0u : 1u);
         }
+        mma_commit(bar(&misc->empty_pair[buf]));      // the pair goes back to the producer at once
       }
-      for (int mb = j; mb < RP; mb += kPvIssuers) mma_commit(bar(&misc->empty_pair[(n * RP + mb) % kPairs]));
       mma_commit(bar(&misc->p_empty[n & 1]));
     }
   }
@@ -316,7 +325,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     // ------------------------------------------------------------------ softmax / epilogue warps
     // Two groups of four warps; group g owns heads [g * NHH, (g + 1) * NHH) of every slot, i.e.
     // TMEM columns g * NHH .. of each score partial and of each output block.
-    reg_alloc<208>();
+    reg_alloc<kRegsSoftmax>();
     constexpr int NHH = NHP / 2;
     const int sw = warp - kFirstSoftmaxWarp;                // 0..7
     const int g = sw >> 2, q = warp & 3;                    // head group; TMEM lane quarter

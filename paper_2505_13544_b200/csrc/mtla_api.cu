@@ -330,9 +330,17 @@ template <int NHP>
 int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_t st) {
 #define MTLA_TC_CASE(RP)                                                                       \
   case RP:                                                                                     \
-    if (!h->attn_smem_ready)                                                                   \
+    if (!h->attn_smem_ready) {                                                                 \
+      /* The kernel re-allocates registers between warpgroups; its launch-time pool must */    \
+      /* cover the budget, or the increase inside the kernel would never be granted.     */    \
+      cudaFuncAttributes fa;                                                                   \
+      MTLA_CUDA(cudaFuncGetAttributes(&fa, decode_attn_tc_kernel<NHP, RP>));                   \
+      if (fa.numRegs * tc::kThreads < (tc::kThreads - tc::kSoftmaxThreads) * tc::kRegsIssuer + \
+                                          tc::kSoftmaxThreads * tc::kRegsSoftmax)              \
+        return MTLA_ERR_CUDA;                                                                  \
       MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP>,                           \
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes)); \
+    }                                                                                          \
     decode_attn_tc_kernel<NHP, RP><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(h->cache_map,   \
                                                                                h->q_map, a);   \
     break;
