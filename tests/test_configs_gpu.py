@@ -1,0 +1,141 @@
+"""The five benchmark configurations at their full sizes, in the launch configuration the
+benchmark times, against the CPU oracle on sampled outputs.
+
+The oracle cannot follow every row of these workloads, so each test follows a few whole
+sequences through the oracle's state updates (cheap) and asks it for the attention output only
+at sampled prefill rows and decode steps; slot counts, cache bytes and positions are checked
+exactly for the whole batch, and the exported cache of the sampled sequences element by element.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mtla_oracle as O
+from paper_2505_13544_b200 import binding as M
+from paper_2505_13544_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def elem_bytes(w):
+    return 4 if w.dtype == "fp32" else 2
+
+
+def check_positions(h, w, tokens):
+    slots = math.ceil(tokens / w.stride)
+    assert M.mtla_position(h) == (tokens, slots, w.batch)
+    assert M.mtla_cache_bytes(h) == w.batch * slots * w.slot_width * elem_bytes(w)
+
+
+def run_prefill_then_decode(w, seqs, prefill_rows, decode_steps_checked):
+    """Prefill the whole batch, then decode w.decode_steps steps; compare sampled outputs."""
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    h = H.gpu_handle(w, weights)
+    try:
+        x = torch.empty(w.batch, w.prefill_tokens, w.d_model, dtype=synth.torch_dtype(w.dtype),
+                        device="cuda")
+        prompts = {}
+        for b in range(w.batch):
+            row = synth.stored(synth.normal(w.seed, f"prompt/{b}", (w.prefill_tokens, w.d_model)),
+                               w.dtype)
+            x[b].copy_(row)
+            if b in seqs:
+                prompts[b] = row.double().numpy()
+        y = M.mtla_prefill(h, x)
+        M.mtla_check(h)
+        check_positions(h, w, w.prefill_tokens)
+        states = {}
+        for b in seqs:
+            want, st = O.decode_sequence(p, prompts[b], rows=prefill_rows)
+            H.assert_close(y[b, prefill_rows], want, w.dtype, f"prefill seq {b}")
+            states[b] = st
+        cache = M.mtla_cache_export(h)
+        H.assert_cache_close(cache[seqs], np.stack([O.cache_array(states[b]) for b in seqs]), w.dtype)
+        del x, y, cache
+        for i in range(w.decode_steps):
+            xi = synth.decode_input(w, i)
+            yi = M.mtla_decode_step(h, xi.cuda())
+            check = i in decode_steps_checked
+            want = [O.decode_step(p, states[b], xi[b].double().numpy(), want_output=check)
+                    for b in seqs]
+            if check:
+                M.mtla_check(h)
+                H.assert_close(yi[seqs], np.stack(want), w.dtype, f"decode step {i}")
+        check_positions(h, w, w.prefill_tokens + w.decode_steps)
+        cache = M.mtla_cache_export(h)
+        H.assert_cache_close(cache[seqs], np.stack([O.cache_array(states[b]) for b in seqs]), w.dtype)
+    finally:
+        M.mtla_destroy(h)
+
+
+def test_config_tiny_every_output():
+    """fp32, batch 1: every prefill row and every decode step is compared."""
+    w = synth.WORKLOADS["tiny"]
+    run_prefill_then_decode(w, [0], list(range(w.prefill_tokens)), set(range(w.decode_steps)))
+
+
+def test_config_paper_scale():
+    w = synth.WORKLOADS["paper"]
+    rows = [0, 1, 2, 3, 127, 128, 129, 511, 1000, 1022, 1023]
+    steps = {0, 1, 2, 63, 64, 500, 1022, 1023}
+    run_prefill_then_decode(w, [0, 17, 31], rows, steps)
+
+
+@pytest.mark.parametrize("s", [1, 2, 3, 4])
+def test_config_stride_sweep(s):
+    """4096 = 3 * 1365 + 1: at s = 3 the prompt leaves an open slot that decoding continues."""
+    w = synth.WORKLOADS[f"sweep_s{s}"]
+    rows = [0, 1, 5, 6, 63, 64, 65, 2047, 4094, 4095]
+    steps = {0, 1, 2, 3, 128, 255}
+    run_prefill_then_decode(w, [0, 63], rows, steps)
+
+
+def test_config_long_context_prefill():
+    w = synth.WORKLOADS["longctx"]
+    rows = [0, 3, 4, 255, 256, 8191, 16380, 16383]
+    run_prefill_then_decode(w, [0, 7], rows, {0, 1, 3, 4, 63})
+
+
+def test_config_large_decode():
+    """Batch 128 over an imported 32768-token context, as bench.py runs it."""
+    w = synth.WORKLOADS["large"]
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    seqs = [0, 1, w.batch - 1]
+    n_slots = math.ceil(w.context_tokens / w.stride)
+    cfg = M.make_config(**H.dims_of(w), max_batch=w.batch,
+                        max_tokens=w.context_tokens + w.decode_steps, max_prefill_tokens=0,
+                        dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    h = M.mtla_create(cfg, {k: v.cuda() for k, v in weights.items()})
+    try:
+        cache = torch.empty(w.batch, n_slots, w.slot_width, dtype=torch.bfloat16, device="cuda")
+        states = {}
+        for b in range(w.batch):
+            row = synth.context_cache_row(w, b)
+            cache[b].copy_(row)
+            if b in seqs:
+                states[b] = O.state_from_cache(row.double().numpy(), w.context_tokens, p)
+        M.mtla_cache_import(h, cache, w.context_tokens)
+        del cache
+        check_positions(h, w, w.context_tokens)
+        checked = {0, 1, 2, 64, 127}
+        for i in range(w.decode_steps):
+            xi = synth.decode_input(w, i)
+            yi = M.mtla_decode_step(h, xi.cuda())
+            check = i in checked
+            want = [O.decode_step(p, states[b], xi[b].double().numpy(), want_output=check)
+                    for b in seqs]
+            if check:
+                M.mtla_check(h)
+                H.assert_close(yi[seqs], np.stack(want), "bf16", f"decode step {i}")
+        check_positions(h, w, w.context_tokens + w.decode_steps)
+        # The 64 slots the decode steps wrote, element by element, for the sampled sequences.
+        tail = M.mtla_cache_export(h)[seqs, n_slots:]
+        want_tail = np.stack([O.cache_array(states[b])[n_slots:] for b in seqs])
+        H.assert_cache_close(tail, want_tail, "bf16")
+    finally:
+        M.mtla_destroy(h)
