@@ -15,9 +15,10 @@
 // Eq. 12; value up-projection, Eq. 10).
 //
 // Activations that were produced in fp32 by an earlier kernel can be passed as two bf16 halves
-// (value = hi + lo); the kernel then runs each K block twice against the same weight tile, the
-// second copy of which comes from L2.  These products are weight-bandwidth bound, so the extra
-// MMAs are free and the intermediate keeps fp32-like precision.
+// (value = hi + lo), which keeps fp32-like precision of the intermediate.  With HILO the two
+// halves of the BN activation rows are stacked as one B tile of 2 BN rows, so a single MMA per
+// k-step multiplies the weight tile by both and the epilogue adds the two column halves of the
+// accumulator; when 2 BN would exceed the MMA's N (BN = 256) each K block is run twice instead.
 //
 // Split-K partials go to a workspace; the last CTA (per 32-row quarter of a tile) to take a
 // ticket sums them in split order, so results do not depend on arrival order and no CTA ever
@@ -59,10 +60,12 @@ constexpr int kBM = 128, kBK = 64;
 constexpr int kABytes = kBM * kBK * 2;
 
 __host__ __device__ constexpr int b_bytes(int bn) { return bn * kBK * 2; }
-__host__ __device__ constexpr int stage_bytes(int bn) { return kABytes + b_bytes(bn); }
-__host__ __device__ constexpr int smem_bytes(int bn, int stages) {
-  return stages * stage_bytes(bn) + 1024 /* alignment slack */ + 256 /* barriers */;
+// `nb` = rows of the B tile (BN, or 2 BN with stacked hi / lo halves).
+__host__ __device__ constexpr int stage_bytes(int nb) { return kABytes + b_bytes(nb); }
+__host__ __device__ constexpr int smem_bytes(int nb, int stages) {
+  return stages * stage_bytes(nb) + 1024 /* alignment slack */ + 256 /* barriers */;
 }
+
 // As many stages as fit one CTA per SM (weight streaming wants bytes in flight), at most 8.
 __host__ __device__ constexpr int deep_stages(int bn) {
   return (200 * 1024) / stage_bytes(bn) > 8 ? 8 : (200 * 1024) / stage_bytes(bn);
@@ -123,7 +126,7 @@ __device__ __forceinline__ void store4(bf16* p, const float (&v)[4], long long l
 
 }  // namespace gtc
 
-template <int BN, int STAGES, typename OutT>
+template <int BN, int STAGES, typename OutT, bool HILO>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                GemmTcArgs g) {
@@ -132,14 +135,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   static_assert(BN == 16 || BN == 32 || BN == 64 || BN == 128 || BN == 256, "BN");
   static_assert(STAGES >= 2 && STAGES <= 8, "STAGES");
   constexpr int CH = BN < 32 ? 16 : 32;             // TMEM columns per epilogue chunk
-  constexpr uint32_t IDESC = make_idesc_bf16(128, BN, 0, 0);
-  constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+  constexpr int NB = HILO ? 2 * BN : BN;            // rows of the B tile = the MMA's N
+  static_assert(NB <= 256, "stacked hi / lo halves exceed the MMA's N");
+  constexpr uint32_t IDESC = make_idesc_bf16(128, NB, 0, 0);
+  constexpr uint32_t TMEM_COLS = NB < 32 ? 32 : NB;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
-  Bars* bars = reinterpret_cast<Bars*>(sm + STAGES * stage_bytes(BN));
+  Bars* bars = reinterpret_cast<Bars*>(sm + STAGES * stage_bytes(NB));
   volatile int* abort_word = &bars->abort_word;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   auto bar = [&](unsigned long long* p) { return smem_u32(p); };
@@ -167,7 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int kb_total = (g.k + kBK - 1) / kBK;
   const int kb0 = split * g.kb_per_split;
   const int n_kb = min(kb_total, kb0 + g.kb_per_split) - kb0;   // >= 1 by construction
-  const int passes = g.b_lo_col > 0 ? 2 : 1;
+  const int passes = (!HILO && g.b_lo_col > 0) ? 2 : 1;
   const int n_it = n_kb * passes;
 
   if (warp == 0 && lane == 0) {
@@ -178,11 +183,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int st = i % STAGES, use = i / STAGES;
       const int kb = kb0 + (passes == 2 ? i >> 1 : i), lo = passes == 2 ? (i & 1) : 0;
       if (!mbar_wait(bar(&bars->empty[st]), (use & 1) ^ 1, abort_word, g.error_word, 11)) break;
-      const uint32_t dst = base + st * stage_bytes(BN);
-      mbar_arrive_expect_tx(bar(&bars->full[st]), stage_bytes(BN));
+      const uint32_t dst = base + st * stage_bytes(NB);
+      mbar_arrive_expect_tx(bar(&bars->full[st]), stage_bytes(NB));
       tma_load_2d(dst, &map_a, bar(&bars->full[st]), a_col + kb * kBK, a_row);
       tma_load_2d(dst + kABytes, &map_b, bar(&bars->full[st]), b_col + lo * g.b_lo_col + kb * kBK,
                   b_row);
+      if (HILO)
+        tma_load_2d(dst + kABytes + b_bytes(BN), &map_b, bar(&bars->full[st]),
+                    b_col + g.b_lo_col + kb * kBK, b_row);
     }
   } else if (warp == 1 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
@@ -192,7 +200,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       ok = mbar_wait(bar(&bars->full[st]), use & 1, abort_word, g.error_word, 12);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t a_smem = base + st * stage_bytes(BN), b_smem = a_smem + kABytes;
+      const uint32_t a_smem = base + st * stage_bytes(NB), b_smem = a_smem + kABytes;
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
         const uint64_t ad = make_smem_desc(a_smem + ks * 32, 16, 1024, kSwizzle128B);
@@ -240,12 +248,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (j0 + j < g.n) put(p + (long long)(j0 + j) * g.c_sn, g.alpha * __uint_as_float(v[j]));
         }
       };
+      // Accumulator columns c0 .. c0 + CH of this thread's row (hi and lo products added).
+      auto load_acc = [&](int c0, uint32_t (&v)[32]) {
+        if (CH == 32) tmem_ld_x32(lane_base + c0, v); else tmem_ld_x16(lane_base + c0, v);
+        if (HILO) {
+          uint32_t w[32];
+          if (CH == 32) tmem_ld_x32(lane_base + BN + c0, w); else tmem_ld_x16(lane_base + BN + c0, w);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < CH; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+        } else {
+          tmem_wait_ld();
+        }
+      };
       if (g.n_split == 1) {
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += CH) {
           uint32_t v[32];
-          if (CH == 32) tmem_ld_x32(lane_base + c0, v); else tmem_ld_x16(lane_base + c0, v);
-          tmem_wait_ld();
+          load_acc(c0, v);
           emit(v, c0);
         }
       } else {
@@ -253,8 +273,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
         for (int c0 = 0; c0 < BN; c0 += CH) {
           uint32_t v[32];
-          if (CH == 32) tmem_ld_x32(lane_base + c0, v); else tmem_ld_x16(lane_base + c0, v);
-          tmem_wait_ld();
+          load_acc(c0, v);
 #pragma unroll
           for (int j = 0; j < CH; ++j) part[(c0 + j) * kBM + row_local] = __uint_as_float(v[j]);
         }

@@ -267,16 +267,16 @@ int make_map_2d(CUtensorMap* map, const void* ptr, long long rows, long long col
   return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
-template <int BN, int STAGES, typename OutT>
+template <int BN, int STAGES, typename OutT, bool HILO>
 int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
                         const GemmTcArgs& g, dim3 grid, cudaStream_t st) {
-  constexpr int smem = gtc::smem_bytes(BN, STAGES);
+  constexpr int smem = gtc::smem_bytes(HILO ? 2 * BN : BN, STAGES);
   if (!(h->gemm_attr_mask & (1u << inst))) {
-    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT>,
+    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     h->gemm_attr_mask |= 1u << inst;
   }
-  gemm_tc_kernel<BN, STAGES, OutT><<<grid, 192, smem, st>>>(ma, mb, g);
+  gemm_tc_kernel<BN, STAGES, OutT, HILO><<<grid, 192, smem, st>>>(ma, mb, g);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
   return MTLA_OK;
@@ -293,9 +293,12 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   g.n_tiles = ceil_div(g.n, bn);
   const long long tiles = (long long)m_tiles * g.n_tiles * batches;
   const int kb_total = ceil_div(g.k, gtc::kBK);
+  // Stacked hi / lo halves double the B tile: one CTA per SM then, two otherwise.
+  const bool hilo = g.b_lo_col > 0 && bn <= 128 && sizeof(OutT) == 2;
+  const int slots = (hilo && bn == 128) || bn == 256 ? kSmCount : kGemmSlots;
   int n_split = 1;
-  if (allow_split && tiles < kGemmSlots)
-    n_split = max(1, min(kb_total / 4, (int)(kGemmSlots / tiles)));
+  // The partials are summed by the last CTA of a tile alone: at most four splits keep that short.
+  if (allow_split && tiles < slots) n_split = max(1, min(min(kb_total / 4, (int)(slots / tiles)), 4));
   g.kb_per_split = ceil_div(kb_total, n_split);
   g.n_split = ceil_div(kb_total, g.kb_per_split);
   g.partial = h->at<float>(h->plan.gemm_part);
@@ -309,12 +312,23 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
               g.c_sn * osz % 16 == 0 && g.c_sz * osz % 16 == 0 && g.c_lo_off * osz % 8 == 0;
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
+  if constexpr (sizeof(OutT) == 2) {
+    if (hilo) {
+      switch (bn) {
+        case 16: return launch_gemm_tc_inst<16, 4, OutT, true>(h, 10, ma, mb, g, grid, st);
+        case 32: return launch_gemm_tc_inst<32, 4, OutT, true>(h, 11, ma, mb, g, grid, st);
+        case 64: return launch_gemm_tc_inst<64, 3, OutT, true>(h, 12, ma, mb, g, grid, st);
+        case 128: return launch_gemm_tc_inst<128, 4, OutT, true>(h, 13, ma, mb, g, grid, st);
+        default: return MTLA_ERR_UNSUPPORTED_SHAPE;
+      }
+    }
+  }
   switch (bn) {
-    case 16: return launch_gemm_tc_inst<16, 4, OutT>(h, 0 + o, ma, mb, g, grid, st);
-    case 32: return launch_gemm_tc_inst<32, 4, OutT>(h, 2 + o, ma, mb, g, grid, st);
-    case 64: return launch_gemm_tc_inst<64, 4, OutT>(h, 4 + o, ma, mb, g, grid, st);
-    case 128: return launch_gemm_tc_inst<128, 3, OutT>(h, 6 + o, ma, mb, g, grid, st);
-    case 256: return launch_gemm_tc_inst<256, 4, OutT>(h, 8 + o, ma, mb, g, grid, st);
+    case 16: return launch_gemm_tc_inst<16, 4, OutT, false>(h, 0 + o, ma, mb, g, grid, st);
+    case 32: return launch_gemm_tc_inst<32, 4, OutT, false>(h, 2 + o, ma, mb, g, grid, st);
+    case 64: return launch_gemm_tc_inst<64, 4, OutT, false>(h, 4 + o, ma, mb, g, grid, st);
+    case 128: return launch_gemm_tc_inst<128, 3, OutT, false>(h, 6 + o, ma, mb, g, grid, st);
+    case 256: return launch_gemm_tc_inst<256, 4, OutT, false>(h, 8 + o, ma, mb, g, grid, st);
     default: return MTLA_ERR_UNSUPPORTED_SHAPE;
   }
 }
