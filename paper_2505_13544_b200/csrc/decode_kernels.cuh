@@ -9,9 +9,14 @@
 
 namespace mtla {
 
-// Column offsets of the fused input projection output row: [ q | q^R | c_raw | k^R ].
+// Column offsets of the fused input projection output row: [ q | q^R | c_raw | k^R | u_hi | u_lo ].
+// The last two blocks (d_w columns each, off_u < 0 when absent) are the hyper-network's
+// Linear(c_i) of Eq. 13 folded through the LayerNorm into the projection:
+//   c A + a = rstd * (c_raw (gamma .* A) - mean * (gamma^T A)) + (beta^T A + a),
+// and c_raw (gamma .* A) = x (W_r diag(gamma) A) = u, one more block of the fused product
+// (its weights kept as bf16 hi + lo halves, so u carries fp32-like precision).
 struct ProjLayout {
-  int off_q, off_qr, off_c, off_kr, width;
+  int off_q, off_qr, off_c, off_kr, off_u, width;
 };
 
 struct PostArgs {
@@ -22,6 +27,8 @@ struct PostArgs {
   const float* hyp_c_w;   // [r][d_w] fp32
   const float* hyp_c_b;   // [d_w]
   const float* gate_pe;   // [d_w]: Linear(pe_j) of Eq. 13 for this step's slot number j
+  const float* gate_s;    // [d_w]: gamma^T A        (folded gate only)
+  const float* gate_t;    // [d_w]: beta^T A + a     (folded gate only)
   const float* rope_cos;  // [d_R/2] for this step's position
   const float* rope_sin;  // [d_R/2]
   float* open_acc;        // [B][r] fp32 running sum of the open slot
@@ -91,6 +98,20 @@ __device__ inline float gate_weight(const float* c, const float* hyp_w, const fl
   return 1.f / (1.f + expf(-logit));
 }
 
+// The same weight from the folded projection block u (see ProjLayout): no matrix is read.
+__device__ inline float gate_weight_folded(const float* u, int dw, float mean, float rstd,
+                                           const float* gate_s, const float* gate_t,
+                                           const float* gate_pe, float* red) {
+  const int tid = threadIdx.x;
+  float prod = 0.f;
+  if (tid < dw) {
+    const float h = rstd * (u[tid] + u[dw + tid] - mean * gate_s[tid]) + gate_t[tid];
+    prod = h * gate_pe[tid];
+  }
+  const float logit = block_sum(prod, red);
+  return 1.f / (1.f + expf(-logit));
+}
+
 // One CTA of 256 threads per sequence.  Section 4.1: c_i = LayerNorm(x_i W_r); Eq. 13 gate;
 // slot update (open: c_hat_j = w c, else c_hat_j += w c); Section 4.3: RoPE key replaces
 // the slot's key, RoPE queries are rotated and written behind the absorbed query.
@@ -122,8 +143,11 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   __syncthreads();
 
   // Hyper-network gate: w = sigmoid(<c A + a, Linear(pe_j)>).
-  const float w = a.use_gate ? gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, a.gate_pe, a.r, a.dw, part_s, red_s)
-                             : 1.f;
+  float w = 1.f;
+  if (a.use_gate)
+    w = a.proj.off_u >= 0
+            ? gate_weight_folded(row + a.proj.off_u, a.dw, mean, rstd, a.gate_s, a.gate_t, a.gate_pe, red_s)
+            : gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, a.gate_pe, a.r, a.dw, part_s, red_s);
 
   // Slot update: fp32 running sum, stored to the cache in the storage type.
   const int W = a.r + a.dr;

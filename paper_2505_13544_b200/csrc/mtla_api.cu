@@ -37,6 +37,7 @@ int act_box_rows(int B) {
 struct ArenaPlan {
   size_t wcat_t, w_k, w_kv_t, w_o_t;
   size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
+  size_t gate_s, gate_t, gate_tmp;
   size_t cache, open_acc, err_flag;
   size_t p1, q16, qt, o_part, ml_part, o, v, x_stage, y_stage, gemm_part, gemm_tickets, attn_tickets;
   size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
@@ -76,6 +77,12 @@ bool normalise(const mtla_config* in, mtla_config* out, Dims* dm) {
   dm->proj.off_c = dm->proj.off_qr + dm->nh * dm->dr;
   dm->proj.off_kr = dm->proj.off_c + dm->r;
   dm->proj.width = dm->proj.off_kr + dm->dr;
+  // bf16 layers with a gate (s > 1) carry the folded Linear(c_i) as 2 d_w more output columns.
+  dm->proj.off_u = -1;
+  if (c.dtype == MTLA_DTYPE_BF16 && c.stride > 1) {
+    dm->proj.off_u = dm->proj.width;
+    dm->proj.width += 2 * dm->dw;
+  }
   dm->ntot = dm->proj.width;
   dm->max_slots = ceil_div(c.max_tokens, c.stride);
   dm->max_units = kTargetCtas + c.max_batch;
@@ -102,6 +109,9 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->hyp_pe_w = take((size_t)dm.r * dm.dw * 4);
   p->hyp_pe_b = take(dm.dw * 4);
   p->gate_pe = take((size_t)dm.max_slots * dm.dw * 4);
+  p->gate_s = take(dm.dw * 4);
+  p->gate_t = take(dm.dw * 4);
+  p->gate_tmp = take(dm.proj.off_u >= 0 ? ((size_t)dm.dw * dm.r + (size_t)dm.dw * dm.d) * 4 : 0);
   p->rope_cos = take((size_t)c.max_tokens * (dm.dr / 2) * 4);
   p->rope_sin = take((size_t)c.max_tokens * (dm.dr / 2) * 4);
   p->cache = take(B * dm.max_slots * dm.W * e);
@@ -397,6 +407,27 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   MTLA_TRY(launch_widen<T>(h, w->hyp_c_b, h->at<float>(p.hyp_c_b), dm.dw, st));
   MTLA_TRY(launch_widen<T>(h, w->hyp_pe_w, h->at<float>(p.hyp_pe_w), (long long)dm.r * dm.dw, st));
   MTLA_TRY(launch_widen<T>(h, w->hyp_pe_b, h->at<float>(p.hyp_pe_b), dm.dw, st));
+  if (dm.proj.off_u >= 0) {
+    // W_g^T = (gamma .* A)^T W_r^T as two bf16 row blocks behind the projection's other rows.
+    float* ga = h->at<float>(p.gate_tmp);
+    float* wg = ga + (size_t)dm.dw * dm.r;
+    gate_fold_scale_kernel<<<ceil_div(dm.r * dm.dw, 256), 256, 0, st>>>(
+        h->at<float>(p.hyp_c_w), h->at<float>(p.gamma), ga, dm.r, dm.dw);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+    MTLA_TRY((gemm<float, T, float>(h, ga, w->w_r, wg, dm.dw, dm.d, dm.r, dm.r, dm.r, dm.d, 1.f, 1,
+                                    0, 0, 0, st)));
+    const long long n_wg = (long long)dm.dw * dm.d;
+    gate_fold_pack_kernel<<<(unsigned)((n_wg + 255) / 256), 256, 0, st>>>(
+        wg, h->at<bf16>(p.wcat_t) + (size_t)dm.proj.off_u * dm.d, dm.dw, dm.d);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+    gate_fold_vectors_kernel<<<ceil_div(dm.dw, 128), 128, 0, st>>>(
+        h->at<float>(p.hyp_c_w), h->at<float>(p.hyp_c_b), h->at<float>(p.gamma),
+        h->at<float>(p.beta), h->at<float>(p.gate_s), h->at<float>(p.gate_t), dm.r, dm.dw);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
   gate_pe_table_kernel<<<dm.max_slots, 256, 0, st>>>(h->at<float>(p.hyp_pe_w), h->at<float>(p.hyp_pe_b),
                                                      h->at<float>(p.gate_pe), dm.r, dm.dw);
   h->launches++;
@@ -521,6 +552,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   pa.hyp_c_w = h->at<float>(p.hyp_c_w);
   pa.hyp_c_b = h->at<float>(p.hyp_c_b);
   pa.gate_pe = h->at<float>(p.gate_pe) + (size_t)slot * dm.dw;
+  pa.gate_s = h->at<float>(p.gate_s);
+  pa.gate_t = h->at<float>(p.gate_t);
   pa.rope_cos = h->at<float>(p.rope_cos) + (size_t)i0 * (dm.dr / 2);
   pa.rope_sin = h->at<float>(p.rope_sin) + (size_t)i0 * (dm.dr / 2);
   pa.open_acc = h->at<float>(p.open_acc);
@@ -643,6 +676,8 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   pa.hyp_c_w = h->at<float>(p.hyp_c_w);
   pa.hyp_c_b = h->at<float>(p.hyp_c_b);
   pa.gate_pe = h->at<float>(p.gate_pe);
+  pa.gate_s = h->at<float>(p.gate_s);
+  pa.gate_t = h->at<float>(p.gate_t);
   pa.rope_cos = h->at<float>(p.rope_cos);
   pa.rope_sin = h->at<float>(p.rope_sin);
   pa.open_acc = h->at<float>(p.open_acc);

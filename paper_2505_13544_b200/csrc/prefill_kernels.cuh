@@ -17,6 +17,8 @@ struct PrefillPostArgs {
   const float* hyp_c_w;   // [r][d_w]
   const float* hyp_c_b;   // [d_w]
   const float* gate_pe;   // [max_slots][d_w]; row j0 is Linear(pe_{j0+1})
+  const float* gate_s;    // [d_w], [d_w]: constants of the folded gate (see ProjLayout)
+  const float* gate_t;
   const float* rope_cos;  // [max_tokens][d_R/2]
   const float* rope_sin;
   float* open_acc;        // [B][r]
@@ -67,8 +69,11 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
       c_s[i] = (c_s[i] - mean) * rstd * a.gamma[i] + a.beta[i];
     __syncthreads();
 
-    const float w = a.use_gate ? gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, gate_pe, a.r, a.dw, part_s, red_s)
-                               : 1.f;
+    float w = 1.f;
+    if (a.use_gate)
+      w = a.proj.off_u >= 0
+              ? gate_weight_folded(row + a.proj.off_u, a.dw, mean, rstd, a.gate_s, a.gate_t, gate_pe, red_s)
+              : gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, gate_pe, a.r, a.dw, part_s, red_s);
 
     T* cp = static_cast<T*>(a.cprime) + rowi * a.r;
     for (int i = tid; i < a.r; i += 256) {

@@ -31,6 +31,42 @@ __global__ void widen_kernel(const T* src, float* dst, long long n) {
   if (i < n) dst[i] = src ? Elem<T>::to_float(src[i]) : 0.f;
 }
 
+// Folding Linear(c_i) of Eq. 13 into the input projection (see ProjLayout).
+// ga[n][i] = gamma[i] * A[i][n]: the [d_w][r] left operand of W_g^T = ga . W_r^T.
+__global__ void gate_fold_scale_kernel(const float* a /*[r][d_w]*/, const float* gamma, float* ga,
+                                       int r, int dw) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= r * dw) return;
+  const int n = idx / r, i = idx % r;
+  ga[idx] = gamma[i] * a[(long long)i * dw + n];
+}
+
+// Splits W_g^T [d_w][d] (fp32) into bf16 halves: rows [0, d_w) of dst receive the rounded
+// values, rows [d_w, 2 d_w) the rounding remainders.
+__global__ void gate_fold_pack_kernel(const float* wg, bf16* dst, int dw, long long d) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= dw * d) return;
+  const bf16 hi = __float2bfloat16_rn(wg[idx]);
+  dst[idx] = hi;
+  dst[dw * d + idx] = __float2bfloat16_rn(wg[idx] - __bfloat162float(hi));
+}
+
+// gate_s[n] = sum_i gamma[i] A[i][n];  gate_t[n] = sum_i beta[i] A[i][n] + a[n].
+__global__ void gate_fold_vectors_kernel(const float* a /*[r][d_w]*/, const float* bias,
+                                         const float* gamma, const float* beta, float* gate_s,
+                                         float* gate_t, int r, int dw) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= dw) return;
+  double s = 0.0, t = bias[n];
+  for (int i = 0; i < r; ++i) {
+    const double w = a[(long long)i * dw + n];
+    s += gamma[i] * w;
+    t += beta[i] * w;
+  }
+  gate_s[n] = (float)s;
+  gate_t[n] = (float)t;
+}
+
 // Row j0 of the table is Linear(pe_j) of Eq. 13 for the 1-based slot number j = j0 + 1:
 // pe_j is the sinusoidal embedding of dimension r (sin at even, cos at odd indices,
 // wavelengths 10000^(2k/r)), evaluated in fp64.  One CTA per slot number.
