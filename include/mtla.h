@@ -177,9 +177,12 @@ int64_t mtla_launch_count(const mtla_handle* h);
  * that streams the cache), 4 cross-split combine, 5 value up-projection (Eq. 10), 6 output
  * projection (Eq. 11).  mtla_profile_end_stages waits for those events, returns the summed
  * duration of every stage in milliseconds (stage_ms host [MTLA_DECODE_STAGES]) and the number
- * of steps covered, and releases the events; mtla_profile_end returns the attention stage only. */
+ * of steps covered, and releases the events; mtla_profile_end returns the attention stage only.
+ * mtla_profile_begin_attention records only the two events around the attention kernel (the
+ * other stages then read 0), which perturbs a timed loop least. */
 enum { MTLA_DECODE_STAGES = 7, MTLA_STAGE_ATTENTION = 3 };
 int mtla_profile_begin(mtla_handle* h, int32_t max_steps);
+int mtla_profile_begin_attention(mtla_handle* h, int32_t max_steps);
 int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps);
 int mtla_profile_end_stages(mtla_handle* h, double* stage_ms, int32_t* steps);
 

@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
     "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
     "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
-    "mtla_profile_end_stages", "mtla_decode_step_static")
+    "mtla_profile_end_stages", "mtla_decode_step_static", "mtla_profile_begin_attention")
 
 DECODE_STAGES = ("input_proj", "norm_gate_update", "absorb", "attention", "combine", "value_proj",
                  "output_proj")
@@ -80,6 +80,7 @@ def load_library() -> ctypes.CDLL:
         "mtla_launch_count": (ctypes.c_int64, [vp]),
         "mtla_attention_variant": (ctypes.c_char_p, [vp]),
         "mtla_profile_begin": (ctypes.c_int, [vp, i32]),
+        "mtla_profile_begin_attention": (ctypes.c_int, [vp, i32]),
         "mtla_profile_end": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(i32)]),
         "mtla_profile_end_stages": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
@@ -275,6 +276,11 @@ def mtla_attention_variant(h: Handle) -> str:
 
 def mtla_profile_begin(h: Handle, max_steps: int) -> None:
     _check(load_library().mtla_profile_begin(h.ptr, max_steps), "mtla_profile_begin")
+
+
+def mtla_profile_begin_attention(h: Handle, max_steps: int) -> None:
+    _check(load_library().mtla_profile_begin_attention(h.ptr, max_steps),
+           "mtla_profile_begin_attention")
 
 
 def mtla_profile_end(h: Handle) -> tuple[float, int]:

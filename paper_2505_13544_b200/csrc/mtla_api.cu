@@ -14,6 +14,7 @@
 #include "decode_kernels.cuh"
 #include "gemm_fma.cuh"
 #include "gemm_tc.cuh"
+#include "prefill_attn_tc.cuh"
 #include "prefill_kernels.cuh"
 #include "setup_kernels.cuh"
 
@@ -173,6 +174,7 @@ struct mtla_handle {
   // Optional timing of the decode step's kernels: MTLA_DECODE_STAGES + 1 events per profiled step.
   std::vector<cudaEvent_t> prof_events;
   int prof_used;
+  bool prof_attention_only;   // record only the two events around the attention kernel
 
   template <typename P> P* at(size_t off) const { return reinterpret_cast<P*>(arena + off); }
 };
@@ -271,6 +273,23 @@ int make_map_2d(CUtensorMap* map, const void* ptr, long long rows, long long col
   const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims,
+                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
+}
+
+// TMA view of bf16 data as [n2][n1][cols] with element strides ld1 / ld2 between rows / planes:
+// boxes of box_rows rows x 64 columns, 128-byte swizzle, zero fill outside.
+int make_map_3d(CUtensorMap* map, const void* ptr, long long cols, long long n1, long long n2,
+                long long ld1, long long ld2, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return MTLA_ERR_CUDA;
+  const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)n1, (cuuint64_t)n2};
+  const cuuint64_t strides[2] = {(cuuint64_t)ld1 * 2, (cuuint64_t)ld2 * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims,
                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -511,6 +530,8 @@ struct AttnScratch {
 // Records the event that closes stage `stage - 1` / opens stage `stage` of a profiled step.
 int prof_mark(mtla_handle* h, bool prof, int stage, cudaStream_t st) {
   if (!prof) return MTLA_OK;
+  if (h->prof_attention_only && stage != MTLA_STAGE_ATTENTION && stage != MTLA_STAGE_ATTENTION + 1)
+    return MTLA_OK;
   MTLA_CUDA(cudaEventRecord(h->prof_events[h->prof_used + stage], st));
   return MTLA_OK;
 }
@@ -690,7 +711,8 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = q_scale;
-  prefill_post_kernel<T, float><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
+  if (h->use_tc) prefill_post_kernel<T, bf16><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
+  else prefill_post_kernel<T, float><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
   if (!y) return MTLA_OK;
@@ -699,44 +721,80 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   if (h->use_tc) {
     CUtensorMap map_c;
     MTLA_TRY(make_map_2d(&map_c, h->at<void>(p.pf_cprime), rows, dm.r, dm.r, kPrefillBn));
-    MTLA_TRY(gemm_tc<float>(h, h->map_wkvt, map_c,
-                            gemm_tc_args(h->at<float>(p.pf_kv), 1, 2 * hd, 2 * hd, rows, dm.r, 1.f),
-                            kPrefillBn, 1, false, st));
-  } else {
-    MTLA_TRY((gemm<T, T, float>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<float>(p.pf_kv),
-                                rows, 2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
-  }
-  PrefillAttnArgs aa;
-  aa.qcat = pa.qcat; aa.kv = h->at<void>(p.pf_kv); aa.kr = pa.kr; aa.out = h->at<void>(p.pf_attn);
-  aa.n_heads = dm.nh; aa.dr = dm.dr; aa.stride = dm.s; aa.T = T_len;
-  const size_t smem = prefill_attn_fma_smem_bytes(dm.dh, dm.dr);
-  dim3 grid(ceil_div(T_len, kPfTile), dm.nh, B);
-#define MTLA_PF_ATTN(TOUT, DH)                                                               \
-  do {                                                                                       \
-    if (!h->pf_smem_ready)                                                                   \
-      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, TOUT, DH>,               \
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    prefill_attn_fma_kernel<float, TOUT, DH><<<grid, 256, smem, st>>>(aa);                   \
-  } while (0)
-  if (h->use_tc) {
-    if (dm.dh == 64) MTLA_PF_ATTN(bf16, 64); else MTLA_PF_ATTN(bf16, 128);
-  } else {
-    if (dm.dh == 64) MTLA_PF_ATTN(float, 64); else MTLA_PF_ATTN(float, 128);
-  }
-#undef MTLA_PF_ATTN
-  h->pf_smem_ready = true;
-  h->launches++;
-  MTLA_CUDA(cudaGetLastError());
-  if (h->use_tc) {
+    // Keys and values as bf16, followed by their rounding remainders: rows of 4 n_h d_h.
+    GemmTcArgs gkv = gemm_tc_args(h->at<bf16>(p.pf_kv), 1, 4 * hd, 2 * hd, rows, dm.r, 1.f);
+    gkv.c_lo_off = 2 * hd;
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wkvt, map_c, gkv, kPrefillBn, 1, false, st));
+    // Attention on the tensor cores; the closed slots are a strided view of the token rows.
+    const int DQ = dm.dh + dm.dr, kt = pft::key_tile(dm.dh);
+    const int n_slots_closed = T_len / dm.s;
+    const bf16* kv = h->at<bf16>(p.pf_kv);
+    const bf16* kr = h->at<bf16>(p.pf_kr);
+    CUtensorMap q_map, kv_closed, kv_self, kr_closed, kr_self;
+    MTLA_TRY(make_map_3d(&q_map, h->at<void>(p.pf_qcat), (long long)dm.nh * DQ, T_len, B,
+                         (long long)dm.nh * DQ, (long long)T_len * dm.nh * DQ, pft::kQTile));
+    MTLA_TRY(make_map_3d(&kv_self, kv, 4 * hd, T_len, B, 4 * hd, (long long)T_len * 4 * hd, kt));
+    MTLA_TRY(make_map_3d(&kr_self, kr, dm.dr, T_len, B, dm.dr, (long long)T_len * dm.dr, kt));
+    if (n_slots_closed > 0) {
+      MTLA_TRY(make_map_3d(&kv_closed, kv + (size_t)(dm.s - 1) * 4 * hd, 4 * hd, n_slots_closed, B,
+                           (long long)dm.s * 4 * hd, (long long)T_len * 4 * hd, kt));
+      MTLA_TRY(make_map_3d(&kr_closed, kr + (size_t)(dm.s - 1) * dm.dr, dm.dr, n_slots_closed, B,
+                           (long long)dm.s * dm.dr, (long long)T_len * dm.dr, kt));
+    } else {
+      kv_closed = kv_self;   // never read: a prompt shorter than the stride closes no slot
+      kr_closed = kr_self;
+    }
+    PrefillAttnTcArgs ta;
+    ta.out = h->at<bf16>(p.pf_attn);
+    ta.error_word = h->at<int>(p.err_flag);
+    ta.n_heads = dm.nh; ta.dr = dm.dr; ta.stride = dm.s; ta.T = T_len;
+    dim3 grid(ceil_div(T_len, pft::kQTile), dm.nh, B);
+    if (dm.dh == 64) {
+      if (!h->pf_smem_ready)
+        MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_tc_kernel<64>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, pft::smem_bytes(64)));
+      prefill_attn_tc_kernel<64><<<grid, pft::kThreads, pft::smem_bytes(64), st>>>(
+          q_map, kv_closed, kv_self, kr_closed, kr_self, ta);
+    } else {
+      if (!h->pf_smem_ready)
+        MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_tc_kernel<128>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, pft::smem_bytes(128)));
+      prefill_attn_tc_kernel<128><<<grid, pft::kThreads, pft::smem_bytes(128), st>>>(
+          q_map, kv_closed, kv_self, kr_closed, kr_self, ta);
+    }
+    h->pf_smem_ready = true;
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
     CUtensorMap map_a;
     MTLA_TRY(make_map_2d(&map_a, h->at<void>(p.pf_attn), rows, 2 * hd, 2 * hd, kPrefillBn));
     GemmTcArgs g = gemm_tc_args(y, 1, dm.d, dm.d, rows, hd, 1.f);
     g.b_lo_col = hd;
     MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, map_a, g, kPrefillBn, 1, false, st));
-  } else {
-    MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd,
-                                hd, dm.d, 1.f, 1, 0, 0, 0, st)));
+    return MTLA_OK;
   }
+  MTLA_TRY((gemm<T, T, float>(h, h->at<T>(p.pf_cprime), h->at<T>(p.w_kv_t), h->at<float>(p.pf_kv),
+                              rows, 2 * hd, dm.r, dm.r, dm.r, 2 * hd, 1.f, 1, 0, 0, 0, st)));
+  PrefillAttnArgs aa;
+  aa.qcat = pa.qcat; aa.kv = h->at<void>(p.pf_kv); aa.kr = pa.kr; aa.out = h->at<void>(p.pf_attn);
+  aa.n_heads = dm.nh; aa.dr = dm.dr; aa.stride = dm.s; aa.T = T_len;
+  const size_t smem = prefill_attn_fma_smem_bytes(dm.dh, dm.dr);
+  dim3 grid(ceil_div(T_len, kPfTile), dm.nh, B);
+  if (dm.dh == 64) {
+    if (!h->pf_smem_ready)
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, float, 64>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    prefill_attn_fma_kernel<float, float, 64><<<grid, 256, smem, st>>>(aa);
+  } else {
+    if (!h->pf_smem_ready)
+      MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_fma_kernel<float, float, 128>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    prefill_attn_fma_kernel<float, float, 128><<<grid, 256, smem, st>>>(aa);
+  }
+  h->pf_smem_ready = true;
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.pf_attn), h->at<T>(p.w_o_t), y, rows, dm.d, hd, hd,
+                              hd, dm.d, 1.f, 1, 0, 0, 0, st)));
   return MTLA_OK;
 }
 
@@ -784,6 +842,7 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   h->tokens = 0; h->batch = 0; h->launches = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
+  h->prof_attention_only = false;
   h->act_bn = 0;
   h->gemm_attr_mask = 0;
   // The tensor-core attention needs bf16 and whole 128-column latent blocks; the
@@ -957,8 +1016,15 @@ int mtla_check(mtla_handle* h, void* stream) {
 
 int64_t mtla_launch_count(const mtla_handle* h) { return h ? h->launches : 0; }
 
+int mtla_profile_begin_attention(mtla_handle* h, int32_t max_steps) {
+  const int rc = mtla_profile_begin(h, max_steps);
+  if (rc == MTLA_OK) h->prof_attention_only = true;
+  return rc;
+}
+
 int mtla_profile_begin(mtla_handle* h, int32_t max_steps) {
   if (!h || max_steps <= 0) return MTLA_ERR_INVALID_ARG;
+  h->prof_attention_only = false;
   for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
   h->prof_events.clear();
   h->prof_used = 0;
@@ -977,6 +1043,7 @@ int mtla_profile_end_stages(mtla_handle* h, double* stage_ms, int32_t* steps) {
   for (int i = 0; i + per_step <= h->prof_used; i += per_step) {
     MTLA_CUDA(cudaEventSynchronize(h->prof_events[i + MTLA_DECODE_STAGES]));
     for (int s = 0; s < MTLA_DECODE_STAGES; ++s) {
+      if (h->prof_attention_only && s != MTLA_STAGE_ATTENTION) continue;
       float ms = 0.f;
       MTLA_CUDA(cudaEventElapsedTime(&ms, h->prof_events[i + s], h->prof_events[i + s + 1]));
       stage_ms[s] += ms;
