@@ -232,20 +232,33 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
       tc_fence_after_sync();
       const bool diag = t >= n_kv;
       const int col0 = diag ? (t - n_kv) * KT : t * KT;     // key index of column 0 (slot, or row offset)
-      // Pass 1: the tile's row maximum under the mask.
-      float s[KT];
-      float mt = -INFINITY;
+      // The tile's scores of this row, then the mask as a predicate on the column index:
+      // closed slots below `lim`, or the row's own column `own` in a diagonal pass.
+      const int lim = diag ? 0 : closed - col0;
+      const int own = (diag && m < a.T) ? row - col0 : -1;
+      uint32_t sv[KT];
 #pragma unroll
       for (int c0 = 0; c0 < KT; c0 += 32) {
-        uint32_t v[32];
+        uint32_t(&v)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sv[c0]);
         tmem_ld_x32(lane_base + (t & 1) * KT + c0, v);
-        tmem_wait_ld();
+      }
+      tmem_wait_ld();
+      float s[KT];
+      float mt = -INFINITY;
+      if (__all_sync(0xffffffffu, lim >= KT)) {
+        // Every column of the tile is visible to every row of this warp: no predicate needed.
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int key = col0 + c0 + j;
-          const bool allowed = diag ? (key == row && m < a.T) : (key < closed);
-          s[c0 + j] = allowed ? __uint_as_float(v[j]) : -INFINITY;
-          mt = fmaxf(mt, s[c0 + j]);
+        for (int c = 0; c < KT; ++c) {
+          s[c] = __uint_as_float(sv[c]);
+          mx[c & 3] = fmaxf(mx[c & 3], s[c]);
+        }
+        mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      } else {
+#pragma unroll
+        for (int c = 0; c < KT; ++c) {
+          s[c] = (c < lim || c == own) ? __uint_as_float(sv[c]) : -INFINITY;
+          mt = fmaxf(mt, s[c]);
         }
       }
       tc_fence_before_sync();
@@ -276,12 +289,15 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
       m_run = m_new;
       const float m_eff = m_run == -INFINITY ? 0.f : m_run;   // a row that has seen nothing yet
       uint32_t pk[KT / 2];
+      float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < KT; c += 2) {
-        const __nv_bfloat162 two = __floats2bfloat162_rn(ex2_approx(s[c] - m_eff), ex2_approx(s[c + 1] - m_eff));
-        l_run += __low2float(two) + __high2float(two);
+        const float p0 = ex2_approx(s[c] - m_eff), p1 = ex2_approx(s[c + 1] - m_eff);
+        lsum[(c >> 1) & 3] += p0 + p1;
+        const __nv_bfloat162 two = __floats2bfloat162_rn(p0, p1);
         pk[c / 2] = *reinterpret_cast<const uint32_t*>(&two);
       }
+      l_run += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
       // The single probability buffer is free once the previous tile's value MMAs have completed.
       ok = mbar_wait(bar(&bars->p_empty), (t & 1) ^ 1, abort_word, a.error_word, 28);
       ok = __all_sync(0xffffffffu, ok);
