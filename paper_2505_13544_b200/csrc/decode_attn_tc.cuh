@@ -202,10 +202,12 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     prefetch_tensormap(&q_map);
   }
   if (warp == 1) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
+  grid_launch_dependents();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = misc->tmem_base;
+  grid_dependency_wait();        // nothing before this line touches the previous kernel's data
 
   // This CTA's share of the tile list.
   const long long tps = a.tiles_per_seq, total = (long long)a.batch * tps, G = gridDim.x;

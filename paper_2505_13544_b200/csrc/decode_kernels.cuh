@@ -123,6 +123,8 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   __shared__ float red_s[33];
   const int b = blockIdx.x, tid = threadIdx.x;
   const float* row = a.p1 + (long long)b * a.proj.width;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();   // the projection kernel's output is read from here on
 
   // LayerNorm over r (two-pass variance).
   float s = 0.f;

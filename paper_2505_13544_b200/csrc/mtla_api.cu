@@ -7,6 +7,7 @@
 #include <new>
 #include <stdlib.h>
 #include <string.h>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -296,18 +297,37 @@ int make_map_3d(CUtensorMap* map, const void* ptr, long long cols, long long n1,
   return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
+// Launches `kernel`; with `dependent` it may start its prologue while the previous kernel on
+// the stream is still running (programmatic dependent launch: the kernel itself waits, with
+// griddepcontrol.wait, before it touches that kernel's data).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                          cudaStream_t st, bool dependent, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 template <int BN, int STAGES, typename OutT, bool HILO>
 int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
-                        const GemmTcArgs& g, dim3 grid, cudaStream_t st) {
+                        const GemmTcArgs& g, dim3 grid, cudaStream_t st, bool dependent) {
   constexpr int smem = gtc::smem_bytes(HILO ? 2 * BN : BN, STAGES);
   if (!(h->gemm_attr_mask & (1u << inst))) {
     MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     h->gemm_attr_mask |= 1u << inst;
   }
-  gemm_tc_kernel<BN, STAGES, OutT, HILO><<<grid, 192, smem, st>>>(ma, mb, g);
+  MTLA_CUDA(launch_kernel(gemm_tc_kernel<BN, STAGES, OutT, HILO>, grid, dim3(192), smem, st,
+                          dependent, ma, mb, g));
   h->launches++;
-  MTLA_CUDA(cudaGetLastError());
   return MTLA_OK;
 }
 
@@ -316,7 +336,7 @@ int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const C
 // several CTAs when the tile count alone would leave most SMs idle.
 template <typename OutT>
 int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTcArgs g, int bn,
-            int batches, bool allow_split, cudaStream_t st) {
+            int batches, bool allow_split, cudaStream_t st, bool dependent = false) {
   const int m_tiles = ceil_div(g.m, gtc::kBM);
   g.m_tiles = m_tiles;
   g.n_tiles = ceil_div(g.n, bn);
@@ -344,20 +364,20 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   if constexpr (sizeof(OutT) == 2) {
     if (hilo) {
       switch (bn) {
-        case 16: return launch_gemm_tc_inst<16, 4, OutT, true>(h, 10, ma, mb, g, grid, st);
-        case 32: return launch_gemm_tc_inst<32, 4, OutT, true>(h, 11, ma, mb, g, grid, st);
-        case 64: return launch_gemm_tc_inst<64, 3, OutT, true>(h, 12, ma, mb, g, grid, st);
-        case 128: return launch_gemm_tc_inst<128, 4, OutT, true>(h, 13, ma, mb, g, grid, st);
+        case 16: return launch_gemm_tc_inst<16, 4, OutT, true>(h, 10, ma, mb, g, grid, st, dependent);
+        case 32: return launch_gemm_tc_inst<32, 4, OutT, true>(h, 11, ma, mb, g, grid, st, dependent);
+        case 64: return launch_gemm_tc_inst<64, 3, OutT, true>(h, 12, ma, mb, g, grid, st, dependent);
+        case 128: return launch_gemm_tc_inst<128, 4, OutT, true>(h, 13, ma, mb, g, grid, st, dependent);
         default: return MTLA_ERR_UNSUPPORTED_SHAPE;
       }
     }
   }
   switch (bn) {
-    case 16: return launch_gemm_tc_inst<16, 4, OutT, false>(h, 0 + o, ma, mb, g, grid, st);
-    case 32: return launch_gemm_tc_inst<32, 4, OutT, false>(h, 2 + o, ma, mb, g, grid, st);
-    case 64: return launch_gemm_tc_inst<64, 4, OutT, false>(h, 4 + o, ma, mb, g, grid, st);
-    case 128: return launch_gemm_tc_inst<128, 3, OutT, false>(h, 6 + o, ma, mb, g, grid, st);
-    case 256: return launch_gemm_tc_inst<256, 4, OutT, false>(h, 8 + o, ma, mb, g, grid, st);
+    case 16: return launch_gemm_tc_inst<16, 4, OutT, false>(h, 0 + o, ma, mb, g, grid, st, dependent);
+    case 32: return launch_gemm_tc_inst<32, 4, OutT, false>(h, 2 + o, ma, mb, g, grid, st, dependent);
+    case 64: return launch_gemm_tc_inst<64, 4, OutT, false>(h, 4 + o, ma, mb, g, grid, st, dependent);
+    case 128: return launch_gemm_tc_inst<128, 3, OutT, false>(h, 6 + o, ma, mb, g, grid, st, dependent);
+    case 256: return launch_gemm_tc_inst<256, 4, OutT, false>(h, 8 + o, ma, mb, g, grid, st, dependent);
     default: return MTLA_ERR_UNSUPPORTED_SHAPE;
   }
 }
@@ -370,7 +390,7 @@ GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, i
 }
 
 template <int NHP>
-int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_t st) {
+int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_t st, bool dependent) {
 #define MTLA_TC_CASE(RP)                                                                       \
   case RP:                                                                                     \
     if (!h->attn_smem_ready) {                                                                 \
@@ -384,8 +404,8 @@ int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_
       MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP>,                           \
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes)); \
     }                                                                                          \
-    decode_attn_tc_kernel<NHP, RP><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(h->cache_map,   \
-                                                                               h->q_map, a);   \
+    MTLA_CUDA(launch_kernel(decode_attn_tc_kernel<NHP, RP>, dim3(grid), dim3(tc::kThreads),    \
+                            tc::kSmemBytes, st, dependent, h->cache_map, h->q_map, a));        \
     break;
   switch (a.r / 128) {
     MTLA_TC_CASE(1)
@@ -397,7 +417,6 @@ int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_
 #undef MTLA_TC_CASE
   h->attn_smem_ready = true;
   h->launches++;
-  MTLA_CUDA(cudaGetLastError());
   return MTLA_OK;
 }
 
@@ -587,10 +606,16 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
-  if (h->use_tc) decode_post_kernel<T, bf16><<<B, 256, 0, st>>>(pa);
-  else decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
+  // On the tensor-core path every kernel after the first is a programmatic dependent launch:
+  // its prologue overlaps the tail of its predecessor (not while events sit between them).
+  const bool pdl = h->use_tc && !(prof && !h->prof_attention_only);
+  if (h->use_tc) {
+    MTLA_CUDA(launch_kernel(decode_post_kernel<T, bf16>, dim3(B), dim3(256), 0, st, pdl, pa));
+  } else {
+    decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
+    MTLA_CUDA(cudaGetLastError());
+  }
   h->launches++;
-  MTLA_CUDA(cudaGetLastError());
 
   MTLA_TRY(prof_mark(h, prof, 2, st));
   // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection
@@ -598,7 +623,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   if (h->use_tc) {
     GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.qt), 1, (long long)dm.nh * dm.W, dm.r, B, dm.dh, pa.q_scale);
     g.c_sz = dm.W; g.a_col_z = dm.dh; g.b_col_z = dm.dh; g.b_lo_col = hd;
-    MTLA_TRY(gemm_tc<bf16>(h, h->map_wk, h->map_q16, g, bn, dm.nh, true, st));
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wk, h->map_q16, g, bn, dm.nh, true, st, pdl));
   } else
     MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
                                     h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
@@ -625,8 +650,9 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     const long long total = (long long)B * ta.tiles_per_seq;
     const int grid = (int)(total < kSmCount ? total : kSmCount);
     aa.n_split = 0;
-    if (dm.nh <= 16) MTLA_TRY(launch_attn_tc_rp<16>(h, ta, grid, st));
-    else MTLA_TRY(launch_attn_tc_rp<32>(h, ta, grid, st));
+    const bool attn_pdl = pdl && !prof;     // the attention kernel is bracketed by events when timed
+    if (dm.nh <= 16) MTLA_TRY(launch_attn_tc_rp<16>(h, ta, grid, st, attn_pdl));
+    else MTLA_TRY(launch_attn_tc_rp<32>(h, ta, grid, st, attn_pdl));
   } else {
     int want = ceil_div(kTargetCtas, B);
     int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
@@ -651,11 +677,11 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   if (h->use_tc) {
     GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.v), 1, 2 * hd, dm.dh, B, dm.r, 1.f);
     g.c_sz = dm.dh; g.a_row_z = dm.dh; g.b_col_z = dm.r; g.b_lo_col = dm.nh * dm.r; g.c_lo_off = hd;
-    MTLA_TRY(gemm_tc<bf16>(h, h->map_wvt, h->map_o16, g, bn, dm.nh, true, st));
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wvt, h->map_o16, g, bn, dm.nh, true, st, pdl && !prof));
     MTLA_TRY(prof_mark(h, prof, 6, st));
     g = gemm_tc_args(y, 1, dm.d, dm.d, B, hd, 1.f);
     g.b_lo_col = hd;
-    MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, h->map_v16, g, bn, 1, true, st));
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, h->map_v16, g, bn, 1, true, st, pdl));
   } else {
     MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r,
                                     h->at<float>(p.v), B, dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f,

@@ -102,6 +102,17 @@ __device__ __forceinline__ void tc_fence_after_sync() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
+// Programmatic dependent launch.  grid_launch_dependents lets the next kernel on the stream
+// (if it was launched with programmatic stream serialization) begin its prologue once every CTA
+// of this grid has got here or exited; grid_dependency_wait blocks until the preceding grid has
+// completed and its memory is visible.  Both are no-ops for ordinary launches.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Per-warpgroup register re-allocation (all four warps of the warpgroup must execute it).
 template <int N>
 __device__ __forceinline__ void reg_alloc() {
