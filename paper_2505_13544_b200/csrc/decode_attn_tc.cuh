@@ -88,6 +88,7 @@ constexpr int kSubBytes = kTile * 128;     // one 64-column sub-tile
 constexpr int kPairBytes = 2 * kSubBytes;
 constexpr int kPairs = 9;
 constexpr int kKrBufs = 3;
+constexpr int kPrefetchAhead = 1;          // tiles asked into L2 ahead of the tile being loaded
 constexpr int kTmemCols = 512;
 constexpr int kSParts = 4;                 // independent partial score accumulators per buffer
 constexpr int kColS = 0;                   // score buffer b, partial k at column (b * 4 + k) * 32
@@ -225,11 +226,22 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     bool ok = true;
     int pc = 0, seg = 0;
     int b = (int)(g0 / tps), t = (int)(g0 - (long long)b * tps);
+    // The ring holds little more than two tiles, too few to cover the DRAM latency of a load
+    // that can only be issued once its slot is free.  So tiles are first asked into L2, a few
+    // tiles ahead; the load proper then finds them there.
+    auto prefetch_tile = [&](int n_ahead) {
+      if (n_ahead >= n_tiles) return;
+      const long long g = g0 + n_ahead;
+      const int pb = (int)(g / tps), slot = (int)(g - (long long)pb * tps) * kTile;
+      for (int c = 0; c < 2 * RP + 1; ++c) tma_prefetch_l2_3d(&cache_map, c * 64, slot, pb);
+    };
+    for (int n = 0; n < kPrefetchAhead; ++n) prefetch_tile(n);
     for (int n = 0; n < n_tiles && ok; ++n, ++t) {
       if (t == (int)tps) {
         t = 0;
         ++b;
       }
+      prefetch_tile(n + kPrefetchAhead);
       if (n == 0 || t == 0) {
         // A segment starts: q~ of sequence b, once the previous segment's score MMAs are done.
         ok = mbar_wait(bar(&misc->q_empty), (seg & 1) ^ 1, abort_word, a.error_word, 1);

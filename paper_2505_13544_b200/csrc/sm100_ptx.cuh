@@ -140,6 +140,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const CUtensorMap
       : "memory");
 }
 
+// Asks for the same box to be brought into L2 only (no shared memory, no barrier).
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+
 // 2-D form of the same load (c0 = column, c1 = row).
 __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* map,
                                             uint32_t bar, int c0, int c1) {
