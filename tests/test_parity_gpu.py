@@ -154,6 +154,37 @@ def test_cache_import_export_and_open_slot(dtype):
         M.mtla_destroy(h)
 
 
+@pytest.mark.parametrize("r,stride", [(64, 2), (192, 3), (320, 1)])
+def test_bf16_layers_off_the_tensor_core_shapes(r, stride):
+    """bf16 layers whose latent rank is not a multiple of 128 run on the CUDA-core kernels
+    (with the folded gate); prefill, hand-over and decode must still match the oracle."""
+    w = SMALL_BF16.scaled(latent_rank=r, hyper_dim=r // 4, stride=stride, prefill_tokens=75,
+                          decode_steps=5, batch=2)
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    prompt = synth.prompt(w)
+    xs = decode_inputs(w, w.decode_steps, w.batch)
+    h = H.gpu_handle(w, weights)
+    try:
+        assert M.mtla_attention_variant(h) == "fma"
+        y = M.mtla_prefill(h, prompt.cuda())
+        states = []
+        for b in range(w.batch):
+            want, st = O.decode_sequence(p, prompt[b].double().numpy())
+            H.assert_close(y[b], want, "bf16", f"prefill seq {b}")
+            states.append(st)
+        for i in range(w.decode_steps):
+            yd = M.mtla_decode_step(h, xs[i].cuda())
+            want = np.stack([O.decode_step(p, states[b], xs[i, b].double().numpy())
+                             for b in range(w.batch)])
+            H.assert_close(yd, want, "bf16", f"decode step {i}")
+        H.assert_cache_close(M.mtla_cache_export(h),
+                             np.stack([O.cache_array(st) for st in states]), "bf16")
+        M.mtla_check(h)
+    finally:
+        M.mtla_destroy(h)
+
+
 def test_peaked_softmax_variant():
     """Queries scaled up 4x give a near one-hot softmax; parity must survive it."""
     w = SMALL_FP32.scaled(stride=2, decode_steps=90, batch=1)
