@@ -737,8 +737,15 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = q_scale;
-  if (h->use_tc) prefill_post_kernel<T, bf16><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
-  else prefill_post_kernel<T, float><<<dim3(ceil_div(T_len, dm.s), B), 256, 0, st>>>(pa);
+  const dim3 post_grid(ceil_div(T_len, dm.s), B);
+  const bool post_fast = (dm.proj.off_u >= 0 || !pa.use_gate) && dm.s <= kPostFastMaxStride;
+  if (h->use_tc) {
+    if (post_fast) prefill_post_fast_kernel<T, bf16><<<post_grid, 256, 0, st>>>(pa);
+    else prefill_post_kernel<T, bf16><<<post_grid, 256, 0, st>>>(pa);
+  } else {
+    if (post_fast) prefill_post_fast_kernel<T, float><<<post_grid, 256, 0, st>>>(pa);
+    else prefill_post_kernel<T, float><<<post_grid, 256, 0, st>>>(pa);
+  }
   h->launches++;
   MTLA_CUDA(cudaGetLastError());
   if (!y) return MTLA_OK;

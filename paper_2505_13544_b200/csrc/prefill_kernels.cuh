@@ -120,6 +120,107 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
     for (int i = tid; i < a.r; i += 256) a.open_acc[(long long)b * a.r + i] = acc_s[i];
 }
 
+// The same work for layers whose gate needs no matrix (folded into the projection, or absent at
+// s = 1) and whose stride is at most 8: the tokens of a chunk are normalised and gated in
+// parallel, one warp per token, and only the running sum walks them in order (in the same fp32
+// order as the decode steps).  One CTA of 256 threads per (chunk, sequence).
+constexpr int kPostFastMaxStride = 8;
+
+template <typename T, typename TQ>
+__global__ void __launch_bounds__(256) prefill_post_fast_kernel(PrefillPostArgs a) {
+  __shared__ float c_s[kPostFastMaxStride][512];   // normalised latents of the chunk's tokens
+  __shared__ float w_s[kPostFastMaxStride];        // their merge weights
+  const int chunk = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int W = a.r + a.dr, DQ = a.head_dim + a.dr, half = a.dr / 2;
+  const int tok0 = chunk * a.stride, ntok = min(a.T, tok0 + a.stride) - tok0;
+  const long long row0 = (long long)b * a.T + tok0;
+
+  if (warp < ntok) {
+    const float* row = a.p1 + (row0 + warp) * a.proj.width;
+    float cv[16];                                   // r <= 512: at most 16 values per lane
+    float sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int i = lane + 32 * k;
+      cv[k] = i < a.r ? row[a.proj.off_c + i] : 0.f;
+      sum += cv[k];
+    }
+    const float mean = warp_sum(sum) / a.r;
+    float sq = 0.f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const float dlt = lane + 32 * k < a.r ? cv[k] - mean : 0.f;
+      sq += dlt * dlt;
+    }
+    const float rstd = rsqrtf(warp_sum(sq) / a.r + a.ln_eps);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const int i = lane + 32 * k;
+      if (i < a.r) c_s[warp][i] = (cv[k] - mean) * rstd * a.gamma[i] + a.beta[i];
+    }
+    float w = 1.f;
+    if (a.use_gate) {
+      const float* u = row + a.proj.off_u;
+      const float* gate_pe = a.gate_pe + (long long)chunk * a.dw;
+      float prod = 0.f;
+      for (int n = lane; n < a.dw; n += 32) {
+        const float h = rstd * (u[n] + u[a.dw + n] - mean * a.gate_s[n]) + a.gate_t[n];
+        prod = fmaf(h, gate_pe[n], prod);
+      }
+      w = 1.f / (1.f + expf(-warp_sum(prod)));
+    }
+    if (lane == 0) w_s[warp] = w;
+  }
+  __syncthreads();
+
+  // Running merge state after each token (Eq. 14's sequence), final state into the cache.
+  T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + chunk) * W;
+  for (int i = tid; i < a.r; i += 256) {
+    float acc = 0.f;
+    for (int t = 0; t < ntok; ++t) {
+      acc += w_s[t] * c_s[t][i];
+      static_cast<T*>(a.cprime)[(row0 + t) * a.r + i] = Elem<T>::from_float(acc);
+    }
+    slot_row[i] = Elem<T>::from_float(acc);
+    if (tok0 + ntok == a.T) a.open_acc[(long long)b * a.r + i] = acc;
+  }
+  // RoPE keys (rounded to the cache type, which is what decoding reads back); the slot keeps
+  // the key of the chunk's last token.
+  for (int idx = tid; idx < ntok * half; idx += 256) {
+    const int t = idx / half, k = idx % half;
+    const float* row = a.p1 + (row0 + t) * a.proj.width;
+    const float cs = a.rope_cos[(long long)(tok0 + t) * half + k], sn = a.rope_sin[(long long)(tok0 + t) * half + k];
+    const float x0 = row[a.proj.off_kr + 2 * k], x1 = row[a.proj.off_kr + 2 * k + 1];
+    const T k0 = Elem<T>::from_float(x0 * cs - x1 * sn), k1 = Elem<T>::from_float(x0 * sn + x1 * cs);
+    TQ* kr = static_cast<TQ*>(a.kr) + (row0 + t) * a.dr;
+    kr[2 * k] = Elem<TQ>::from_float(Elem<T>::to_float(k0));
+    kr[2 * k + 1] = Elem<TQ>::from_float(Elem<T>::to_float(k1));
+    if (t == ntok - 1) {
+      slot_row[a.r + 2 * k] = k0;
+      slot_row[a.r + 2 * k + 1] = k1;
+    }
+  }
+  // Scaled queries and rotated, scaled RoPE queries.
+  const int hd = a.n_heads * a.head_dim;
+  for (int idx = tid; idx < ntok * hd; idx += 256) {
+    const int t = idx / hd, i = idx % hd;
+    const float* row = a.p1 + (row0 + t) * a.proj.width;
+    static_cast<TQ*>(a.qcat)[(row0 + t) * a.n_heads * DQ + (i / a.head_dim) * DQ + i % a.head_dim] =
+        Elem<TQ>::from_float(row[a.proj.off_q + i] * a.q_scale);
+  }
+  const int nqr = a.n_heads * half;
+  for (int idx = tid; idx < ntok * nqr; idx += 256) {
+    const int t = idx / nqr, i = idx % nqr, h = i / half, k = i % half;
+    const float* row = a.p1 + (row0 + t) * a.proj.width;
+    const float cs = a.rope_cos[(long long)(tok0 + t) * half + k], sn = a.rope_sin[(long long)(tok0 + t) * half + k];
+    const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k], x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
+    TQ* qc = static_cast<TQ*>(a.qcat) + (row0 + t) * a.n_heads * DQ + h * DQ + a.head_dim;
+    qc[2 * k] = Elem<TQ>::from_float((x0 * cs - x1 * sn) * a.q_scale);
+    qc[2 * k + 1] = Elem<TQ>::from_float((x0 * sn + x1 * cs) * a.q_scale);
+  }
+}
+
 struct PrefillAttnArgs {
   const void* qcat;   // [B*T][n_h][d_h + d_R], pre-scaled by log2(e)/sqrt(d_h)
   const void* kv;     // [B*T][2*n_h*d_h]: keys then values up-projected from cprime (Eq. 9-10)
