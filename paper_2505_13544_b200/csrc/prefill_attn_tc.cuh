@@ -23,7 +23,9 @@
 // Accumulators live in TMEM (two score buffers, one output block of two halves); TMEM lane i is query row i,
 // so each of the 128 softmax threads owns one row and its maximum and sum are thread-local.
 // The reference maximum of a row is raised only when a tile exceeds it by more than 2^8; a warp
-// rescales its 32 rows of O in TMEM only when one of them must.
+// rescales its 32 rows of O in TMEM only when one of them must.  On fully visible tiles the
+// maximum is not even computed: the exponentials are taken against the current reference and
+// the tile's sum tells whether the reference was outgrown.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = score MMA issuer and TMEM owner, warp 2 = value
 // MMA issuer, warp 3 idle, warps 4-7 = softmax and epilogue.  Every wait is a bounded mbarrier
@@ -64,7 +66,7 @@ __host__ __device__ constexpr int smem_bytes(int dh) {
 }
 
 struct Bars {
-  unsigned long long q_full, kv_full[kStages], kv_empty[kStages];
+  unsigned long long q_full, k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   unsigned long long s_full[2], s_empty[2], p_full, p_empty;
   uint32_t tmem_base;
   int abort_word;
@@ -111,8 +113,10 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
   if (threadIdx.x == 0) {
     mbar_init(bar(&bars->q_full), 1);
     for (int i = 0; i < kStages; ++i) {
-      mbar_init(bar(&bars->kv_full[i]), 1);
-      mbar_init(bar(&bars->kv_empty[i]), 2);        // score issuer + value issuer
+      mbar_init(bar(&bars->k_full[i]), 1);
+      mbar_init(bar(&bars->k_empty[i]), 1);         // score issuer
+      mbar_init(bar(&bars->v_full[i]), 1);
+      mbar_init(bar(&bars->v_empty[i]), 1);         // value issuer
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(&bars->s_full[i]), 1);
@@ -150,25 +154,51 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
     mbar_arrive_expect_tx(bar(&bars->q_full), q_bytes(DH));
     for (int c = 0; c <= CK; ++c)
       tma_load_3d(q_u32 + c * QSUB, &q_map, bar(&bars->q_full), h * (DH + a.dr) + c * 64, q0, b);
-    for (int t = 0; t < n_tiles; ++t) {
-      const int st = t % kStages;
-      if (!mbar_wait(bar(&bars->kv_empty[st]), ((t / kStages) & 1) ^ 1, abort_word, a.error_word, 21))
-        break;
+    // A stage's key part (K hi, K lo, RoPE keys) is free as soon as its score MMAs are done,
+    // its value part only after the value MMAs: the keys of tile t + 1 are therefore requested
+    // before the values of tile t, which keeps the score MMAs one load latency ahead.
+    auto tile_source = [&](int t, const CUtensorMap*& kvm, const CUtensorMap*& krm, int& row) {
       const bool diag = t >= n_kv;
-      const CUtensorMap* kvm = diag ? &kv_self : &kv_closed;
-      const CUtensorMap* krm = diag ? &kr_self : &kr_closed;
-      const int row = diag ? q0 + (t - n_kv) * KT : t * KT;   // token, or closed-slot index
+      kvm = diag ? &kv_self : &kv_closed;
+      krm = diag ? &kr_self : &kr_closed;
+      row = diag ? q0 + (t - n_kv) * KT : t * KT;   // token, or closed-slot index
+    };
+    // Stage layout in chunks: K hi [0, CK), K lo [CK, 2CK), RoPE keys 2CK, V hi, V lo.
+    auto load_keys = [&](int t) {
+      const int st = t % kStages;
+      if (!mbar_wait(bar(&bars->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_word, a.error_word, 21))
+        return false;
+      const CUtensorMap *kvm, *krm;
+      int row;
+      tile_source(t, kvm, krm, row);
       const uint32_t dst = kv_u32 + st * stage_bytes(DH);
-      mbar_arrive_expect_tx(bar(&bars->kv_full[st]), stage_bytes(DH));
-      // Stage layout in chunks: K hi [0, CK), K lo [CK, 2CK), RoPE keys 2CK, V hi, V lo.
-      for (int c = 0; c < CK; ++c) {
-        for (int half = 0; half < 2; ++half) {
-          const int col = half * 2 * hd + h * DH + c * 64;        // remainders sit 2 n_h d_h further
-          tma_load_3d(dst + (half * CK + c) * SUB, kvm, bar(&bars->kv_full[st]), col, row, b);
-          tma_load_3d(dst + ((2 + half) * CK + 1 + c) * SUB, kvm, bar(&bars->kv_full[st]), hd + col, row, b);
-        }
-      }
-      tma_load_3d(dst + 2 * CK * SUB, krm, bar(&bars->kv_full[st]), 0, row, b);
+      mbar_arrive_expect_tx(bar(&bars->k_full[st]), (2 * CK + 1) * SUB);
+      for (int c = 0; c < CK; ++c)
+        for (int half = 0; half < 2; ++half)       // remainders sit 2 n_h d_h columns further
+          tma_load_3d(dst + (half * CK + c) * SUB, kvm, bar(&bars->k_full[st]),
+                      half * 2 * hd + h * DH + c * 64, row, b);
+      tma_load_3d(dst + 2 * CK * SUB, krm, bar(&bars->k_full[st]), 0, row, b);
+      return true;
+    };
+    auto load_values = [&](int t) {
+      const int st = t % kStages;
+      if (!mbar_wait(bar(&bars->v_empty[st]), ((t / kStages) & 1) ^ 1, abort_word, a.error_word, 20))
+        return false;
+      const CUtensorMap *kvm, *krm;
+      int row;
+      tile_source(t, kvm, krm, row);
+      const uint32_t dst = kv_u32 + st * stage_bytes(DH) + (2 * CK + 1) * SUB;
+      mbar_arrive_expect_tx(bar(&bars->v_full[st]), 2 * CK * SUB);
+      for (int c = 0; c < CK; ++c)
+        for (int half = 0; half < 2; ++half)
+          tma_load_3d(dst + (half * CK + c) * SUB, kvm, bar(&bars->v_full[st]),
+                      hd + half * 2 * hd + h * DH + c * 64, row, b);
+      return true;
+    };
+    bool ok = load_keys(0);
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      if (t + 1 < n_tiles) ok = load_keys(t + 1);
+      if (ok) ok = load_values(t);
     }
   } else if (warp == 1 && lane == 0) {
     // ------------------------------------------------------------------ score MMA issuer
@@ -176,7 +206,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
     for (int t = 0; t < n_tiles && ok; ++t) {
       const int st = t % kStages;
       ok = mbar_wait(bar(&bars->s_empty[t & 1]), ((t >> 1) & 1) ^ 1, abort_word, a.error_word, 23) &&
-           mbar_wait(bar(&bars->kv_full[st]), (t / kStages) & 1, abort_word, a.error_word, 24);
+           mbar_wait(bar(&bars->k_full[st]), (t / kStages) & 1, abort_word, a.error_word, 24);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t kbase = kv_u32 + st * stage_bytes(DH);
@@ -194,14 +224,15 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
         }
       }
       mma_commit(bar(&bars->s_full[t & 1]));
-      mma_commit(bar(&bars->kv_empty[st]));
+      mma_commit(bar(&bars->k_empty[st]));
     }
   } else if (warp == 2 && lane == 0) {
     // ------------------------------------------------------------------ value MMA issuer
     bool ok = true;
     for (int t = 0; t < n_tiles && ok; ++t) {
       const int st = t % kStages;
-      ok = mbar_wait(bar(&bars->p_full), t & 1, abort_word, a.error_word, 25);
+      ok = mbar_wait(bar(&bars->p_full), t & 1, abort_word, a.error_word, 25) &&
+           mbar_wait(bar(&bars->v_full[st]), (t / kStages) & 1, abort_word, a.error_word, 19);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t vbase = kv_u32 + st * stage_bytes(DH) + (2 * CK + 1) * SUB;
@@ -214,7 +245,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
         const uint64_t bd = make_smem_desc(vbase + ks * 2048, SUB, 1024, kSwizzle128B);
         mma_bf16_ss(tmem_base + kColO, ad, bd, IDESC_PV, (t > 0 || ks > 0) ? 1u : 0u);
       }
-      mma_commit(bar(&bars->kv_empty[st]));
+      mma_commit(bar(&bars->v_empty[st]));
       mma_commit(bar(&bars->p_empty));
     }
   } else if (warp >= 4) {
@@ -243,61 +274,73 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap q_map,
         tmem_ld_x32(lane_base + (t & 1) * KT + c0, v);
       }
       tmem_wait_ld();
-      float s[KT];
-      float mt = -INFINITY;
-      if (__all_sync(0xffffffffu, lim >= KT)) {
-        // Every column of the tile is visible to every row of this warp: no predicate needed.
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int c = 0; c < KT; ++c) {
-          s[c] = __uint_as_float(sv[c]);
-          mx[c & 3] = fmaxf(mx[c & 3], s[c]);
-        }
-        mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      } else {
-#pragma unroll
-        for (int c = 0; c < KT; ++c) {
-          s[c] = (c < lim || c == own) ? __uint_as_float(sv[c]) : -INFINITY;
-          mt = fmaxf(mt, s[c]);
-        }
-      }
       tc_fence_before_sync();
-      mbar_arrive(bar(&bars->s_empty[t & 1]));
-      // Lazy reference: raise it only when this tile outgrows it by more than 2^8.
-      const bool raise = mt > m_run + kRescaleThreshold;
-      const float m_new = raise ? mt : m_run;
-      const float fac = (raise && m_run != -INFINITY) ? exp2f(m_run - m_new) : 1.f;
-      if (__any_sync(0xffffffffu, raise && t > 0)) {
-        // O rows are scaled to the old references: wait for the previous tile's value MMAs.
-        ok = mbar_wait(bar(&bars->p_empty), (t & 1) ^ 1, abort_word, a.error_word, 27);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int c0 = 0; c0 < 2 * DH; c0 += 32) {
-          uint32_t ov[32];
-          tmem_ld_x32(lane_base + kColO + c0, ov);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * fac);
-          tmem_st_x32(lane_base + kColO + c0, ov);
-        }
-        tmem_wait_st();
-        tc_fence_before_sync();
-      }
-      l_run *= fac;
-      m_run = m_new;
-      const float m_eff = m_run == -INFINITY ? 0.f : m_run;   // a row that has seen nothing yet
+      mbar_arrive(bar(&bars->s_empty[t & 1]));            // the scores are in registers now
       uint32_t pk[KT / 2];
-      float lsum[4] = {0.f, 0.f, 0.f, 0.f};
+      // Common case: the whole tile is visible to every row of the warp and every row has a
+      // reference already.  Then the probabilities are formed at once, and the row maximum is
+      // never computed: a tile that had outgrown a reference by 2^8 would show in its sum
+      // (sum <= 2^15 guarantees every probability <= 2^15), in which case the careful path
+      // below redoes the tile.  The comparison also catches an overflow to infinity.
+      bool fast = __all_sync(0xffffffffu, lim >= KT && m_run != -INFINITY);
+      if (fast) {
+        float lsum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < KT; c += 2) {
-        const float p0 = ex2_approx(s[c] - m_eff), p1 = ex2_approx(s[c + 1] - m_eff);
-        lsum[(c >> 1) & 3] += p0 + p1;
-        const __nv_bfloat162 two = __floats2bfloat162_rn(p0, p1);
-        pk[c / 2] = *reinterpret_cast<const uint32_t*>(&two);
+        for (int c = 0; c < KT; c += 2) {
+          const float p0 = ex2_approx(__uint_as_float(sv[c]) - m_run);
+          const float p1 = ex2_approx(__uint_as_float(sv[c + 1]) - m_run);
+          lsum[(c >> 1) & 3] += p0 + p1;
+          const __nv_bfloat162 two = __floats2bfloat162_rn(p0, p1);
+          pk[c / 2] = *reinterpret_cast<const uint32_t*>(&two);
+        }
+        const float tile_sum = (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
+        fast = __all_sync(0xffffffffu, tile_sum <= 32768.f);
+        if (fast) l_run += tile_sum;
       }
-      l_run += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
+      if (!fast) {
+        // Careful path: predicate, row maximum, lazy raise of the reference (by more than 2^8
+        // only), rescale of this warp's O rows when one of them raised.
+        float mt = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < KT; ++c) {
+          if (!(c < lim || c == own)) sv[c] = 0xff800000u;   // -inf
+          mt = fmaxf(mt, __uint_as_float(sv[c]));
+        }
+        const bool raise = mt > m_run + kRescaleThreshold;
+        const float m_new = raise ? mt : m_run;
+        const float fac = (raise && m_run != -INFINITY) ? exp2f(m_run - m_new) : 1.f;
+        if (__any_sync(0xffffffffu, raise && t > 0)) {
+          // O rows are scaled to the old references: wait for the previous tile's value MMAs.
+          ok = mbar_wait(bar(&bars->p_empty), (t & 1) ^ 1, abort_word, a.error_word, 27);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after_sync();
+#pragma unroll
+          for (int c0 = 0; c0 < 2 * DH; c0 += 32) {
+            uint32_t ov[32];
+            tmem_ld_x32(lane_base + kColO + c0, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * fac);
+            tmem_st_x32(lane_base + kColO + c0, ov);
+          }
+          tmem_wait_st();
+          tc_fence_before_sync();
+        }
+        l_run *= fac;
+        m_run = m_new;
+        const float m_eff = m_run == -INFINITY ? 0.f : m_run;   // a row that has seen nothing yet
+        float lsum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < KT; c += 2) {
+          const float p0 = ex2_approx(__uint_as_float(sv[c]) - m_eff);
+          const float p1 = ex2_approx(__uint_as_float(sv[c + 1]) - m_eff);
+          lsum[(c >> 1) & 3] += p0 + p1;
+          const __nv_bfloat162 two = __floats2bfloat162_rn(p0, p1);
+          pk[c / 2] = *reinterpret_cast<const uint32_t*>(&two);
+        }
+        l_run += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
+      }
       // The single probability buffer is free once the previous tile's value MMAs have completed.
       ok = mbar_wait(bar(&bars->p_empty), (t & 1) ^ 1, abort_word, a.error_word, 28);
       ok = __all_sync(0xffffffffu, ok);
