@@ -45,6 +45,19 @@ def measured_peaks() -> dict:
             "source": "fallback"}
 
 
+def kernel_code_hash() -> str:
+    """Hash of the decode-attention kernel's code (comments and blank space removed), to tell
+    whether the committed ncu counters still describe the kernel that is being timed."""
+    csrc = os.path.join(ROOT, "paper_2505_13544_b200", "csrc")
+    text = ""
+    for name in ("decode_attn_tc.cuh", "sm100_ptx.cuh"):
+        for line in open(os.path.join(csrc, name)):
+            code = line.split("//")[0].strip()
+            if code:
+                text += " ".join(code.split()) + "\n"
+    return hashlib.sha256(text.encode()).hexdigest()
+
+
 def algorithmic_work(w: synth.Workload, n_slots: float) -> dict:
     """Bytes and FLOP one decode step must move/compute (weights once, cache once)."""
     e = 2 if w.dtype == "bf16" else 4
@@ -355,10 +368,7 @@ def main() -> None:
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
         t = json.load(open(tpath)).get(M.mtla_attention_variant(h), {})
-        csrc = os.path.join(ROOT, "paper_2505_13544_b200", "csrc")
-        sha = hashlib.sha256(open(os.path.join(csrc, "decode_attn_tc.cuh"), "rb").read()
-                             + open(os.path.join(csrc, "sm100_ptx.cuh"), "rb").read()).hexdigest()
-        if t.get("dram_bytes_per_cache_byte") is not None and t.get("kernel_source_sha256") == sha:
+        if t.get("dram_bytes_per_cache_byte") is not None and t.get("kernel_code_sha256") == kernel_code_hash():
             traffic = t["dram_bytes_per_cache_byte"] * work["cache_bytes"]
 
     line = {

@@ -24,25 +24,27 @@
 //
 // Shared memory: a ring of nine 16 KB "pairs" (two adjacent sub-tiles = a 128-row MN-major
 // operand block), three 8 KB sub-tiles for the RoPE-key columns, q~ as a K-major swizzled B
-// operand (TMA-loaded per segment), and two bf16 probability buffers.  The ring holds more
-// than two tiles, and the MMA warp issues whichever of "score the next tile" / "accumulate the
-// tile whose probabilities are ready" can go, so loads stay in flight through every phase.
+// operand (TMA-loaded per segment), and two bf16 probability buffers.  The ring holds a little
+// more than two tiles, and a load can only be issued once its slot is free; to keep the DRAM
+// latency off that path the producer also asks the tile after the one it is loading into L2
+// (cp.async.bulk.prefetch), so the load proper is an L2 hit.
 //
 // The online softmax raises a head's reference maximum only when a tile exceeds it by more
 // than 2^8.  The common tile therefore needs no cross-thread reduction: each thread compares
 // its scores with the shared references, raises a flag if one is outgrown, and forms its
 // probabilities at once; the flag is collected through a split mbarrier arrive / wait that
 // overlaps that work, and only a raised flag (always at a sequence's first tile, otherwise
-// rare) sends the 128 threads through the reduction, the TMEM rescale of O and a second
+// rare) sends the softmax threads through the reduction, the TMEM rescale of O and a second
 // exponentiation.  Results are exact either way because the same reference enters numerator
 // and denominator.
 //
 // One thread can issue a tcgen05.mma only about every hundred cycles, far slower than these
 // small-N MMAs execute, so issue is spread over eight single-thread issuers in eight warps:
 // four for the scores (issuer k owns partial accumulator k) and four for the values (issuer j
-// owns output block j and returns its pair to the ring as soon as its four MMAs are in).  The softmax is instruction-bound too, so it runs on eight warps: with
-// M = 64 only lanes 0-15 of a warp's TMEM quarter hold scores, and two warps per quarter split
-// the heads between them.  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
+// owns output block j and returns its pair to the ring as soon as its four MMAs are in).
+// The softmax is instruction- and latency-bound too, so it runs on eight warps: with M = 64
+// only lanes 0-15 of a warp's TMEM quarter hold scores, and two warps per quarter split the
+// heads between them.  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
 // warps 5-8 = value issuers, warps 9-11 idle, warps 12-19 = softmax and epilogue.  The first
 // three warpgroups give most of their registers to the other two (setmaxnreg).
 //

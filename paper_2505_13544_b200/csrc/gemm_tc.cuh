@@ -66,11 +66,6 @@ __host__ __device__ constexpr int smem_bytes(int nb, int stages) {
   return stages * stage_bytes(nb) + 1024 /* alignment slack */ + 256 /* barriers */;
 }
 
-// As many stages as fit one CTA per SM (weight streaming wants bytes in flight), at most 8.
-__host__ __device__ constexpr int deep_stages(int bn) {
-  return (200 * 1024) / stage_bytes(bn) > 8 ? 8 : (200 * 1024) / stage_bytes(bn);
-}
-
 struct Bars {
   unsigned long long full[8], empty[8], acc_full;
   uint32_t tmem_base;

@@ -46,19 +46,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Non-blocking probe of a phase (no hardware suspend): for loops that poll several barriers.
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
 // Every wait in these kernels is bounded: it gives up after kWaitBudgetNs of wall time (or
 // as soon as another thread of the CTA has given up), raises the CTA-wide abort word and
 // records a code in the global error word.  Callers unwind without touching the barrier again.
