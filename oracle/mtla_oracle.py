@@ -32,7 +32,8 @@ Readings of points the paper leaves open (each is a documented convention):
 
 Parity pins: tests/test_oracle_pins.py checks Form I against Form II, Form I(s=1)
 against Form III, the paper's worked merge example, closed forms (uniform attention,
-single slot, zero hyper-network => w = 1/2), slot counts and RoPE shift invariance.
+single slot, zero hyper-network => w = 1/2), slot counts and RoPE shift invariance;
+reorder_states against hypotheses decoded one by one from their full token histories.
 Parity unpinned (free conventions the paper does not fix, shared with the CUDA path):
 the sinusoid's exact form, LayerNorm eps, the RoPE pairing, bias presence.
 """
@@ -195,6 +196,16 @@ def decode_sequence(p: Params, xs: np.ndarray, st: State | None = None, rows=Non
         if y is not None:
             ys.append(y)
     return (np.stack(ys) if ys else np.zeros((0, p.d_model))), st
+
+
+def reorder_states(states: list, parents) -> list:
+    """Beam-search re-parenting: hypothesis b of the new beam continues old hypothesis
+    parents[b].  The paper decodes with beam search; its cache rules (Sections 4.1, 4.3) are
+    per sequence, so a forked hypothesis simply starts from a copy of its parent's caches and
+    token count.  Every returned State owns its arrays: siblings never share storage."""
+    return [State(c_hat=[v.copy() for v in states[q].c_hat],
+                  kr_hat=[v.copy() for v in states[q].kr_hat], tokens=states[q].tokens)
+            for q in (int(v) for v in parents)]
 
 
 def state_from_cache(cache: np.ndarray, tokens: int, p: Params) -> State:

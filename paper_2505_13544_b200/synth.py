@@ -163,3 +163,24 @@ def context_cache_row(w: Workload, seq: int, n_slots: int | None = None) -> torc
     row = normal(w.seed, f"ctx/{seq}", (n, w.slot_width))
     row[:, : w.latent_rank] *= gains.astype(np.float32)
     return stored(row, w.dtype)
+
+
+def ragged_lengths(seed: int, n: int, lo: int, hi: int) -> list[int]:
+    """n prompt lengths drawn uniformly from [lo, hi], a stand-in for utterances of
+    different durations (the paper's test sets are variable-length speech and text)."""
+    return [int(v) for v in _generator(seed, "ragged_lengths").integers(lo, hi + 1, size=n)]
+
+
+def beam_parents(seed: int, step: int, n_utt: int, beam: int) -> list[int]:
+    """Parent indices of one beam-search step for n_utt utterances with `beam` hypotheses
+    each (batch index = utterance * beam + rank).  Every surviving hypothesis continues one of
+    its own utterance's hypotheses; better-ranked parents are chosen more often (rank k with
+    weight 1 / (k + 1)), as in a real search where most survivors extend the top entries."""
+    g = _generator(seed, f"beam_parents/{step}")
+    weights = 1.0 / (1.0 + np.arange(beam))
+    weights /= weights.sum()
+    out = []
+    for u in range(n_utt):
+        picks = np.sort(g.choice(beam, size=beam, p=weights))
+        out += [u * beam + int(k) for k in picks]
+    return out

@@ -307,6 +307,44 @@ def test_state_from_cache_round_trip():
     np.testing.assert_array_equal(O.decode_step(p, st, x_new), O.decode_step(p, st2, x_new))
 
 
+# ------------------------------------------------------------------ beam re-parenting
+
+def test_reorder_equals_hypotheses_decoded_from_scratch():
+    """Two rounds of forking: every hypothesis equals the same token history run alone, and a
+    planted mistake (children sharing their parent's arrays) is caught by the same check."""
+    p = make_params(seed=5, s=3)
+    prompt = inputs(40, 7)
+
+    def run(reorder):
+        _, root = O.decode_sequence(p, prompt)
+        states = reorder([root], [0, 0, 0])
+        histories = [list(prompt) for _ in range(3)]
+        outs = None
+        for step in range(9):
+            xs = inputs(50 + step, 3)
+            outs = [O.decode_step(p, states[b], xs[b]) for b in range(3)]
+            for b in range(3):
+                histories[b].append(xs[b])
+            if step in (2, 5):
+                parents = [2, 0, 2] if step == 2 else [1, 1, 0]
+                states = reorder(states, parents)
+                histories = [list(histories[q]) for q in parents]
+        worst = 0.0
+        for b in range(3):
+            alone, st = O.decode_sequence(p, np.stack(histories[b]))
+            assert st.tokens == states[b].tokens and st.n_slots == states[b].n_slots
+            worst = max(worst, np.abs(outs[b] - alone[-1]).max(),
+                        np.abs(O.cache_array(states[b]) - O.cache_array(st)).max())
+        return worst
+
+    assert run(O.reorder_states) < 1e-12
+
+    def aliasing(states, parents):          # the mistake: no copies, siblings write one list
+        return [states[q] for q in parents]
+    with pytest.raises((AssertionError, IndexError)):
+        assert run(aliasing) < 1e-12
+
+
 # ------------------------------------------------------------------ planted mistakes are caught
 
 def _forms_disagree(p, xs):
