@@ -83,6 +83,18 @@ typedef struct {
   const void* hyp_pe_b;  /* [d_w] or NULL */
 } mtla_weights;
 
+/* Paged storage of the cache, for ragged batches and beam search (the paper decodes with beam
+ * search over utterances of different lengths, Section 5 and the appendix on decoding
+ * set-ups).  The slots live in a pool of pages of page_slots slots; every sequence has its own
+ * token count and holds the pages of its slots.  Closed slots never change (Section 4.1 only
+ * ever writes a sequence's newest slot), so beams that continue one hypothesis share its pages
+ * and only the page of the newest slot is copied when a beam first writes to it. */
+typedef struct {
+  int32_t page_slots;   /* slots per page: 64 (one tile of the decode attention) */
+  int32_t n_pages;      /* pages in the pool; 0 selects max_batch * ceil(ceil(max_tokens/s)/64),
+                           enough for max_batch unshared sequences of max_tokens tokens */
+} mtla_paging;
+
 /* Device bytes mtla_create needs for this configuration (weights, tables, cache, decode
  * scratch and, if max_prefill_tokens > 0, the prefill workspace).  0 if cfg is invalid. */
 size_t mtla_arena_bytes(const mtla_config* cfg);
@@ -94,6 +106,16 @@ size_t mtla_arena_bytes(const mtla_config* cfg);
 int mtla_create(const mtla_config* cfg, const mtla_weights* weights, void* arena,
                 size_t arena_bytes, void* stream, mtla_handle** out);
 
+/* The same layer with the cache in paged storage (see mtla_paging) and a token count per
+ * sequence.  On such a handle mtla_decode_step advances every sequence from its own position
+ * (the slot, the merge weight's pe_j and the RoPE angle of Section 4.1 / 4.3 are those of the
+ * sequence), mtla_prefill_seqs fills chosen sequences, mtla_beam_reorder re-parents the batch,
+ * and every other call keeps its meaning.  At most 1022 sequences on the tensor-core path.
+ * mtla_arena_bytes_paged is the arena size for the pair (cfg, paging); 0 if invalid. */
+size_t mtla_arena_bytes_paged(const mtla_config* cfg, const mtla_paging* paging);
+int mtla_create_paged(const mtla_config* cfg, const mtla_paging* paging, const mtla_weights* weights,
+                      void* arena, size_t arena_bytes, void* stream, mtla_handle** out);
+
 /* Parallel prefill (Section 4.2 with the RoPE shortcut of Section 4.3): consumes T prompt
  * tokens for each of B sequences, x device [B][T][d], and reproduces what T decode steps
  * would have produced: y device [B][T][d] (may be NULL to skip the outputs), the
@@ -101,6 +123,14 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* weights, void* arena
  * causal mask is applied as a predicate, never materialised.  Requires an empty cache
  * (tokens == 0), B <= max_batch, T <= min(max_prefill_tokens, max_tokens). */
 int mtla_prefill(mtla_handle* h, const void* x, int32_t B, int32_t T, void* y, void* stream);
+
+/* Paged handles only: the prefill of mtla_prefill for sequences seq0 .. seq0 + B - 1, which must
+ * be empty; x device [B][T][d], y device [B][T][d] or NULL.  seq0 may not exceed the current
+ * batch (sequences are numbered without gaps); the batch becomes max(batch, seq0 + B).  Calls
+ * with different T build a ragged batch.  MTLA_ERR_STATE on a handle without paging or a
+ * non-empty sequence, MTLA_ERR_CAPACITY if the pool has too few free pages. */
+int mtla_prefill_seqs(mtla_handle* h, int32_t seq0, const void* x, int32_t B, int32_t T, void* y,
+                      void* stream);
 
 /* One incremental decoding step (Section 4.1, Eq. 13, Eq. 17) for every sequence:
  * x device [B][d] is token number tokens+1; its latent is merged into slot
@@ -140,7 +170,8 @@ int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y
 #define MTLA_STATIC_SCRATCH_BYTES (4u << 20)
 int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, void* stream);
 
-/* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3). */
+/* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3);
+ * with per-sequence token counts, the sum over the sequences. */
 size_t mtla_cache_bytes(const mtla_handle* h);
 
 /* Releases the host-side handle.  The arena is the caller's. */
@@ -151,17 +182,58 @@ int mtla_destroy(mtla_handle* h);
 /* Empties the cache (tokens = 0, batch unset).  Nothing is enqueued. */
 int mtla_reset(mtla_handle* h);
 
-/* Current position: tokens consumed per sequence, slots held (= ceil(tokens/s)), batch. */
+/* Current position: tokens consumed per sequence (the longest sequence's on a paged handle),
+ * slots held (= ceil(tokens/s)), batch. */
 int mtla_position(const mtla_handle* h, int32_t* tokens, int32_t* slots, int32_t* batch);
 
 /* Copies the cache in use to dst (device), layout [B][slots][r + d_R], element type dtype;
- * `bytes` must be >= mtla_cache_bytes(h). */
+ * `bytes` must be >= mtla_cache_bytes(h).  MTLA_ERR_STATE on a paged handle whose sequences
+ * differ in length (use mtla_cache_export_seq). */
 int mtla_cache_export(mtla_handle* h, void* dst, size_t bytes, void* stream);
 
 /* Replaces the cache by src (device) [B][ceil(tokens/s)][r + d_R] and sets the position to
  * `tokens`.  If tokens is not a multiple of s the last slot is open and its fp32
  * accumulator is initialised from the stored value. */
 int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens, void* stream);
+
+/* Beam reordering (paged handles): sequence b of the new batch continues old sequence
+ * parents[b] (host array of n_new indices into the current batch; an index may repeat or be
+ * absent).  Positions, page tables and the fp32 state of the open slot follow on `stream`;
+ * pages are shared, not copied, and pages that no sequence holds any more return to the pool.
+ * The batch becomes n_new.  The parents array is read before the call returns. */
+int mtla_beam_reorder(mtla_handle* h, const int32_t* parents, int32_t n_new, void* stream);
+
+/* Tokens consumed by sequences 0 .. n-1 (host array; 0 beyond the batch).  On a handle without
+ * paging every sequence reports the common count. */
+int mtla_seq_positions(const mtla_handle* h, int32_t* tokens, int32_t n);
+
+/* Pages of the pool that some sequence holds (shared pages count once); -1 without paging.
+ * Physical cache bytes = pages * 64 * (r + d_R) * sizeof(element), while mtla_cache_bytes
+ * reports the logical sum over sequences of ceil(tokens/s) slots. */
+int64_t mtla_pages_in_use(const mtla_handle* h);
+
+/* Copies the slots of one sequence to dst (device) [ceil(tokens/s)][r + d_R]; works with and
+ * without paging. */
+int mtla_cache_export_seq(mtla_handle* h, int32_t seq, void* dst, size_t bytes, void* stream);
+
+/* The page pool's bookkeeping on its own, host-only (no GPU is touched): the object a paged
+ * handle uses to decide which pages to allocate, share and copy.  A scheduler can run it ahead
+ * of the GPU to see whether a batch fits; the tests drive it against a model of the sharing
+ * rules.  prepare(seq, n_slots, write_slot): make slots [0, n_slots) of seq addressable and,
+ * if write_slot >= 0, the page holding it private to seq; returns the number of page copies
+ * that implies and writes up to max_copies triples (source page, destination page, rows) to
+ * `copies`, or MTLA_ERR_CAPACITY (state unchanged) if the pool has too few free pages.
+ * reorder: as mtla_beam_reorder.  row: the pages seq holds, returns their count.  ref: how
+ * many sequences hold a page. */
+typedef struct mtla_page_pool mtla_page_pool;
+mtla_page_pool* mtla_page_pool_create(int32_t n_pages, int32_t max_seqs, int32_t max_pages_per_seq);
+void mtla_page_pool_destroy(mtla_page_pool* p);
+int mtla_page_pool_prepare(mtla_page_pool* p, int32_t seq, int32_t n_slots, int32_t write_slot,
+                           int32_t* copies, int32_t max_copies);
+int mtla_page_pool_reorder(mtla_page_pool* p, const int32_t* parents, int32_t n_new, int32_t n_old);
+int mtla_page_pool_row(const mtla_page_pool* p, int32_t seq, int32_t* pages, int32_t max_pages);
+int mtla_page_pool_in_use(const mtla_page_pool* p);
+int mtla_page_pool_ref(const mtla_page_pool* p, int32_t page);
 
 /* Synchronises `stream` and reports a sticky device-side status (MTLA_ERR_DEVICE_TIMEOUT if
  * a bounded wait inside a kernel gave up; MTLA_ERR_CUDA if the stream is in error). */

@@ -27,7 +27,13 @@ EXPORTED_SYMBOLS = (
     "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
     "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
     "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
-    "mtla_profile_end_stages", "mtla_decode_step_static", "mtla_profile_begin_attention")
+    "mtla_profile_end_stages", "mtla_decode_step_static", "mtla_profile_begin_attention",
+    "mtla_arena_bytes_paged", "mtla_create_paged", "mtla_prefill_seqs", "mtla_beam_reorder",
+    "mtla_seq_positions", "mtla_pages_in_use", "mtla_cache_export_seq",
+    "mtla_page_pool_create", "mtla_page_pool_destroy", "mtla_page_pool_prepare",
+    "mtla_page_pool_reorder", "mtla_page_pool_row", "mtla_page_pool_in_use", "mtla_page_pool_ref")
+
+PAGE_SLOTS = 64
 
 DECODE_STAGES = ("input_proj", "norm_gate_update", "absorb", "attention", "combine", "value_proj",
                  "output_proj")
@@ -46,6 +52,10 @@ class mtla_config(ctypes.Structure):
         ("ln_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
 
 
+class mtla_paging(ctypes.Structure):
+    _fields_ = [("page_slots", ctypes.c_int32), ("n_pages", ctypes.c_int32)]
+
+
 class mtla_weights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES]
 
@@ -62,7 +72,22 @@ def load_library() -> ctypes.CDLL:
     lib = ctypes.CDLL(LIB_PATH)
     vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
     cfg_p, w_p = ctypes.POINTER(mtla_config), ctypes.POINTER(mtla_weights)
+    pg_p, i32_p = ctypes.POINTER(mtla_paging), ctypes.POINTER(ctypes.c_int32)
     sigs = {
+        "mtla_arena_bytes_paged": (sz, [cfg_p, pg_p]),
+        "mtla_create_paged": (ctypes.c_int, [cfg_p, pg_p, w_p, vp, sz, vp, ctypes.POINTER(vp)]),
+        "mtla_prefill_seqs": (ctypes.c_int, [vp, i32, vp, i32, i32, vp, vp]),
+        "mtla_beam_reorder": (ctypes.c_int, [vp, i32_p, i32, vp]),
+        "mtla_seq_positions": (ctypes.c_int, [vp, i32_p, i32]),
+        "mtla_pages_in_use": (ctypes.c_int64, [vp]),
+        "mtla_cache_export_seq": (ctypes.c_int, [vp, i32, vp, sz, vp]),
+        "mtla_page_pool_create": (vp, [i32, i32, i32]),
+        "mtla_page_pool_destroy": (None, [vp]),
+        "mtla_page_pool_prepare": (ctypes.c_int, [vp, i32, i32, i32, i32_p, i32]),
+        "mtla_page_pool_reorder": (ctypes.c_int, [vp, i32_p, i32, i32]),
+        "mtla_page_pool_row": (ctypes.c_int, [vp, i32, i32_p, i32]),
+        "mtla_page_pool_in_use": (ctypes.c_int, [vp]),
+        "mtla_page_pool_ref": (ctypes.c_int, [vp, i32]),
         "mtla_arena_bytes": (sz, [cfg_p]),
         "mtla_create": (ctypes.c_int, [cfg_p, w_p, vp, sz, vp, ctypes.POINTER(vp)]),
         "mtla_prefill": (ctypes.c_int, [vp, vp, i32, i32, vp, vp]),
@@ -130,10 +155,13 @@ def mtla_arena_bytes(cfg: mtla_config) -> int:
     return load_library().mtla_arena_bytes(ctypes.byref(cfg))
 
 
-def mtla_create(cfg: mtla_config, weights: dict, device="cuda:0", stream=None) -> Handle:
-    """weights: name -> CUDA tensor, row-major [in][out], dtype matching cfg.dtype."""
+def mtla_create(cfg: mtla_config, weights: dict, device="cuda:0", stream=None,
+                paging: mtla_paging | None = None) -> Handle:
+    """weights: name -> CUDA tensor, row-major [in][out], dtype matching cfg.dtype.
+    With `paging` the call is mtla_create_paged."""
     lib = load_library()
-    nbytes = lib.mtla_arena_bytes(ctypes.byref(cfg))
+    nbytes = (lib.mtla_arena_bytes(ctypes.byref(cfg)) if paging is None
+              else lib.mtla_arena_bytes_paged(ctypes.byref(cfg), ctypes.byref(paging)))
     if nbytes == 0:
         raise MTLAError(-2, "mtla_arena_bytes")
     device = torch.device(device)
@@ -155,8 +183,12 @@ def mtla_create(cfg: mtla_config, weights: dict, device="cuda:0", stream=None) -
             setattr(w, name, t.data_ptr())
         out = ctypes.c_void_p()
         st = _stream_ptr(stream)
-        _check(lib.mtla_create(ctypes.byref(cfg), ctypes.byref(w), base, nbytes, st,
-                               ctypes.byref(out)), "mtla_create")
+        if paging is None:
+            _check(lib.mtla_create(ctypes.byref(cfg), ctypes.byref(w), base, nbytes, st,
+                                   ctypes.byref(out)), "mtla_create")
+        else:
+            _check(lib.mtla_create_paged(ctypes.byref(cfg), ctypes.byref(paging), ctypes.byref(w),
+                                         base, nbytes, st, ctypes.byref(out)), "mtla_create_paged")
         torch.cuda.current_stream().synchronize()   # packing done: weight tensors may be freed
     return Handle(out.value, cfg, arena, dtype, device)
 
@@ -181,6 +213,106 @@ def mtla_prefill(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, want
                                        y.data_ptr() if y is not None else None,
                                        _stream_ptr(stream)), "mtla_prefill")
     return y
+
+
+def mtla_create_paged(cfg: mtla_config, weights: dict, n_pages: int = 0, device="cuda:0",
+                      stream=None) -> Handle:
+    """A layer whose cache lives in 64-slot pages, with a token count per sequence."""
+    return mtla_create(cfg, weights, device, stream, paging=mtla_paging(PAGE_SLOTS, n_pages))
+
+
+def mtla_arena_bytes_paged(cfg: mtla_config, n_pages: int = 0) -> int:
+    pg = mtla_paging(PAGE_SLOTS, n_pages)
+    return load_library().mtla_arena_bytes_paged(ctypes.byref(cfg), ctypes.byref(pg))
+
+
+def mtla_prefill_seqs(h: Handle, seq0: int, x: torch.Tensor, y: torch.Tensor | None = None,
+                      want_output=True, stream=None):
+    """Prefill of the empty sequences seq0 .. seq0 + B - 1 of a paged handle; x [B][T][d]."""
+    b, t, d = x.shape
+    _expect(x, h, (b, t, h.config.d_model), "x")
+    if want_output and y is None:
+        y = torch.empty_like(x)
+    if y is not None:
+        _expect(y, h, x.shape, "y")
+    _check(load_library().mtla_prefill_seqs(h.ptr, seq0, x.data_ptr(), b, t,
+                                            y.data_ptr() if y is not None else None,
+                                            _stream_ptr(stream)), "mtla_prefill_seqs")
+    return y
+
+
+def _i32_array(values):
+    return (ctypes.c_int32 * len(values))(*[int(v) for v in values])
+
+
+def mtla_beam_reorder(h: Handle, parents, stream=None) -> None:
+    """Sequence b of the new batch continues old sequence parents[b]."""
+    _check(load_library().mtla_beam_reorder(h.ptr, _i32_array(parents), len(parents),
+                                            _stream_ptr(stream)), "mtla_beam_reorder")
+
+
+def mtla_seq_positions(h: Handle) -> list[int]:
+    """Tokens consumed by each sequence of the batch."""
+    batch = mtla_position(h)[2]
+    out = (ctypes.c_int32 * max(batch, 1))()
+    _check(load_library().mtla_seq_positions(h.ptr, out, batch), "mtla_seq_positions")
+    return list(out)[:batch]
+
+
+def mtla_pages_in_use(h: Handle) -> int:
+    return load_library().mtla_pages_in_use(h.ptr)
+
+
+def mtla_cache_export_seq(h: Handle, seq: int, stream=None) -> torch.Tensor:
+    """The slots of one sequence as a tensor [slots][r + d_R]."""
+    tokens = mtla_seq_positions(h)[seq]
+    slots = -(-tokens // h.config.stride)
+    width = h.config.latent_rank + h.config.rope_dim
+    out = torch.empty(slots, width, dtype=h.dtype, device=h.device)
+    if out.numel():
+        _check(load_library().mtla_cache_export_seq(h.ptr, seq, out.data_ptr(),
+                                                    out.numel() * out.element_size(),
+                                                    _stream_ptr(stream)), "mtla_cache_export_seq")
+    return out
+
+
+class PagePool:
+    """The library's host-only page bookkeeping (mtla_page_pool_*); needs no GPU."""
+
+    def __init__(self, n_pages: int, max_seqs: int, max_pages_per_seq: int):
+        self._lib = load_library()
+        self.max_pages = max_pages_per_seq
+        self.ptr = self._lib.mtla_page_pool_create(n_pages, max_seqs, max_pages_per_seq)
+        if not self.ptr:
+            raise MTLAError(-1, "mtla_page_pool_create")
+
+    def close(self) -> None:
+        if self.ptr:
+            self._lib.mtla_page_pool_destroy(self.ptr)
+            self.ptr = None
+
+    def prepare(self, seq: int, n_slots: int, write_slot: int = -1) -> list[tuple[int, int, int]]:
+        """Returns the page copies (source, destination, rows) the call implies."""
+        buf = (ctypes.c_int32 * 6)()
+        n = self._lib.mtla_page_pool_prepare(self.ptr, seq, n_slots, write_slot, buf, 2)
+        _check(min(n, 0), "mtla_page_pool_prepare")
+        return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n)]
+
+    def reorder(self, parents, n_old: int) -> None:
+        _check(self._lib.mtla_page_pool_reorder(self.ptr, _i32_array(parents), len(parents), n_old),
+               "mtla_page_pool_reorder")
+
+    def row(self, seq: int) -> list[int]:
+        buf = (ctypes.c_int32 * self.max_pages)()
+        n = self._lib.mtla_page_pool_row(self.ptr, seq, buf, self.max_pages)
+        _check(min(n, 0), "mtla_page_pool_row")
+        return list(buf)[:n]
+
+    def in_use(self) -> int:
+        return self._lib.mtla_page_pool_in_use(self.ptr)
+
+    def ref(self, page: int) -> int:
+        return self._lib.mtla_page_pool_ref(self.ptr, page)
 
 
 def mtla_decode_step(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, stream=None):

@@ -14,6 +14,21 @@ constexpr int kWarp = 32;
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 __host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Where the compressed cache keeps slot `slot` of sequence `b`, as a row index into `base`
+// (rows of r + d_R elements).  Contiguous storage: [max_batch][max_slots] rows.  Paged storage
+// (page_table != nullptr): a pool of 64-slot pages and, per sequence, the pages it holds.
+struct CacheView {
+  void* base;
+  const int* page_table;   // [max_batch][max_pages] or nullptr
+  int max_pages;
+  int max_slots;
+};
+__device__ inline long long cache_row(const CacheView& v, int b, int slot) {
+  if (v.page_table)
+    return (long long)v.page_table[(long long)b * v.max_pages + (slot >> 6)] * 64 + (slot & 63);
+  return (long long)b * v.max_slots + slot;
+}
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
   static constexpr int kVec = 4;  // elements per 16-byte access

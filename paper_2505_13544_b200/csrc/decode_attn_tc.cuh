@@ -48,6 +48,13 @@
 // warps 5-8 = value issuers, warps 9-11 idle, warps 12-19 = softmax and epilogue.  The first
 // three warpgroups give most of their registers to the other two (setmaxnreg).
 //
+// Ragged, paged batches (template parameter RAGGED): every sequence has its own length and its
+// slots live in 64-slot pages of a pool, found through a per-sequence page table.  A page is a
+// tile, so only the tile's TMA coordinate changes; the tile list is then B variable-length runs,
+// whose prefix sums every CTA forms in shared memory before it locates its share, and the page
+// numbers of the share's first tiles are staged in shared memory so that no load waits for a
+// table lookup.
+//
 // Every wait is a bounded mbarrier wait (see sm100_ptx.cuh), the rendezvous of the softmax
 // threads included; on a timeout the CTA raises its abort word, all roles unwind, and the host
 // sees MTLA_ERR_DEVICE_TIMEOUT from mtla_check.
@@ -68,6 +75,10 @@ struct AttnTcArgs {
   int* error_word;
   int n_heads, r, dr, n_slots, batch;
   int tiles_per_seq;   // ceil(n_slots / 64)
+  // Ragged, paged batches only (otherwise nullptr / unused):
+  const int* seq_tokens;   // [B] tokens per sequence, this step's included
+  const int* page_table;   // [B][max_pages] page of tile t of sequence b
+  int max_pages, stride;
 };
 
 namespace tc {
@@ -107,6 +118,14 @@ constexpr int kOffMisc = kOffP + 2 * kPBytes;
 constexpr int kMiscBytes = 4096;
 constexpr int kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + slack for 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+// Ragged batches add the tile prefix sums of up to kMaxRaggedBatch sequences and the page
+// numbers of the first kStagedPages tiles of the CTA's share.
+constexpr int kMaxRaggedBatch = 1022;
+constexpr int kStagedPages = 1024;
+constexpr int kOffPrefix = kOffMisc + kMiscBytes;
+constexpr int kOffStaged = kOffPrefix + (kMaxRaggedBatch + 2) * 4;
+constexpr int kSmemBytesRagged = kOffStaged + kStagedPages * 4 + 1024;
+static_assert(kSmemBytesRagged <= 227 * 1024, "shared memory budget (ragged)");
 
 struct Misc {
   unsigned long long full_pair[kPairs], empty_pair[kPairs];
@@ -151,10 +170,46 @@ __host__ __device__ inline long long share_owner(long long g, long long total, l
   return ((g + 1) * G - 1) / total;
 }
 
+// Position in the tile list: tile t of sequence b, which has tps tiles.  Lock-step batches
+// have tps tiles everywhere; ragged ones read the prefix sums.
+template <bool RAGGED>
+struct TileCursor {
+  int b, t, tps;
+  // List index of the sequence's first tile.
+  __device__ __forceinline__ long long start(const int* prefix) const {
+    if constexpr (RAGGED) return prefix[b];
+    else return (long long)b * tps;
+  }
+  __device__ __forceinline__ void locate(long long g, int tps_uniform, const int* prefix, int batch) {
+    if constexpr (RAGGED) {
+      int lo = 0, hi = batch;               // largest b with prefix[b] <= g
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (prefix[mid] <= g) lo = mid; else hi = mid;
+      }
+      b = lo;
+      tps = prefix[b + 1] - prefix[b];
+    } else {
+      b = (int)(g / tps_uniform);
+      tps = tps_uniform;
+    }
+    t = (int)(g - start(prefix));
+  }
+  __device__ __forceinline__ void next(const int* prefix) {
+    if (++t == tps) {
+      t = 0;
+      ++b;
+      if constexpr (RAGGED) tps = prefix[b + 1] - prefix[b];   // prefix has one entry to spare
+    }
+  }
+  __device__ __forceinline__ bool seq_first() const { return t == 0; }
+  __device__ __forceinline__ bool seq_last() const { return t + 1 == tps; }
+};
+
 }  // namespace tc
 
 // NHP: heads padded to the MMA's N (16 or 32).  RP: r / 128 (pairs per tile).
-template <int NHP, int RP>
+template <int NHP, int RP, bool RAGGED>
 __global__ void __launch_bounds__(tc::kThreads, 1)
 decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
                       const __grid_constant__ CUtensorMap q_map, AttnTcArgs a) {
@@ -213,9 +268,48 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   grid_dependency_wait();        // nothing before this line touches the previous kernel's data
 
   // This CTA's share of the tile list.
-  const long long tps = a.tiles_per_seq, total = (long long)a.batch * tps, G = gridDim.x;
+  int* prefix = reinterpret_cast<int*>(sm + kOffPrefix);     // ragged only
+  int* staged = reinterpret_cast<int*>(sm + kOffStaged);     // ragged only
+  long long total = (long long)a.batch * a.tiles_per_seq;
+  if constexpr (RAGGED) {
+    // prefix[b] = tiles of the sequences before b; prefix[batch + 1] repeats the total.
+    for (int i = threadIdx.x; i < a.batch; i += kThreads)
+      prefix[i + 1] = ceil_div(ceil_div(a.seq_tokens[i], a.stride), kTile);
+    __syncthreads();
+    if (warp == 0) {
+      const int per = ceil_div(a.batch, 32);
+      const int lo = min(a.batch, lane * per), hi = min(a.batch, lo + per);
+      int sum = 0;
+      for (int i = lo; i < hi; ++i) sum += prefix[i + 1];
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      int run = incl - sum;
+      for (int i = lo; i < hi; ++i) {
+        run += prefix[i + 1];
+        prefix[i + 1] = run;
+      }
+      if (lane == 0) prefix[0] = 0;
+    }
+    __syncthreads();
+    total = prefix[a.batch];
+    if (threadIdx.x == 0) prefix[a.batch + 1] = (int)total;
+  }
+  const long long G = gridDim.x;
   const long long g0 = share_begin(blockIdx.x, total, G), g1 = share_begin(blockIdx.x + 1, total, G);
   const int n_tiles = (int)(g1 - g0);
+  const int tps_u = a.tiles_per_seq;
+  if constexpr (RAGGED) {
+    for (int n = threadIdx.x; n < min(n_tiles, kStagedPages); n += kThreads) {
+      TileCursor<true> c;
+      c.locate(g0 + n, 0, prefix, a.batch);
+      staged[n] = a.page_table[(long long)c.b * a.max_pages + c.t];
+    }
+    __syncthreads();
+  }
 
   const uint32_t pairs_u32 = base + kOffPairs, kr_u32 = base + kOffKr;
   const uint32_t q_u32 = base + kOffQ, p_u32 = base + kOffP;
@@ -227,24 +321,35 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     // ------------------------------------------------------------------ TMA producer
     bool ok = true;
     int pc = 0, seg = 0;
-    int b = (int)(g0 / tps), t = (int)(g0 - (long long)b * tps);
+    TileCursor<RAGGED> cur, ahead;
+    cur.locate(g0, tps_u, prefix, a.batch);
+    ahead = cur;
+    // TMA coordinates (slot, plane) of a tile: its place in the sequence's row range, or its page.
+    auto tile_coords = [&](const TileCursor<RAGGED>& c, int n, int& c_slot, int& c_plane) {
+      if constexpr (RAGGED) {
+        c_slot = 0;
+        c_plane = n < kStagedPages ? staged[n] : __ldg(a.page_table + (long long)c.b * a.max_pages + c.t);
+      } else {
+        c_slot = c.t * kTile;
+        c_plane = c.b;
+      }
+    };
     // The ring holds little more than two tiles, too few to cover the DRAM latency of a load
     // that can only be issued once its slot is free.  So tiles are first asked into L2, a few
     // tiles ahead; the load proper then finds them there.
+    // Called for n_ahead = 0, 1, 2, ... in turn: `ahead` walks the list with it.
     auto prefetch_tile = [&](int n_ahead) {
       if (n_ahead >= n_tiles) return;
-      const long long g = g0 + n_ahead;
-      const int pb = (int)(g / tps), slot = (int)(g - (long long)pb * tps) * kTile;
-      for (int c = 0; c < 2 * RP + 1; ++c) tma_prefetch_l2_3d(&cache_map, c * 64, slot, pb);
+      int slot, plane;
+      tile_coords(ahead, n_ahead, slot, plane);
+      for (int c = 0; c < 2 * RP + 1; ++c) tma_prefetch_l2_3d(&cache_map, c * 64, slot, plane);
+      ahead.next(prefix);
     };
     for (int n = 0; n < kPrefetchAhead; ++n) prefetch_tile(n);
-    for (int n = 0; n < n_tiles && ok; ++n, ++t) {
-      if (t == (int)tps) {
-        t = 0;
-        ++b;
-      }
+    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix)) {
+      const int b = cur.b;
       prefetch_tile(n + kPrefetchAhead);
-      if (n == 0 || t == 0) {
+      if (n == 0 || cur.seq_first()) {
         // A segment starts: q~ of sequence b, once the previous segment's score MMAs are done.
         ok = mbar_wait(bar(&misc->q_empty), (seg & 1) ^ 1, abort_word, a.error_word, 1);
         if (!ok) break;
@@ -253,12 +358,13 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
           tma_load_3d(q_u32 + ch * QCHUNK, &q_map, bar(&misc->q_full), ch * 64, 0, b);
         ++seg;
       }
-      const int slot = t * kTile;
+      int slot, plane;
+      tile_coords(cur, n, slot, plane);
       const int kb = n % kKrBufs;
       ok = mbar_wait(bar(&misc->empty_kr[kb]), ((n / kKrBufs) & 1) ^ 1, abort_word, a.error_word, 2);
       if (!ok) break;
       mbar_arrive_expect_tx(bar(&misc->full_kr[kb]), kSubBytes);
-      tma_load_3d(kr_u32 + kb * kSubBytes, &cache_map, bar(&misc->full_kr[kb]), a.r, slot, b);
+      tma_load_3d(kr_u32 + kb * kSubBytes, &cache_map, bar(&misc->full_kr[kb]), a.r, slot, plane);
       for (int c = 0; c < RP && ok; ++c, ++pc) {
         const int buf = pc % kPairs;
         ok = mbar_wait(bar(&misc->empty_pair[buf]), ((pc / kPairs) & 1) ^ 1, abort_word,
@@ -266,8 +372,8 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         if (!ok) break;
         const uint32_t dst = pairs_u32 + buf * kPairBytes;
         mbar_arrive_expect_tx(bar(&misc->full_pair[buf]), kPairBytes);
-        tma_load_3d(dst, &cache_map, bar(&misc->full_pair[buf]), c * 128, slot, b);
-        tma_load_3d(dst + kSubBytes, &cache_map, bar(&misc->full_pair[buf]), c * 128 + 64, slot, b);
+        tma_load_3d(dst, &cache_map, bar(&misc->full_pair[buf]), c * 128, slot, plane);
+        tma_load_3d(dst + kSubBytes, &cache_map, bar(&misc->full_pair[buf]), c * 128 + 64, slot, plane);
       }
     }
   } else if (warp >= 1 && warp <= kQkIssuers && lane == 0) {
@@ -276,16 +382,16 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     const int k = warp - 1;
     bool ok = true;
     int seg = 0;
-    int t = (int)(g0 % tps);
-    for (int n = 0; n < n_tiles && ok; ++n, ++t) {
-      if (t == (int)tps) t = 0;
+    TileCursor<RAGGED> cur;
+    cur.locate(g0, tps_u, prefix, a.batch);
+    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix)) {
       const uint32_t d_tmem = tmem_base + kColS + (n & 1) * (kSParts * 32) + k * 32;
       auto qk = [&](uint32_t a_smem, int chunk, uint32_t accumulate) {
         const uint64_t ad = make_smem_desc(a_smem + k * 32, 16, 1024, kSwizzle128B);
         const uint64_t bd = make_smem_desc(q_u32 + chunk * QCHUNK + k * 32, 16, 1024, kSwizzle128B);
         mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, accumulate);
       };
-      if (n == 0 || t == 0) {
+      if (n == 0 || cur.seq_first()) {
         ok = mbar_wait(bar(&misc->q_full), seg & 1, abort_word, a.error_word, 4);
         if (!ok) break;
         ++seg;
@@ -308,7 +414,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       }
       if (!ok) break;
       mma_commit(bar(&misc->s_full[n & 1]));
-      if (n + 1 == n_tiles || t + 1 == tps) mma_commit(bar(&misc->q_empty));   // segment's last tile
+      if (n + 1 == n_tiles || cur.seq_last()) mma_commit(bar(&misc->q_empty));   // segment's last tile
     }
   } else if (warp > kQkIssuers && warp <= kQkIssuers + kPvIssuers && lane == 0) {
     // ------------------------------------------------------------------ value issuer j
@@ -316,13 +422,13 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     // are published, and hands the pairs it read back to the producer.
     const int j = warp - 1 - kQkIssuers;
     bool ok = true;
-    int t = (int)(g0 % tps);
-    for (int n = 0; n < n_tiles && ok; ++n, ++t) {
-      if (t == (int)tps) t = 0;
+    TileCursor<RAGGED> cur;
+    cur.locate(g0, tps_u, prefix, a.batch);
+    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix)) {
       ok = mbar_wait(bar(&misc->p_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 12);
       if (!ok) break;
       tc_fence_after_sync();
-      const bool seg_first = n == 0 || t == 0;
+      const bool seg_first = n == 0 || cur.seq_first();
       for (int mb = j; mb < RP; mb += kPvIssuers) {
         const int buf = (n * RP + mb) % kPairs;
         const uint32_t src = pairs_u32 + buf * kPairBytes;
@@ -381,15 +487,15 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       return is_max ? fmaxf(fmaxf(r0[0], r0[32]), fmaxf(r0[64], r0[96])) : r0[0] + r0[32] + r0[64] + r0[96];
     };
     float l_acc[NHH];
-    int b = (int)(g0 / tps), t = (int)(g0 - (long long)b * tps);
-    for (int n = 0; n < n_tiles; ++n, ++t) {
-      if (t == (int)tps) {
-        t = 0;
-        ++b;
-      }
-      const bool seg_first = n == 0 || t == 0;
-      const bool seg_last = n + 1 == n_tiles || t + 1 == (int)tps;
+    TileCursor<RAGGED> cur;
+    cur.locate(g0, tps_u, prefix, a.batch);
+    int n_slots = a.n_slots;
+    for (int n = 0; n < n_tiles; ++n, cur.next(prefix)) {
+      const int b = cur.b, t = cur.t;
+      const bool seg_first = n == 0 || cur.seq_first();
+      const bool seg_last = n + 1 == n_tiles || cur.seq_last();
       if (seg_first) {
+        if constexpr (RAGGED) n_slots = ceil_div(__ldg(a.seq_tokens + b), a.stride);
         // New sequence: empty references (shared by all threads) and denominators.
         if (sidx < 32) misc->m_used[sidx] = -INFINITY;
 #pragma unroll
@@ -414,7 +520,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
                  (__uint_as_float(sp[2][i]) + __uint_as_float(sp[3][i]));
         tc_fence_before_sync();
       }
-      const bool valid = ok && active && t * kTile + row < a.n_slots;
+      const bool valid = ok && active && t * kTile + row < n_slots;
       float m_ref[NHH];
       bool exceed = false;
 #pragma unroll
@@ -540,8 +646,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         __threadfence();
       }
       // Ticket: the CTA that delivers the sequence's last partial combines them.
-      const long long c_first = share_owner((long long)b * tps, total, G);
-      const int n_parts = (int)(share_owner((long long)(b + 1) * tps - 1, total, G) - c_first) + 1;
+      const long long seq_start = cur.start(prefix);
+      const long long c_first = share_owner(seq_start, total, G);
+      const int n_parts = (int)(share_owner(seq_start + cur.tps - 1, total, G) - c_first) + 1;
       group_sync();
       if (sidx == 0) {
         int last = 0;

@@ -26,19 +26,21 @@ struct PostArgs {
   const float* beta;      // [r]
   const float* hyp_c_w;   // [r][d_w] fp32
   const float* hyp_c_b;   // [d_w]
-  const float* gate_pe;   // [d_w]: Linear(pe_j) of Eq. 13 for this step's slot number j
+  const float* gate_pe;   // [max_slots][d_w]: row j0 is Linear(pe_{j0+1}) of Eq. 13
   const float* gate_s;    // [d_w]: gamma^T A        (folded gate only)
   const float* gate_t;    // [d_w]: beta^T A + a     (folded gate only)
-  const float* rope_cos;  // [d_R/2] for this step's position
-  const float* rope_sin;  // [d_R/2]
+  const float* rope_cos;  // [max_tokens][d_R/2]
+  const float* rope_sin;  // [max_tokens][d_R/2]
   float* open_acc;        // [B][r] fp32 running sum of the open slot
-  void* cache;            // [max_batch][max_slots][r + d_R]
+  CacheView cache;
+  int* seq_tokens;        // [B] tokens each sequence has consumed, advanced by this kernel; or
+                          // nullptr when all sequences stand at `tokens`
   void* qt;               // [B][n_h][r + d_R] absorbed query; this kernel writes the RoPE tail
   bf16* q16;              // [B][2*n_h*d_h]: q as bf16 [hi | lo] halves (q = hi + lo) for the
                           // tensor-core absorption, or nullptr
   int n_heads, head_dim, r, dr, dw;
-  int max_slots, slot;    // slot = 0-based slot index receiving this token
-  int new_slot;           // 1 when the token opens the slot (tokens mod s == 0)
+  int tokens;             // tokens consumed so far = 0-based index of this token (lock-step batch)
+  int stride;             // s: slot tokens / s receives the token, opened when tokens mod s == 0
   int use_gate;           // 0 at s == 1 (w = 1)
   float ln_eps;
   float q_scale;          // log2(e) / sqrt(d_h), folded into the absorbed query
@@ -125,6 +127,12 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   const float* row = a.p1 + (long long)b * a.proj.width;
   ptx::grid_launch_dependents();
   ptx::grid_dependency_wait();   // the projection kernel's output is read from here on
+  const int i0 = a.seq_tokens ? a.seq_tokens[b] : a.tokens;
+  const int slot = i0 / a.stride;
+  const bool new_slot = i0 % a.stride == 0;
+  const float* gate_pe = a.gate_pe + (long long)slot * a.dw;
+  const float* rope_cos = a.rope_cos + (long long)i0 * (a.dr / 2);
+  const float* rope_sin = a.rope_sin + (long long)i0 * (a.dr / 2);
 
   // LayerNorm over r (two-pass variance).
   float s = 0.f;
@@ -148,22 +156,22 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   float w = 1.f;
   if (a.use_gate)
     w = a.proj.off_u >= 0
-            ? gate_weight_folded(row + a.proj.off_u, a.dw, mean, rstd, a.gate_s, a.gate_t, a.gate_pe, red_s)
-            : gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, a.gate_pe, a.r, a.dw, part_s, red_s);
+            ? gate_weight_folded(row + a.proj.off_u, a.dw, mean, rstd, a.gate_s, a.gate_t, gate_pe, red_s)
+            : gate_weight(c_s, a.hyp_c_w, a.hyp_c_b, gate_pe, a.r, a.dw, part_s, red_s);
 
   // Slot update: fp32 running sum, stored to the cache in the storage type.
   const int W = a.r + a.dr;
-  T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + a.slot) * W;
+  T* slot_row = static_cast<T*>(a.cache.base) + cache_row(a.cache, b, slot) * W;
   float* acc = a.open_acc + (long long)b * a.r;
   for (int i = tid; i < a.r; i += 256) {
-    const float v = (a.new_slot ? 0.f : acc[i]) + w * c_s[i];
+    const float v = (new_slot ? 0.f : acc[i]) + w * c_s[i];
     acc[i] = v;
     slot_row[i] = Elem<T>::from_float(v);
   }
   // RoPE key of this token replaces the slot's key.
   for (int k = tid; k < a.dr / 2; k += 256) {
     const float x0 = row[a.proj.off_kr + 2 * k], x1 = row[a.proj.off_kr + 2 * k + 1];
-    const float cs = a.rope_cos[k], sn = a.rope_sin[k];
+    const float cs = rope_cos[k], sn = rope_sin[k];
     slot_row[a.r + 2 * k] = Elem<T>::from_float(x0 * cs - x1 * sn);
     slot_row[a.r + 2 * k + 1] = Elem<T>::from_float(x0 * sn + x1 * cs);
   }
@@ -185,18 +193,21 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
     const int h = i / half, k = i % half;
     const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k];
     const float x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
-    const float cs = a.rope_cos[k], sn = a.rope_sin[k];
+    const float cs = rope_cos[k], sn = rope_sin[k];
     qt[h * W + a.r + 2 * k] = Elem<TQ>::from_float((x0 * cs - x1 * sn) * a.q_scale);
     qt[h * W + a.r + 2 * k + 1] = Elem<TQ>::from_float((x0 * sn + x1 * cs) * a.q_scale);
   }
+  // Every thread read the position before the first block-wide reduction above.
+  if (a.seq_tokens && tid == 0) a.seq_tokens[b] = i0 + 1;
 }
 
 struct AttnArgs {
   const void* qt;      // [B][n_h][r + d_R], pre-scaled by log2(e)/sqrt(d_h)
-  const void* cache;   // [max_batch][max_slots][r + d_R]
+  CacheView cache;
   float* o_part;       // [B * n_split][n_h][r] un-normalised partial outputs
   float* ml_part;      // [B * n_split][n_h][2]: running max (log2 units), sum
-  int n_heads, r, dr, max_slots, n_slots, slots_per_split, n_split;
+  const int* seq_tokens;   // [B] tokens per sequence (this step's included), or nullptr: n_slots
+  int n_heads, r, dr, stride, n_slots, slots_per_split, n_split;
 };
 
 constexpr int kAttnFmaTile = 16;
@@ -224,9 +235,11 @@ __global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
   float* fac_s = m_s + NH;
   const int tid = threadIdx.x, b = blockIdx.y, split = blockIdx.x;
   const int slot0 = split * a.slots_per_split;
-  const int slot1 = min(a.n_slots, slot0 + a.slots_per_split);
+  // A split beyond a short sequence's end leaves an empty partial (maximum -inf, sum 0).
+  const int n_slots = a.seq_tokens ? ceil_div(a.seq_tokens[b], a.stride) : a.n_slots;
+  const int slot1 = min(n_slots, slot0 + a.slots_per_split);
   const TQ* qt = static_cast<const TQ*>(a.qt) + (long long)b * a.n_heads * W;
-  const T* cache = static_cast<const T*>(a.cache) + (long long)b * a.max_slots * W;
+  const T* cache = static_cast<const T*>(a.cache.base);
 
   for (int v = tid; v < NH * (W / VQ); v += 256) {
     const int h = v / (W / VQ), kv = (v % (W / VQ)) * VQ;
@@ -254,7 +267,7 @@ __global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
       const int sl = v / (W / V), kv = (v % (W / V)) * V;
       float tmp[V];
       if (t0 + sl < slot1) {
-        load_vec(cache + (long long)(t0 + sl) * W + kv, tmp);
+        load_vec(cache + cache_row(a.cache, b, t0 + sl) * W + kv, tmp);
       } else {
 #pragma unroll
         for (int e = 0; e < V; ++e) tmp[e] = 0.f;

@@ -4,6 +4,7 @@
 
 #include <cuda.h>
 #include <math.h>
+#include <algorithm>
 #include <new>
 #include <stdlib.h>
 #include <string.h>
@@ -18,6 +19,8 @@
 #include "prefill_attn_tc.cuh"
 #include "prefill_kernels.cuh"
 #include "setup_kernels.cuh"
+#include "paging_kernels.cuh"
+#include "page_pool.h"
 
 using namespace mtla;
 
@@ -41,6 +44,7 @@ struct ArenaPlan {
   size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
   size_t gate_s, gate_t, gate_tmp;
   size_t cache, open_acc, err_flag;
+  size_t page_table, seq_tokens;   // paged handles: two buffers each (beam reordering flips them)
   size_t p1, q16, qt, o_part, ml_part, o, v, x_stage, y_stage, gemm_part, gemm_tickets, attn_tickets;
   size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
   size_t total;
@@ -48,11 +52,12 @@ struct ArenaPlan {
 
 struct Dims {
   int d, nh, dh, r, dr, dw, s, W, ntot, max_slots, max_units;
+  int n_pages, max_pages;   // paged handles: pool size, pages per sequence; 0 otherwise
   size_t elem;
   ProjLayout proj;
 };
 
-bool normalise(const mtla_config* in, mtla_config* out, Dims* dm) {
+bool normalise(const mtla_config* in, const mtla_paging* pg, mtla_config* out, Dims* dm) {
   if (!in) return false;
   mtla_config c = *in;
   if (c.hyper_dim == 0) c.hyper_dim = c.latent_rank / 4;
@@ -88,6 +93,14 @@ bool normalise(const mtla_config* in, mtla_config* out, Dims* dm) {
   dm->ntot = dm->proj.width;
   dm->max_slots = ceil_div(c.max_tokens, c.stride);
   dm->max_units = kTargetCtas + c.max_batch;
+  dm->n_pages = dm->max_pages = 0;
+  if (pg) {
+    if (pg->page_slots != kPageSlots || pg->n_pages < 0) return false;
+    dm->max_pages = ceil_div(dm->max_slots, kPageSlots);
+    const long long full = (long long)c.max_batch * dm->max_pages;
+    if (full > (1ll << 30) || pg->n_pages > full) return false;
+    dm->n_pages = pg->n_pages ? pg->n_pages : (int)full;
+  }
   return true;
 }
 
@@ -116,8 +129,11 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->gate_tmp = take(dm.proj.off_u >= 0 ? ((size_t)dm.dw * dm.r + (size_t)dm.dw * dm.d) * 4 : 0);
   p->rope_cos = take((size_t)c.max_tokens * (dm.dr / 2) * 4);
   p->rope_sin = take((size_t)c.max_tokens * (dm.dr / 2) * 4);
-  p->cache = take(B * dm.max_slots * dm.W * e);
-  p->open_acc = take(B * dm.r * 4);
+  const size_t paged = dm.n_pages > 0;
+  p->cache = take(paged ? (size_t)dm.n_pages * kPageSlots * dm.W * e : B * dm.max_slots * dm.W * e);
+  p->open_acc = take((1 + paged) * B * dm.r * 4);
+  p->page_table = take(paged * 2 * B * dm.max_pages * sizeof(int));
+  p->seq_tokens = take(paged * 2 * B * sizeof(int));
   p->err_flag = take(16);
   p->p1 = take(B * dm.ntot * 4);
   p->q16 = take(B * 2 * hd * 2);
@@ -159,8 +175,14 @@ struct mtla_handle {
   Dims dm;
   ArenaPlan plan;
   char* arena;
-  int tokens;   // tokens consumed per sequence
+  int tokens;   // tokens consumed per sequence (paged handles: the longest sequence's)
   int batch;    // 0 while the cache is empty and no batch has been fixed
+  // Paged handles (mtla_create_paged): per-sequence positions and the page pool.  The device
+  // keeps its own copy of the positions, advanced by the decode step's kernels; host-side
+  // changes (prefill, import, reset) mark it stale and the next call re-sends them.
+  PagePool* pool;
+  std::vector<int> seq_tokens;
+  bool tokens_stale;
   int64_t launches;
   bool attn_smem_ready, pf_smem_ready;
   // Tensor-core decode attention (bf16, r a multiple of 128): TMA view of the cache.
@@ -178,6 +200,25 @@ struct mtla_handle {
   bool prof_attention_only;   // record only the two events around the attention kernel
 
   template <typename P> P* at(size_t off) const { return reinterpret_cast<P*>(arena + off); }
+  bool paged() const { return pool != nullptr; }
+  int buf() const { return pool ? pool->current_buffer() : 0; }
+  int* d_page_table(int which) const {
+    return at<int>(plan.page_table) + (size_t)which * cfg.max_batch * dm.max_pages;
+  }
+  int* d_seq_tokens(int which) const { return at<int>(plan.seq_tokens) + (size_t)which * cfg.max_batch; }
+  float* d_open_acc(int which) const {
+    return at<float>(plan.open_acc) + (size_t)which * cfg.max_batch * dm.r;
+  }
+  // The cache as the kernels address it, under the current page table.
+  CacheView cache_view() const {
+    CacheView v;
+    v.base = at<void>(plan.cache);
+    v.page_table = pool ? d_page_table(buf()) : nullptr;
+    v.max_pages = dm.max_pages;
+    v.max_slots = dm.max_slots;
+    return v;
+  }
+  int seq_len(int b) const { return pool ? seq_tokens[b] : tokens; }
 };
 
 namespace {
@@ -245,8 +286,11 @@ int make_cache_map(mtla_handle* h) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return MTLA_ERR_CUDA;
   const Dims& dm = h->dm;
-  const cuuint64_t dims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.max_slots, (cuuint64_t)h->cfg.max_batch};
-  const cuuint64_t strides[2] = {(cuuint64_t)dm.W * 2, (cuuint64_t)dm.max_slots * dm.W * 2};
+  // Paged: the planes are the pool's 64-slot pages instead of the sequences' row ranges.
+  const cuuint64_t plane_rows = h->paged() ? kPageSlots : dm.max_slots;
+  const cuuint64_t planes = h->paged() ? dm.n_pages : h->cfg.max_batch;
+  const cuuint64_t dims[3] = {(cuuint64_t)dm.W, plane_rows, planes};
+  const cuuint64_t strides[2] = {(cuuint64_t)dm.W * 2, plane_rows * dm.W * 2};
   const cuuint32_t box[3] = {64, (cuuint32_t)tc::kTile, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   CUresult rc = fn(
@@ -389,23 +433,24 @@ GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, i
   return g;
 }
 
-template <int NHP>
+template <int NHP, bool RAGGED>
 int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_t st, bool dependent) {
+  constexpr int kSmem = RAGGED ? tc::kSmemBytesRagged : tc::kSmemBytes;
 #define MTLA_TC_CASE(RP)                                                                       \
   case RP:                                                                                     \
     if (!h->attn_smem_ready) {                                                                 \
       /* The kernel re-allocates registers between warpgroups; its launch-time pool must */    \
       /* cover the budget, or the increase inside the kernel would never be granted.     */    \
       cudaFuncAttributes fa;                                                                   \
-      MTLA_CUDA(cudaFuncGetAttributes(&fa, decode_attn_tc_kernel<NHP, RP>));                   \
+      MTLA_CUDA(cudaFuncGetAttributes(&fa, decode_attn_tc_kernel<NHP, RP, RAGGED>));                   \
       if (fa.numRegs * tc::kThreads < (tc::kThreads - tc::kSoftmaxThreads) * tc::kRegsIssuer + \
                                           tc::kSoftmaxThreads * tc::kRegsSoftmax)              \
         return MTLA_ERR_CUDA;                                                                  \
-      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP>,                           \
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes)); \
+      MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP, RAGGED>,                           \
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem)); \
     }                                                                                          \
-    MTLA_CUDA(launch_kernel(decode_attn_tc_kernel<NHP, RP>, dim3(grid), dim3(tc::kThreads),    \
-                            tc::kSmemBytes, st, dependent, h->cache_map, h->q_map, a));        \
+    MTLA_CUDA(launch_kernel(decode_attn_tc_kernel<NHP, RP, RAGGED>, dim3(grid), dim3(tc::kThreads),    \
+                            kSmem, st, dependent, h->cache_map, h->q_map, a));                 \
     break;
   switch (a.r / 128) {
     MTLA_TC_CASE(1)
@@ -479,8 +524,9 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.err_flag), 0, 16, st));
   // Unused cache rows must hold finite values: the tensor-core kernel multiplies rows
   // beyond the valid range by a zero probability.
-  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.cache), 0,
-                            (size_t)h->cfg.max_batch * dm.max_slots * dm.W * dm.elem, st));
+  const size_t cache_rows = h->paged() ? (size_t)dm.n_pages * kPageSlots
+                                       : (size_t)h->cfg.max_batch * dm.max_slots;
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.cache), 0, cache_rows * dm.W * dm.elem, st));
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.gemm_tickets), 0, (size_t)kGemmSlots * 4 * sizeof(int), st));
   MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.attn_tickets), 0, (size_t)h->cfg.max_batch * sizeof(int), st));
   if (h->use_tc) {
@@ -563,9 +609,21 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   const Dims& dm = h->dm;
   const ArenaPlan& p = h->plan;
   const int hd = dm.nh * dm.dh;
-  const int i0 = h->tokens;            // 0-based index of this token
-  const int slot = i0 / dm.s;
-  const int n_slots = slot + 1;
+  // Lock-step batches: every sequence is at token i0.  Paged handles: each at its own, kept on
+  // the device; n_slots is then the longest sequence's count after this step.
+  const int i0 = h->tokens;
+  int n_slots = i0 / dm.s + 1;
+  long long ragged_tiles = 0;
+  if (h->paged()) {
+    n_slots = 0;
+    for (int b = 0; b < B; ++b) {
+      const int nb = h->seq_tokens[b] / dm.s + 1;
+      n_slots = max(n_slots, nb);
+      ragged_tiles += ceil_div(nb, tc::kTile);
+    }
+  }
+  const int buf = h->buf();
+  int* seq_tokens = h->paged() ? h->d_seq_tokens(buf) : nullptr;
 
   const bool prof = h->prof_used + MTLA_DECODE_STAGES + 1 <= (int)h->prof_events.size();
   MTLA_TRY(prof_mark(h, prof, 0, st));
@@ -591,18 +649,18 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   pa.beta = h->at<float>(p.beta);
   pa.hyp_c_w = h->at<float>(p.hyp_c_w);
   pa.hyp_c_b = h->at<float>(p.hyp_c_b);
-  pa.gate_pe = h->at<float>(p.gate_pe) + (size_t)slot * dm.dw;
+  pa.gate_pe = h->at<float>(p.gate_pe);
   pa.gate_s = h->at<float>(p.gate_s);
   pa.gate_t = h->at<float>(p.gate_t);
-  pa.rope_cos = h->at<float>(p.rope_cos) + (size_t)i0 * (dm.dr / 2);
-  pa.rope_sin = h->at<float>(p.rope_sin) + (size_t)i0 * (dm.dr / 2);
-  pa.open_acc = h->at<float>(p.open_acc);
-  pa.cache = h->at<void>(p.cache);
+  pa.rope_cos = h->at<float>(p.rope_cos);
+  pa.rope_sin = h->at<float>(p.rope_sin);
+  pa.open_acc = h->d_open_acc(buf);
+  pa.cache = h->cache_view();
+  pa.seq_tokens = seq_tokens;
   pa.qt = h->at<void>(p.qt);
   pa.q16 = h->use_tc ? h->at<bf16>(p.q16) : nullptr;
   pa.n_heads = dm.nh; pa.head_dim = dm.dh; pa.r = dm.r; pa.dr = dm.dr; pa.dw = dm.dw;
-  pa.max_slots = dm.max_slots; pa.slot = slot;
-  pa.new_slot = (i0 % dm.s) == 0;
+  pa.tokens = i0; pa.stride = dm.s;
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
@@ -632,10 +690,11 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   MTLA_TRY(prof_mark(h, prof, 3, st));
   AttnArgs aa;
   aa.qt = h->at<void>(p.qt);
-  aa.cache = h->at<void>(p.cache);
+  aa.cache = h->cache_view();
   aa.o_part = scratch ? scratch->o_part : h->at<float>(p.o_part);
   aa.ml_part = scratch ? scratch->ml_part : h->at<float>(p.ml_part);
-  aa.n_heads = dm.nh; aa.r = dm.r; aa.dr = dm.dr; aa.max_slots = dm.max_slots;
+  aa.seq_tokens = seq_tokens;
+  aa.n_heads = dm.nh; aa.r = dm.r; aa.dr = dm.dr; aa.stride = dm.s;
   aa.n_slots = n_slots;
   if (h->use_tc) {
     // One persistent CTA per SM; the step's 64-slot tiles are dealt out in equal shares, and
@@ -647,12 +706,20 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     ta.error_word = h->at<int>(p.err_flag);
     ta.n_heads = dm.nh; ta.r = dm.r; ta.dr = dm.dr; ta.n_slots = n_slots; ta.batch = B;
     ta.tiles_per_seq = ceil_div(n_slots, tc::kTile);
-    const long long total = (long long)B * ta.tiles_per_seq;
+    ta.seq_tokens = seq_tokens;
+    ta.page_table = h->paged() ? h->d_page_table(buf) : nullptr;
+    ta.max_pages = dm.max_pages; ta.stride = dm.s;
+    const long long total = h->paged() ? ragged_tiles : (long long)B * ta.tiles_per_seq;
     const int grid = (int)(total < kSmCount ? total : kSmCount);
     aa.n_split = 0;
     const bool attn_pdl = pdl && !prof;     // the attention kernel is bracketed by events when timed
-    if (dm.nh <= 16) MTLA_TRY(launch_attn_tc_rp<16>(h, ta, grid, st, attn_pdl));
-    else MTLA_TRY(launch_attn_tc_rp<32>(h, ta, grid, st, attn_pdl));
+    if (h->paged()) {
+      if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, true>(h, ta, grid, st, attn_pdl)));
+      else MTLA_TRY((launch_attn_tc_rp<32, true>(h, ta, grid, st, attn_pdl)));
+    } else {
+      if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, false>(h, ta, grid, st, attn_pdl)));
+      else MTLA_TRY((launch_attn_tc_rp<32, false>(h, ta, grid, st, attn_pdl)));
+    }
   } else {
     int want = ceil_div(kTargetCtas, B);
     int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
@@ -696,7 +763,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
 }
 
 template <typename T>
-int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaStream_t st) {
+int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void* y, cudaStream_t st) {
   const Dims& dm = h->dm;
   const ArenaPlan& p = h->plan;
   const int hd = dm.nh * dm.dh;
@@ -727,8 +794,9 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   pa.gate_t = h->at<float>(p.gate_t);
   pa.rope_cos = h->at<float>(p.rope_cos);
   pa.rope_sin = h->at<float>(p.rope_sin);
-  pa.open_acc = h->at<float>(p.open_acc);
-  pa.cache = h->at<void>(p.cache);
+  pa.open_acc = h->d_open_acc(h->buf());
+  pa.cache = h->cache_view();
+  pa.seq0 = seq0;
   pa.qcat = h->at<void>(p.pf_qcat);
   pa.cprime = h->at<void>(p.pf_cprime);
   pa.kr = h->at<void>(p.pf_kr);
@@ -831,6 +899,58 @@ int prefill_impl(mtla_handle* h, const void* x, int B, int T_len, void* y, cudaS
   return MTLA_OK;
 }
 
+// dst[idx] = val for every pair, in launches of at most kScatterOps pairs.
+int send_scatter(mtla_handle* h, int* dst, const std::vector<int>& idx, const std::vector<int>& val,
+                 cudaStream_t st) {
+  for (size_t at = 0; at < idx.size(); at += kScatterOps) {
+    IntScatter ops;
+    ops.n = (int)std::min<size_t>(kScatterOps, idx.size() - at);
+    for (int i = 0; i < ops.n; ++i) {
+      ops.idx[i] = idx[at + i];
+      ops.val[i] = val[at + i];
+    }
+    int_scatter_kernel<<<ceil_div(ops.n, 128), 128, 0, st>>>(dst, ops);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
+  return MTLA_OK;
+}
+
+// Re-sends the per-sequence positions after the host changed them.
+int sync_tokens(mtla_handle* h, cudaStream_t st) {
+  if (!h->paged() || !h->tokens_stale) return MTLA_OK;
+  std::vector<int> idx(h->cfg.max_batch), val(h->seq_tokens);
+  for (int b = 0; b < h->cfg.max_batch; ++b) idx[b] = b;
+  MTLA_TRY(send_scatter(h, h->d_seq_tokens(h->buf()), idx, val, st));
+  h->tokens_stale = false;
+  return MTLA_OK;
+}
+
+// Enqueues what the page pool decided: page copies first, then the table entries.
+int apply_page_ops(mtla_handle* h, const std::vector<PageSet>& sets, const std::vector<PageCopy>& copies,
+                   cudaStream_t st) {
+  const long long page_bytes = (long long)kPageSlots * h->dm.W * h->dm.elem;
+  for (size_t at = 0; at < copies.size(); at += kPageCopyOps) {
+    PageCopies ops;
+    ops.n = (int)std::min<size_t>(kPageCopyOps, copies.size() - at);
+    for (int i = 0; i < ops.n; ++i) {
+      ops.src[i] = copies[at + i].src;
+      ops.dst[i] = copies[at + i].dst;
+      ops.rows[i] = copies[at + i].rows;
+    }
+    page_copy_kernel<<<ops.n, 256, 0, st>>>(h->at<char>(h->plan.cache), page_bytes,
+                                            (int)(h->dm.W * h->dm.elem), ops);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
+  std::vector<int> idx(sets.size()), val(sets.size());
+  for (size_t i = 0; i < sets.size(); ++i) {
+    idx[i] = sets[i].seq * h->dm.max_pages + sets[i].index;
+    val[i] = sets[i].page;
+  }
+  return send_scatter(h, h->d_page_table(h->buf()), idx, val, st);
+}
+
 int check_step_args(mtla_handle* h, const void* x, int32_t B, const void* y) {
   if (!h || !x || !y || B <= 0) return MTLA_ERR_INVALID_ARG;
   if (h->batch == 0) {
@@ -838,9 +958,83 @@ int check_step_args(mtla_handle* h, const void* x, int32_t B, const void* y) {
   } else if (B != h->batch) {
     return MTLA_ERR_BATCH_MISMATCH;
   }
-  if (h->tokens + 1 > h->cfg.max_tokens) return MTLA_ERR_CAPACITY;
+  if (!h->paged()) return h->tokens + 1 > h->cfg.max_tokens ? MTLA_ERR_CAPACITY : MTLA_OK;
+  if (h->use_tc && B > tc::kMaxRaggedBatch) return MTLA_ERR_CAPACITY;
+  int need = 0;
+  for (int b = 0; b < B; ++b) {
+    if (h->seq_tokens[b] + 1 > h->cfg.max_tokens) return MTLA_ERR_CAPACITY;
+    const int slot = h->seq_tokens[b] / h->dm.s;
+    need += h->pool->pages_needed(b, slot + 1, slot);
+  }
+  return need > h->pool->pages_free() ? MTLA_ERR_CAPACITY : MTLA_OK;
+}
+
+// Paged handles, before the kernels of a decode step: every sequence gets the page its new
+// token's slot lives in, private to it (copy-on-write after a beam fork).
+int step_begin(mtla_handle* h, int B, cudaStream_t st) {
+  if (!h->paged()) return MTLA_OK;
+  MTLA_TRY(sync_tokens(h, st));
+  std::vector<PageSet> sets;
+  std::vector<PageCopy> copies;
+  for (int b = 0; b < B; ++b) {
+    const int slot = h->seq_tokens[b] / h->dm.s;
+    if (!h->pool->prepare(b, slot + 1, slot, &sets, &copies)) return MTLA_ERR_STATE;
+  }
+  return apply_page_ops(h, sets, copies, st);
+}
+
+void step_end(mtla_handle* h, int B) {
+  if (h->paged()) {
+    for (int b = 0; b < B; ++b) {
+      h->seq_tokens[b] += 1;
+      h->tokens = max(h->tokens, h->seq_tokens[b]);
+    }
+  } else {
+    h->tokens += 1;
+  }
+  h->batch = B;
+}
+
+template <typename T>
+int dispatch_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
+                    const AttnScratch* scratch) {
+  MTLA_TRY(step_begin(h, B, st));
+  MTLA_TRY(decode_impl<T>(h, x, B, y, st, scratch));
+  step_end(h, B);
   return MTLA_OK;
 }
+
+int run_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
+               const AttnScratch* scratch = nullptr) {
+  return h->cfg.dtype == MTLA_DTYPE_BF16 ? dispatch_decode<bf16>(h, x, B, y, st, scratch)
+                                         : dispatch_decode<float>(h, x, B, y, st, scratch);
+}
+
+// Prefill of sequences seq0 .. seq0 + B - 1 (all empty), T tokens each.
+int run_prefill(mtla_handle* h, const void* x, int seq0, int B, int T, void* y, cudaStream_t st) {
+  const int n_slots = ceil_div(T, h->dm.s);
+  if (h->paged()) {
+    if (B * PagePool::pages_for(n_slots) > h->pool->pages_free()) return MTLA_ERR_CAPACITY;
+    std::vector<PageSet> sets;
+    std::vector<PageCopy> copies;
+    for (int b = seq0; b < seq0 + B; ++b)
+      if (!h->pool->prepare(b, n_slots, -1, &sets, &copies)) return MTLA_ERR_STATE;
+    MTLA_TRY(apply_page_ops(h, sets, copies, st));
+  }
+  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? prefill_impl<bf16>(h, x, seq0, B, T, y, st)
+                                                 : prefill_impl<float>(h, x, seq0, B, T, y, st);
+  if (rc != MTLA_OK) return rc;
+  if (h->paged()) {
+    for (int b = seq0; b < seq0 + B; ++b) h->seq_tokens[b] = T;
+    h->tokens_stale = true;
+  }
+  h->tokens = max(h->tokens, T);
+  h->batch = max(h->batch, seq0 + B);
+  return MTLA_OK;
+}
+
+int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_weights* w, void* arena,
+                  size_t arena_bytes, void* stream, mtla_handle** out);
 
 }  // namespace
 
@@ -849,7 +1043,16 @@ extern "C" {
 size_t mtla_arena_bytes(const mtla_config* cfg) {
   mtla_config c;
   Dims dm;
-  if (!normalise(cfg, &c, &dm)) return 0;
+  if (!normalise(cfg, nullptr, &c, &dm)) return 0;
+  ArenaPlan p;
+  plan_arena(c, dm, &p);
+  return p.total;
+}
+
+size_t mtla_arena_bytes_paged(const mtla_config* cfg, const mtla_paging* paging) {
+  mtla_config c;
+  Dims dm;
+  if (!paging || !normalise(cfg, paging, &c, &dm)) return 0;
   ArenaPlan p;
   plan_arena(c, dm, &p);
   return p.total;
@@ -857,10 +1060,25 @@ size_t mtla_arena_bytes(const mtla_config* cfg) {
 
 int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size_t arena_bytes,
                 void* stream, mtla_handle** out) {
+  return create_handle(cfg, nullptr, w, arena, arena_bytes, stream, out);
+}
+
+int mtla_create_paged(const mtla_config* cfg, const mtla_paging* paging, const mtla_weights* w,
+                      void* arena, size_t arena_bytes, void* stream, mtla_handle** out) {
+  if (!paging) return MTLA_ERR_INVALID_ARG;
+  return create_handle(cfg, paging, w, arena, arena_bytes, stream, out);
+}
+
+}  // extern "C"
+
+namespace {
+
+int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_weights* w, void* arena,
+                  size_t arena_bytes, void* stream, mtla_handle** out) {
   if (!cfg || !w || !arena || !out) return MTLA_ERR_INVALID_ARG;
   mtla_config c;
   Dims dm;
-  if (!normalise(cfg, &c, &dm)) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  if (!normalise(cfg, paging, &c, &dm)) return MTLA_ERR_UNSUPPORTED_SHAPE;
   const void* required[] = {w->w_q, w->w_qr, w->w_r, w->w_kr, w->ln_gamma, w->ln_beta,
                             w->w_k, w->w_v, w->w_o, w->hyp_c_w, w->hyp_pe_w};
   for (const void* ptr : required)
@@ -878,6 +1096,17 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   h->prof_attention_only = false;
   h->act_bn = 0;
   h->gemm_attr_mask = 0;
+  h->pool = nullptr;
+  h->tokens_stale = false;
+  if (paging) {
+    h->pool = new (std::nothrow) PagePool(dm.n_pages, c.max_batch, dm.max_pages);
+    if (!h->pool) {
+      delete h;
+      return MTLA_ERR_INVALID_ARG;
+    }
+    h->seq_tokens.assign(c.max_batch, 0);
+    h->tokens_stale = true;
+  }
   // The tensor-core attention needs bf16 and whole 128-column latent blocks; the
   // MTLA_ATTENTION=fma environment override keeps the CUDA-core kernel for comparisons.
   const char* force = getenv("MTLA_ATTENTION");
@@ -885,6 +1114,7 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int rc = c.dtype == MTLA_DTYPE_BF16 ? create_impl<bf16>(h, w, st) : create_impl<float>(h, w, st);
   if (rc != MTLA_OK) {
+    delete h->pool;
     delete h;
     return rc;
   }
@@ -892,32 +1122,37 @@ int mtla_create(const mtla_config* cfg, const mtla_weights* w, void* arena, size
   return MTLA_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
 int mtla_prefill(mtla_handle* h, const void* x, int32_t B, int32_t T, void* y, void* stream) {
   if (!h || !x || B <= 0 || T <= 0) return MTLA_ERR_INVALID_ARG;
   if (!aligned16(x) || (y && !aligned16(y))) return MTLA_ERR_INVALID_ARG;
-  if (h->tokens != 0) return MTLA_ERR_STATE;
+  if (h->tokens != 0 || h->batch != 0) return MTLA_ERR_STATE;
   if (B > h->cfg.max_batch || T > h->cfg.max_prefill_tokens || T > h->cfg.max_tokens)
     return MTLA_ERR_CAPACITY;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? prefill_impl<bf16>(h, x, B, T, y, st)
-                                                 : prefill_impl<float>(h, x, B, T, y, st);
-  if (rc != MTLA_OK) return rc;
-  h->tokens = T;
-  h->batch = B;
-  return MTLA_OK;
+  return run_prefill(h, x, 0, B, T, y, static_cast<cudaStream_t>(stream));
+}
+
+int mtla_prefill_seqs(mtla_handle* h, int32_t seq0, const void* x, int32_t B, int32_t T, void* y,
+                      void* stream) {
+  if (!h || !x || B <= 0 || T <= 0 || seq0 < 0) return MTLA_ERR_INVALID_ARG;
+  if (!aligned16(x) || (y && !aligned16(y))) return MTLA_ERR_INVALID_ARG;
+  if (!h->paged()) return MTLA_ERR_STATE;
+  if (seq0 > h->batch) return MTLA_ERR_STATE;           // sequences are numbered without gaps
+  if (seq0 + B > h->cfg.max_batch || T > h->cfg.max_prefill_tokens || T > h->cfg.max_tokens)
+    return MTLA_ERR_CAPACITY;
+  for (int b = seq0; b < seq0 + B; ++b)
+    if (h->seq_tokens[b] != 0) return MTLA_ERR_STATE;
+  return run_prefill(h, x, seq0, B, T, y, static_cast<cudaStream_t>(stream));
 }
 
 int mtla_decode_step(mtla_handle* h, const void* x, int32_t B, void* y, void* stream) {
   const int chk = check_step_args(h, x, B, y);
   if (chk != MTLA_OK) return chk;
   if (!aligned16(x) || !aligned16(y)) return MTLA_ERR_INVALID_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? decode_impl<bf16>(h, x, B, y, st)
-                                                 : decode_impl<float>(h, x, B, y, st);
-  if (rc != MTLA_OK) return rc;
-  h->tokens += 1;
-  h->batch = B;
-  return MTLA_OK;
+  return run_decode(h, x, B, y, static_cast<cudaStream_t>(stream));
 }
 
 int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y_host,
@@ -929,12 +1164,8 @@ int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y
   void* xs = h->at<void>(h->plan.x_stage);
   void* ys = h->at<void>(h->plan.y_stage);
   MTLA_CUDA(cudaMemcpyAsync(xs, x_host, bytes, cudaMemcpyHostToDevice, st));
-  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? decode_impl<bf16>(h, xs, B, ys, st)
-                                                 : decode_impl<float>(h, xs, B, ys, st);
-  if (rc != MTLA_OK) return rc;
+  MTLA_TRY(run_decode(h, xs, B, ys, st));
   MTLA_CUDA(cudaMemcpyAsync(y_host, ys, bytes, cudaMemcpyDeviceToHost, st));
-  h->tokens += 1;
-  h->batch = B;
   return MTLA_OK;
 }
 
@@ -966,22 +1197,20 @@ int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, v
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // The array keeps whatever the previous call left: the tickets must start at zero.
   MTLA_CUDA(cudaMemsetAsync(sc.tickets, 0, (size_t)B * sizeof(int), st));
-  const int rc = h->cfg.dtype == MTLA_DTYPE_BF16 ? decode_impl<bf16>(h, x, B, y, st, &sc)
-                                                 : decode_impl<float>(h, x, B, y, st, &sc);
-  if (rc != MTLA_OK) return rc;
-  h->tokens += 1;
-  h->batch = B;
-  return MTLA_OK;
+  return run_decode(h, x, B, y, st, &sc);
 }
 
 size_t mtla_cache_bytes(const mtla_handle* h) {
   if (!h) return 0;
-  return (size_t)h->batch * ceil_div(h->tokens, h->dm.s) * h->dm.W * h->dm.elem;
+  size_t slots = 0;
+  for (int b = 0; b < h->batch; ++b) slots += ceil_div(h->seq_len(b), h->dm.s);
+  return slots * h->dm.W * h->dm.elem;
 }
 
 int mtla_destroy(mtla_handle* h) {
   if (!h) return MTLA_ERR_INVALID_ARG;
   for (cudaEvent_t e : h->prof_events) cudaEventDestroy(e);
+  delete h->pool;
   delete h;
   return MTLA_OK;
 }
@@ -990,6 +1219,11 @@ int mtla_reset(mtla_handle* h) {
   if (!h) return MTLA_ERR_INVALID_ARG;
   h->tokens = 0;
   h->batch = 0;
+  if (h->paged()) {
+    h->pool->reset();
+    h->seq_tokens.assign(h->cfg.max_batch, 0);
+    h->tokens_stale = true;
+  }
   return MTLA_OK;
 }
 
@@ -1006,6 +1240,18 @@ int mtla_cache_export(mtla_handle* h, void* dst, size_t bytes, void* stream) {
   const size_t need = mtla_cache_bytes(h);
   if (bytes < need) return MTLA_ERR_CAPACITY;
   if (need == 0) return MTLA_OK;
+  if (h->paged()) {
+    if (!aligned16(dst)) return MTLA_ERR_INVALID_ARG;
+    for (int b = 0; b < h->batch; ++b)
+      if (h->seq_tokens[b] != h->tokens) return MTLA_ERR_STATE;   // ragged: use mtla_cache_export_seq
+    const int n_slots = ceil_div(h->tokens, h->dm.s);
+    cache_rows_copy_kernel<<<dim3(ceil_div(n_slots, kPageSlots), h->batch), 256, 0,
+                             static_cast<cudaStream_t>(stream)>>>(
+        h->cache_view(), 0, n_slots, (int)(h->dm.W * h->dm.elem), static_cast<char*>(dst), 0);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+    return MTLA_OK;
+  }
   const size_t row = (size_t)ceil_div(h->tokens, h->dm.s) * h->dm.W * h->dm.elem;
   const size_t pitch = (size_t)h->dm.max_slots * h->dm.W * h->dm.elem;
   MTLA_CUDA(cudaMemcpy2DAsync(dst, row, h->at<char>(h->plan.cache), pitch, row, h->batch,
@@ -1020,23 +1266,139 @@ int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens
   const int n_slots = ceil_div(tokens, h->dm.s);
   const size_t row = (size_t)n_slots * h->dm.W * h->dm.elem;
   const size_t pitch = (size_t)h->dm.max_slots * h->dm.W * h->dm.elem;
-  MTLA_CUDA(cudaMemcpy2DAsync(h->at<char>(h->plan.cache), pitch, src, row, row, B,
-                              cudaMemcpyDeviceToDevice, st));
+  if (h->paged()) {
+    // The import replaces everything: all pages go back to the pool first.
+    if ((long long)B * PagePool::pages_for(n_slots) > h->pool->n_pages()) return MTLA_ERR_CAPACITY;
+    h->pool->reset();
+    std::vector<PageSet> sets;
+    std::vector<PageCopy> copies;
+    for (int b = 0; b < B; ++b)
+      if (!h->pool->prepare(b, n_slots, -1, &sets, &copies)) return MTLA_ERR_STATE;
+    MTLA_TRY(apply_page_ops(h, sets, copies, st));
+    cache_rows_copy_kernel<<<dim3(ceil_div(n_slots, kPageSlots), B), 256, 0, st>>>(
+        h->cache_view(), 0, n_slots, (int)(h->dm.W * h->dm.elem),
+        const_cast<char*>(static_cast<const char*>(src)), 1);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+    h->seq_tokens.assign(h->cfg.max_batch, 0);
+    for (int b = 0; b < B; ++b) h->seq_tokens[b] = tokens;
+    h->tokens_stale = true;
+  } else {
+    MTLA_CUDA(cudaMemcpy2DAsync(h->at<char>(h->plan.cache), pitch, src, row, row, B,
+                                cudaMemcpyDeviceToDevice, st));
+  }
   if (tokens % h->dm.s != 0) {
     if (h->cfg.dtype == MTLA_DTYPE_BF16)
-      open_acc_from_cache_kernel<bf16><<<B, 256, 0, st>>>(h->at<bf16>(h->plan.cache),
-                                                          h->at<float>(h->plan.open_acc), h->dm.r,
-                                                          h->dm.W, h->dm.max_slots, n_slots - 1);
+      open_acc_from_cache_kernel<bf16><<<B, 256, 0, st>>>(h->cache_view(), h->d_open_acc(h->buf()),
+                                                          h->dm.r, h->dm.W, 0, n_slots - 1);
     else
-      open_acc_from_cache_kernel<float><<<B, 256, 0, st>>>(h->at<float>(h->plan.cache),
-                                                           h->at<float>(h->plan.open_acc), h->dm.r,
-                                                           h->dm.W, h->dm.max_slots, n_slots - 1);
+      open_acc_from_cache_kernel<float><<<B, 256, 0, st>>>(h->cache_view(), h->d_open_acc(h->buf()),
+                                                           h->dm.r, h->dm.W, 0, n_slots - 1);
     h->launches++;
     MTLA_CUDA(cudaGetLastError());
   }
   h->tokens = tokens;
   h->batch = B;
   return MTLA_OK;
+}
+
+int mtla_beam_reorder(mtla_handle* h, const int32_t* parents, int32_t n_new, void* stream) {
+  if (!h || !parents || n_new <= 0) return MTLA_ERR_INVALID_ARG;
+  if (!h->paged() || h->batch == 0) return MTLA_ERR_STATE;
+  if (n_new > h->cfg.max_batch) return MTLA_ERR_CAPACITY;
+  for (int b = 0; b < n_new; ++b)
+    if (parents[b] < 0 || parents[b] >= h->batch) return MTLA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  MTLA_TRY(sync_tokens(h, st));
+  const int old = h->buf(), nxt = old ^ 1;
+  BeamArgs a;
+  a.tokens_old = h->d_seq_tokens(old); a.tokens_new = h->d_seq_tokens(nxt);
+  a.table_old = h->d_page_table(old); a.table_new = h->d_page_table(nxt);
+  a.acc_old = h->d_open_acc(old); a.acc_new = h->d_open_acc(nxt);
+  a.max_pages = h->dm.max_pages; a.r = h->dm.r; a.stride = h->dm.s;
+  for (int at = 0; at < n_new; at += kBeamChunk) {
+    BeamParents p;
+    p.n = min(kBeamChunk, n_new - at);
+    p.first = at;
+    for (int i = 0; i < p.n; ++i) p.parent[i] = parents[at + i];
+    beam_gather_kernel<<<p.n, 128, 0, st>>>(a, p);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
+  h->pool->reorder(parents, n_new, h->batch);
+  std::vector<int> moved(h->cfg.max_batch, 0);
+  h->tokens = 0;
+  for (int b = 0; b < n_new; ++b) {
+    moved[b] = h->seq_tokens[parents[b]];
+    h->tokens = max(h->tokens, moved[b]);
+  }
+  h->seq_tokens.swap(moved);
+  h->batch = n_new;
+  // Rows beyond the new batch keep stale positions on the device; they are re-sent (as 0) with
+  // the next host-side change and are not read before.
+  return MTLA_OK;
+}
+
+int mtla_seq_positions(const mtla_handle* h, int32_t* tokens, int32_t n) {
+  if (!h || !tokens || n < 0 || n > h->cfg.max_batch) return MTLA_ERR_INVALID_ARG;
+  for (int b = 0; b < n; ++b) tokens[b] = b < h->batch ? h->seq_len(b) : 0;
+  return MTLA_OK;
+}
+
+int64_t mtla_pages_in_use(const mtla_handle* h) { return h && h->paged() ? h->pool->pages_in_use() : -1; }
+
+int mtla_cache_export_seq(mtla_handle* h, int32_t seq, void* dst, size_t bytes, void* stream) {
+  if (!h || !dst || !aligned16(dst) || seq < 0 || seq >= h->batch) return MTLA_ERR_INVALID_ARG;
+  const int n_slots = ceil_div(h->seq_len(seq), h->dm.s);
+  if (bytes < (size_t)n_slots * h->dm.W * h->dm.elem) return MTLA_ERR_CAPACITY;
+  if (n_slots == 0) return MTLA_OK;
+  cache_rows_copy_kernel<<<dim3(ceil_div(n_slots, kPageSlots), 1), 256, 0,
+                           static_cast<cudaStream_t>(stream)>>>(
+      h->cache_view(), seq, n_slots, (int)(h->dm.W * h->dm.elem), static_cast<char*>(dst), 0);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  return MTLA_OK;
+}
+
+/* Host-only access to the page pool's decisions (no GPU involved). */
+mtla_page_pool* mtla_page_pool_create(int32_t n_pages, int32_t max_seqs, int32_t max_pages_per_seq) {
+  if (n_pages <= 0 || max_seqs <= 0 || max_pages_per_seq <= 0) return nullptr;
+  return reinterpret_cast<mtla_page_pool*>(new (std::nothrow) PagePool(n_pages, max_seqs, max_pages_per_seq));
+}
+void mtla_page_pool_destroy(mtla_page_pool* p) { delete reinterpret_cast<PagePool*>(p); }
+int mtla_page_pool_prepare(mtla_page_pool* pp, int32_t seq, int32_t n_slots, int32_t write_slot,
+                           int32_t* copies, int32_t max_copies) {
+  PagePool* p = reinterpret_cast<PagePool*>(pp);
+  if (!p || seq < 0 || n_slots < 0) return MTLA_ERR_INVALID_ARG;
+  if (p->pages_needed(seq, n_slots, write_slot) > p->pages_free()) return MTLA_ERR_CAPACITY;
+  std::vector<PageSet> sets;
+  std::vector<PageCopy> cp;
+  if (!p->prepare(seq, n_slots, write_slot, &sets, &cp)) return MTLA_ERR_STATE;
+  for (size_t i = 0; i < cp.size() && (int)i < max_copies; ++i) {
+    copies[3 * i] = cp[i].src; copies[3 * i + 1] = cp[i].dst; copies[3 * i + 2] = cp[i].rows;
+  }
+  return (int)cp.size();
+}
+int mtla_page_pool_reorder(mtla_page_pool* pp, const int32_t* parents, int32_t n_new, int32_t n_old) {
+  PagePool* p = reinterpret_cast<PagePool*>(pp);
+  if (!p || !parents || n_new <= 0 || n_old <= 0) return MTLA_ERR_INVALID_ARG;
+  p->reorder(parents, n_new, n_old);
+  return MTLA_OK;
+}
+int mtla_page_pool_row(const mtla_page_pool* pp, int32_t seq, int32_t* pages, int32_t max_pages) {
+  const PagePool* p = reinterpret_cast<const PagePool*>(pp);
+  if (!p || seq < 0) return MTLA_ERR_INVALID_ARG;
+  const int n = p->pages_held(seq);
+  for (int k = 0; k < n && k < max_pages; ++k) pages[k] = p->row(seq)[k];
+  return n;
+}
+int mtla_page_pool_in_use(const mtla_page_pool* pp) {
+  const PagePool* p = reinterpret_cast<const PagePool*>(pp);
+  return p ? p->pages_in_use() : MTLA_ERR_INVALID_ARG;
+}
+int mtla_page_pool_ref(const mtla_page_pool* pp, int32_t page) {
+  const PagePool* p = reinterpret_cast<const PagePool*>(pp);
+  return p && page >= 0 && page < p->n_pages() ? p->ref(page) : MTLA_ERR_INVALID_ARG;
 }
 
 int mtla_check(mtla_handle* h, void* stream) {

@@ -22,7 +22,8 @@ struct PrefillPostArgs {
   const float* rope_cos;  // [max_tokens][d_R/2]
   const float* rope_sin;
   float* open_acc;        // [B][r]
-  void* cache;            // [max_batch][max_slots][r + d_R]
+  CacheView cache;
+  int seq0;               // the call's sequences are seq0, seq0 + 1, ... of the cache
   void* qcat;             // [B*T][n_h][d_h + d_R]: scaled query and rotated RoPE query
   void* cprime;           // [B*T][r]: running merge state after each token (Eq. 14's sequence)
   void* kr;               // [B*T][d_R]: rotated RoPE key of each token (query element type)
@@ -111,13 +112,13 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
 
   // The chunk's state after its last available token is what the cache holds.
   const long long last = (long long)b * a.T + (tok1 - 1);
-  T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + chunk) * W;
+  T* slot_row = static_cast<T*>(a.cache.base) + cache_row(a.cache, a.seq0 + b, chunk) * W;
   const TQ* kr = static_cast<const TQ*>(a.kr) + last * a.dr;
   for (int i = tid; i < a.r; i += 256) slot_row[i] = Elem<T>::from_float(acc_s[i]);
   for (int i = tid; i < a.dr; i += 256)
     slot_row[a.r + i] = Elem<T>::from_float(Elem<TQ>::to_float(kr[i]));
   if (tok1 == a.T)
-    for (int i = tid; i < a.r; i += 256) a.open_acc[(long long)b * a.r + i] = acc_s[i];
+    for (int i = tid; i < a.r; i += 256) a.open_acc[(long long)(a.seq0 + b) * a.r + i] = acc_s[i];
 }
 
 // The same work for layers whose gate needs no matrix (folded into the projection, or absent at
@@ -175,7 +176,7 @@ __global__ void __launch_bounds__(256) prefill_post_fast_kernel(PrefillPostArgs 
   __syncthreads();
 
   // Running merge state after each token (Eq. 14's sequence), final state into the cache.
-  T* slot_row = static_cast<T*>(a.cache) + ((long long)b * a.max_slots + chunk) * W;
+  T* slot_row = static_cast<T*>(a.cache.base) + cache_row(a.cache, a.seq0 + b, chunk) * W;
   for (int i = tid; i < a.r; i += 256) {
     float acc = 0.f;
     for (int t = 0; t < ntok; ++t) {
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(256) prefill_post_fast_kernel(PrefillPostArgs 
       static_cast<T*>(a.cprime)[(row0 + t) * a.r + i] = Elem<T>::from_float(acc);
     }
     slot_row[i] = Elem<T>::from_float(acc);
-    if (tok0 + ntok == a.T) a.open_acc[(long long)b * a.r + i] = acc;
+    if (tok0 + ntok == a.T) a.open_acc[(long long)(a.seq0 + b) * a.r + i] = acc;
   }
   // RoPE keys (rounded to the cache type, which is what decoding reads back); the slot keeps
   // the key of the chunk's last token.

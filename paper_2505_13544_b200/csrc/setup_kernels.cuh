@@ -101,12 +101,13 @@ __global__ void rope_table_kernel(float* cos_t, float* sin_t, int positions, int
   sin_t[i] = (float)sin(angle);
 }
 
-// Initialises the fp32 accumulator of the open slot from a stored cache row.
+// Initialises the fp32 accumulator of the open slot of sequences seq0 + blockIdx.x from the
+// stored cache row `slot`.
 template <typename T>
-__global__ void open_acc_from_cache_kernel(const T* cache, float* open_acc, int r, int W,
-                                           int max_slots, int slot) {
-  const int b = blockIdx.x;
-  const T* row = cache + ((long long)b * max_slots + slot) * W;
+__global__ void open_acc_from_cache_kernel(CacheView cache, float* open_acc, int r, int W,
+                                           int seq0, int slot) {
+  const int b = seq0 + blockIdx.x;
+  const T* row = static_cast<const T*>(cache.base) + cache_row(cache, b, slot) * W;
   for (int i = threadIdx.x; i < r; i += blockDim.x)
     open_acc[(long long)b * r + i] = Elem<T>::to_float(row[i]);
 }

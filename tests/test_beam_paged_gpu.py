@@ -1,0 +1,149 @@
+"""Paged cache, ragged batches and beam re-parenting on the GPU, through the C ABI, against
+the CPU oracle's per-sequence states (copied on every re-parenting)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mtla_oracle as O
+from paper_2505_13544_b200 import binding as M
+from paper_2505_13544_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+PAGE = 64
+
+
+def paged_handle(w, weights, max_batch, max_tokens, max_prefill, n_pages=0):
+    cfg = M.make_config(**H.dims_of(w), max_batch=max_batch, max_tokens=max_tokens,
+                        max_prefill_tokens=max_prefill, dtype=w.dtype, ln_eps=w.ln_eps,
+                        rope_theta=w.rope_theta)
+    return M.mtla_create_paged(cfg, {k: v.cuda() for k, v in weights.items()}, n_pages=n_pages)
+
+
+def slots_of(tokens, s):
+    return -(-tokens // s)
+
+
+def beam_search_against_oracle(w, n_utt, beam, lengths, steps, reorder_every=1):
+    """Ragged prompts (one per utterance, copied to its `beam` hypotheses by a re-parenting),
+    then decode steps with a re-parenting in between; every output is compared."""
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    n_seq = n_utt * beam
+    h = paged_handle(w, weights, n_seq, max(lengths) + steps, max(lengths))
+    try:
+        # One prefill call per utterance builds the ragged batch of n_utt sequences.
+        states = []
+        for u, t_len in enumerate(lengths):
+            x = synth.stored(synth.normal(w.seed, f"utt/{u}", (1, t_len, w.d_model)), w.dtype)
+            y = M.mtla_prefill_seqs(h, u, x.cuda())
+            want, st = O.decode_sequence(p, x[0].double().numpy())
+            H.assert_close(y[0], want, w.dtype, f"prefill of utterance {u}")
+            states.append(st)
+        assert M.mtla_seq_positions(h) == list(lengths)
+        assert M.mtla_pages_in_use(h) == sum(-(-slots_of(t, w.stride) // PAGE) for t in lengths)
+        # Fork every utterance into its beam.
+        parents = [u for u in range(n_utt) for _ in range(beam)]
+        M.mtla_beam_reorder(h, parents)
+        states = O.reorder_states(states, parents)
+        assert M.mtla_pages_in_use(h) == sum(-(-slots_of(t, w.stride) // PAGE) for t in lengths)
+        for i in range(steps):
+            x = synth.stored(synth.normal(w.seed, f"beam_x/{i}", (n_seq, w.d_model)), w.dtype)
+            y = M.mtla_decode_step(h, x.cuda())
+            want = np.stack([O.decode_step(p, states[b], x[b].double().numpy()) for b in range(n_seq)])
+            H.assert_close(y, want, w.dtype, f"decode step {i}")
+            assert M.mtla_seq_positions(h) == [st.tokens for st in states]
+            if (i + 1) % reorder_every == 0:
+                parents = synth.beam_parents(w.seed, i, n_utt, beam)
+                M.mtla_beam_reorder(h, parents)
+                states = O.reorder_states(states, parents)
+        M.mtla_check(h)
+        assert M.mtla_cache_bytes(h) == sum(st.n_slots for st in states) * w.slot_width * (
+            4 if w.dtype == "fp32" else 2)
+        for b in range(n_seq):
+            H.assert_cache_close(M.mtla_cache_export_seq(h, b), O.cache_array(states[b]), w.dtype)
+        # Shared pages count once: never more than unshared storage would need.
+        assert M.mtla_pages_in_use(h) <= sum(-(-st.n_slots // PAGE) for st in states)
+    finally:
+        M.mtla_destroy(h)
+
+
+@pytest.mark.parametrize("s", [1, 2, 3])
+def test_beam_search_fp32(s):
+    """CUDA-core path at fp32 tolerance; prompts below, at and above a page boundary."""
+    w = synth.WORKLOADS["tiny"].scaled(stride=s, seed=20 + s)
+    lengths = [PAGE * s - 1, PAGE * s, PAGE * s + 1, 5, 2 * PAGE * s + s + 1]
+    beam_search_against_oracle(w, n_utt=5, beam=3, lengths=lengths, steps=2 * s + 70)
+
+
+@pytest.mark.parametrize("s,heads", [(2, 8), (3, 32)])
+def test_beam_search_bf16_tensor_cores(s, heads):
+    w = synth.WORKLOADS["paper"].scaled(stride=s, n_heads=heads, seed=30 + s)
+    lengths = [PAGE * s * 2 + 3, 17, PAGE * s, 3 * PAGE * s - 1]
+    beam_search_against_oracle(w, n_utt=4, beam=4, lengths=lengths, steps=40)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("paper", {"prefill_tokens": 300, "decode_steps": 140})])
+def test_lock_step_on_a_paged_handle_is_bit_identical(name, kw):
+    """Same kernels, same order of operations: only the slot addresses differ."""
+    w = synth.WORKLOADS[name].scaled(batch=3, **kw)
+    weights = synth.make_weights(w)
+    flat = H.gpu_handle(w, weights, max_tokens=w.max_tokens + 1)
+    paged = paged_handle(w, weights, w.batch, w.max_tokens + 1, w.prefill_tokens)
+    try:
+        x = synth.prompt(w).cuda()
+        assert torch.equal(M.mtla_prefill(flat, x), M.mtla_prefill(paged, x))
+        for i in range(w.decode_steps):
+            xi = synth.decode_input(w, i).cuda()
+            assert torch.equal(M.mtla_decode_step(flat, xi), M.mtla_decode_step(paged, xi)), i
+        assert torch.equal(M.mtla_cache_export(flat), M.mtla_cache_export(paged))
+        assert M.mtla_position(flat) == M.mtla_position(paged)
+        # Export, re-import into the paged handle, continue: still identical.
+        cache = M.mtla_cache_export(flat)
+        tokens = M.mtla_position(flat)[0]
+        M.mtla_cache_import(paged, cache, tokens)
+        xi = synth.decode_input(w, 0).cuda()
+        assert torch.equal(M.mtla_decode_step(flat, xi), M.mtla_decode_step(paged, xi))
+        M.mtla_check(flat)
+        M.mtla_check(paged)
+    finally:
+        M.mtla_destroy(flat)
+        M.mtla_destroy(paged)
+
+
+def test_pool_exhaustion_is_reported_before_anything_runs():
+    w = synth.WORKLOADS["tiny"].scaled(batch=2)
+    weights = synth.make_weights(w)
+    h = paged_handle(w, weights, 2, 4 * PAGE * w.stride, 2 * PAGE * w.stride, n_pages=3)
+    try:
+        x = synth.prompt(w, batch=2, tokens=PAGE * w.stride).cuda()      # one full page each
+        M.mtla_prefill(h, x)
+        xi = synth.decode_input(w, 0, batch=2).cuda()
+        with pytest.raises(M.MTLAError) as err:      # both sequences need a second page; one is left
+            M.mtla_decode_step(h, xi)
+        assert err.value.status == -4
+        assert M.mtla_seq_positions(h) == [PAGE * w.stride] * 2 and M.mtla_pages_in_use(h) == 2
+        M.mtla_beam_reorder(h, [1])                  # keep one hypothesis: its page need fits
+        M.mtla_decode_step(h, xi[:1].contiguous())
+        assert M.mtla_seq_positions(h) == [PAGE * w.stride + 1] and M.mtla_pages_in_use(h) == 2
+        M.mtla_reset(h)
+        assert M.mtla_pages_in_use(h) == 0 and M.mtla_position(h) == (0, 0, 0)
+        M.mtla_check(h)
+    finally:
+        M.mtla_destroy(h)
+
+
+def test_paging_calls_are_refused_without_paging():
+    w = synth.WORKLOADS["tiny"]
+    h = H.gpu_handle(w, synth.make_weights(w))
+    try:
+        with pytest.raises(M.MTLAError) as err:
+            M.mtla_beam_reorder(h, [0])
+        assert err.value.status == -7
+        with pytest.raises(M.MTLAError) as err:
+            M.mtla_prefill_seqs(h, 0, synth.prompt(w).cuda())
+        assert err.value.status == -7
+        assert M.mtla_pages_in_use(h) == -1
+    finally:
+        M.mtla_destroy(h)
