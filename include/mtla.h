@@ -196,6 +196,12 @@ int mtla_cache_export(mtla_handle* h, void* dst, size_t bytes, void* stream);
  * accumulator is initialised from the stored value. */
 int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens, void* stream);
 
+/* Paged handles only: mtla_cache_import for the empty sequences seq0 .. seq0 + B - 1, leaving
+ * the others as they are; src device [B][ceil(tokens/s)][r + d_R].  seq0 may not exceed the
+ * current batch; the batch becomes max(batch, seq0 + B). */
+int mtla_cache_import_seqs(mtla_handle* h, int32_t seq0, const void* src, int32_t B, int32_t tokens,
+                           void* stream);
+
 /* Beam reordering (paged handles): sequence b of the new batch continues old sequence
  * parents[b] (host array of n_new indices into the current batch; an index may repeat or be
  * absent).  Positions, page tables and the fp32 state of the open slot follow on `stream`;

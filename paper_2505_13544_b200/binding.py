@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = (
     "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
     "mtla_profile_end_stages", "mtla_decode_step_static", "mtla_profile_begin_attention",
     "mtla_arena_bytes_paged", "mtla_create_paged", "mtla_prefill_seqs", "mtla_beam_reorder",
-    "mtla_seq_positions", "mtla_pages_in_use", "mtla_cache_export_seq",
+    "mtla_seq_positions", "mtla_pages_in_use", "mtla_cache_export_seq", "mtla_cache_import_seqs",
     "mtla_page_pool_create", "mtla_page_pool_destroy", "mtla_page_pool_prepare",
     "mtla_page_pool_reorder", "mtla_page_pool_row", "mtla_page_pool_in_use", "mtla_page_pool_ref")
 
@@ -78,6 +78,7 @@ def load_library() -> ctypes.CDLL:
         "mtla_create_paged": (ctypes.c_int, [cfg_p, pg_p, w_p, vp, sz, vp, ctypes.POINTER(vp)]),
         "mtla_prefill_seqs": (ctypes.c_int, [vp, i32, vp, i32, i32, vp, vp]),
         "mtla_beam_reorder": (ctypes.c_int, [vp, i32_p, i32, vp]),
+        "mtla_cache_import_seqs": (ctypes.c_int, [vp, i32, vp, i32, i32, vp]),
         "mtla_seq_positions": (ctypes.c_int, [vp, i32_p, i32]),
         "mtla_pages_in_use": (ctypes.c_int64, [vp]),
         "mtla_cache_export_seq": (ctypes.c_int, [vp, i32, vp, sz, vp]),
@@ -239,6 +240,15 @@ def mtla_prefill_seqs(h: Handle, seq0: int, x: torch.Tensor, y: torch.Tensor | N
                                             y.data_ptr() if y is not None else None,
                                             _stream_ptr(stream)), "mtla_prefill_seqs")
     return y
+
+
+def mtla_cache_import_seqs(h: Handle, seq0: int, cache: torch.Tensor, tokens: int, stream=None) -> None:
+    """cache [B][ceil(tokens/s)][r + d_R] on the device, for the empty sequences seq0 .. seq0 + B - 1."""
+    b = cache.shape[0]
+    slots = -(-tokens // h.config.stride)
+    _expect(cache, h, (b, slots, h.config.latent_rank + h.config.rope_dim), "cache")
+    _check(load_library().mtla_cache_import_seqs(h.ptr, seq0, cache.data_ptr(), b, tokens,
+                                                 _stream_ptr(stream)), "mtla_cache_import_seqs")
 
 
 def _i32_array(values):

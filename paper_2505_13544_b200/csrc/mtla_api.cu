@@ -1302,6 +1302,43 @@ int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens
   return MTLA_OK;
 }
 
+int mtla_cache_import_seqs(mtla_handle* h, int32_t seq0, const void* src, int32_t B, int32_t tokens,
+                           void* stream) {
+  if (!h || !src || B <= 0 || tokens <= 0 || seq0 < 0 || !aligned16(src)) return MTLA_ERR_INVALID_ARG;
+  if (!h->paged() || seq0 > h->batch) return MTLA_ERR_STATE;
+  if (seq0 + B > h->cfg.max_batch || tokens > h->cfg.max_tokens) return MTLA_ERR_CAPACITY;
+  for (int b = seq0; b < seq0 + B; ++b)
+    if (h->seq_tokens[b] != 0) return MTLA_ERR_STATE;
+  const int n_slots = ceil_div(tokens, h->dm.s);
+  if ((long long)B * PagePool::pages_for(n_slots) > h->pool->pages_free()) return MTLA_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::vector<PageSet> sets;
+  std::vector<PageCopy> copies;
+  for (int b = seq0; b < seq0 + B; ++b)
+    if (!h->pool->prepare(b, n_slots, -1, &sets, &copies)) return MTLA_ERR_STATE;
+  MTLA_TRY(apply_page_ops(h, sets, copies, st));
+  cache_rows_copy_kernel<<<dim3(ceil_div(n_slots, kPageSlots), B), 256, 0, st>>>(
+      h->cache_view(), seq0, n_slots, (int)(h->dm.W * h->dm.elem),
+      const_cast<char*>(static_cast<const char*>(src)), 1);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  if (tokens % h->dm.s != 0) {
+    if (h->cfg.dtype == MTLA_DTYPE_BF16)
+      open_acc_from_cache_kernel<bf16><<<B, 256, 0, st>>>(h->cache_view(), h->d_open_acc(h->buf()),
+                                                          h->dm.r, h->dm.W, seq0, n_slots - 1);
+    else
+      open_acc_from_cache_kernel<float><<<B, 256, 0, st>>>(h->cache_view(), h->d_open_acc(h->buf()),
+                                                           h->dm.r, h->dm.W, seq0, n_slots - 1);
+    h->launches++;
+    MTLA_CUDA(cudaGetLastError());
+  }
+  for (int b = seq0; b < seq0 + B; ++b) h->seq_tokens[b] = tokens;
+  h->tokens_stale = true;
+  h->tokens = max(h->tokens, tokens);
+  h->batch = max(h->batch, seq0 + B);
+  return MTLA_OK;
+}
+
 int mtla_beam_reorder(mtla_handle* h, const int32_t* parents, int32_t n_new, void* stream) {
   if (!h || !parents || n_new <= 0) return MTLA_ERR_INVALID_ARG;
   if (!h->paged() || h->batch == 0) return MTLA_ERR_STATE;

@@ -165,6 +165,38 @@ def context_cache_row(w: Workload, seq: int, n_slots: int | None = None) -> torc
     return stored(row, w.dtype)
 
 
+@dataclass(frozen=True)
+class BeamWorkload:
+    """Beam-search decoding over utterances of different lengths: n_utt utterances with `beam`
+    hypotheses each (batch index = utterance * beam + rank), contexts of min_context ..
+    max_context tokens, a re-parenting after every decode step."""
+    name: str
+    layer: Workload       # dims, dtype, seed; its batch / context fields are not used
+    n_utt: int
+    beam: int
+    min_context: int
+    max_context: int
+    decode_steps: int
+
+    @property
+    def n_seq(self) -> int:
+        return self.n_utt * self.beam
+
+    def contexts(self) -> list[int]:
+        return ragged_lengths(self.layer.seed, self.n_utt, self.min_context, self.max_context)
+
+
+def _beam_workloads() -> dict:
+    # The paper decodes with beam sizes 10 to 50 on its d 512 models; the second entry is the
+    # beam-search counterpart of the "large" decode workload (16 x 8 = its 128 sequences).
+    return {
+        "beam_paper": BeamWorkload("beam_paper", WORKLOADS["paper"], n_utt=24, beam=10,
+                                   min_context=64, max_context=1024, decode_steps=64),
+        "beam_large": BeamWorkload("beam_large", WORKLOADS["large"], n_utt=16, beam=8,
+                                   min_context=8192, max_context=32768, decode_steps=72),
+    }
+
+
 def ragged_lengths(seed: int, n: int, lo: int, hi: int) -> list[int]:
     """n prompt lengths drawn uniformly from [lo, hi], a stand-in for utterances of
     different durations (the paper's test sets are variable-length speech and text)."""
@@ -184,3 +216,6 @@ def beam_parents(seed: int, step: int, n_utt: int, beam: int) -> list[int]:
         picks = np.sort(g.choice(beam, size=beam, p=weights))
         out += [u * beam + int(k) for k in picks]
     return out
+
+
+BEAM_WORKLOADS: dict[str, BeamWorkload] = _beam_workloads()

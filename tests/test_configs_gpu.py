@@ -139,3 +139,78 @@ def test_config_large_decode():
         H.assert_cache_close(tail, want_tail, "bf16")
     finally:
         M.mtla_destroy(h)
+
+
+def run_beam_workload(bw, utts, beams_checked, steps_checked):
+    """Beam search on a paged handle at the workload's full size: ragged contexts imported per
+    utterance, forked into beams, a re-parenting after every step.  The oracle follows whole
+    beams of the sampled utterances (state updates every step, outputs at the sampled steps)."""
+    w = bw.layer
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    contexts = bw.contexts()
+    s, beam = w.stride, bw.beam
+
+    def pages(tokens):
+        return -(-math.ceil(tokens / s) // M.PAGE_SLOTS)
+
+    cfg = M.make_config(**H.dims_of(w), max_batch=bw.n_seq, max_tokens=max(contexts) + bw.decode_steps,
+                        max_prefill_tokens=0, dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    # A pool that only fits because beams share their utterance's closed pages.
+    n_pages = sum(pages(t) for t in contexts) + bw.n_seq * (pages(bw.decode_steps) + 2)
+    assert n_pages < sum(beam * pages(t + bw.decode_steps) for t in contexts)
+    h = M.mtla_create_paged(cfg, {k: v.cuda() for k, v in weights.items()}, n_pages=n_pages)
+    try:
+        states = {}
+        for u, t in enumerate(contexts):
+            row = synth.context_cache_row(w, u, math.ceil(t / s))
+            M.mtla_cache_import_seqs(h, u, row[None].cuda(), t)
+            if u in utts:
+                states[u] = [O.state_from_cache(row.double().numpy(), t, p)]
+        assert M.mtla_seq_positions(h) == contexts
+        M.mtla_beam_reorder(h, [u for u in range(bw.n_utt) for _ in range(beam)])
+        for u in utts:
+            states[u] = O.reorder_states(states[u], [0] * beam)
+        assert M.mtla_pages_in_use(h) == sum(pages(t) for t in contexts)
+        for i in range(bw.decode_steps):
+            x = synth.stored(synth.normal(w.seed, f"beam_x/{i}", (bw.n_seq, w.d_model)), w.dtype)
+            y = M.mtla_decode_step(h, x.cuda())
+            check = i in steps_checked
+            for u in utts:
+                for k in range(beam):
+                    b = u * beam + k
+                    want = O.decode_step(p, states[u][k], x[b].double().numpy(),
+                                         want_output=check and k in beams_checked)
+                    if want is not None:
+                        H.assert_close(y[b], want, w.dtype, f"step {i}, utterance {u}, beam {k}")
+            if check:
+                M.mtla_check(h)
+            parents = synth.beam_parents(w.seed, i, bw.n_utt, beam)
+            M.mtla_beam_reorder(h, parents)
+            for u in utts:
+                states[u] = O.reorder_states(states[u], [q - u * beam for q in parents[u * beam:(u + 1) * beam]])
+        M.mtla_check(h)
+        assert M.mtla_seq_positions(h) == [t + bw.decode_steps for t in contexts for _ in range(beam)]
+        assert M.mtla_position(h) == (max(contexts) + bw.decode_steps,
+                                      math.ceil((max(contexts) + bw.decode_steps) / s), bw.n_seq)
+        assert M.mtla_cache_bytes(h) == sum(beam * math.ceil((t + bw.decode_steps) / s) for t in contexts) * (
+            w.slot_width * elem_bytes(w))
+        assert M.mtla_pages_in_use(h) <= n_pages
+        for u in utts:
+            for k in beams_checked:
+                H.assert_cache_close(M.mtla_cache_export_seq(h, u * beam + k),
+                                     O.cache_array(states[u][k]), w.dtype)
+    finally:
+        M.mtla_destroy(h)
+
+
+def test_beam_search_paper_scale():
+    """24 utterances x beam 10 on the paper's layer; three whole beams followed at every step."""
+    bw = synth.BEAM_WORKLOADS["beam_paper"]
+    run_beam_workload(bw, [0, 11, 23], set(range(bw.beam)), set(range(bw.decode_steps)))
+
+
+def test_beam_search_large():
+    """16 utterances x beam 8 at the large layer's size, contexts of 8k to 32k tokens."""
+    bw = synth.BEAM_WORKLOADS["beam_large"]
+    run_beam_workload(bw, [0, 15], {0, 3, 7}, {0, 1, 40, 71})
