@@ -214,15 +214,146 @@ def run_reference(args) -> None:
 
 # --------------------------------------------------------------------------- GPU arm
 
-def build_layer(w: synth.Workload, extra_steps: int, device):
+def build_layer(w: synth.Workload, extra_steps: int, device, paged: bool = False):
     from paper_2505_13544_b200 import binding as M
     weights = synth.make_weights(w)
     cfg = M.make_config(**dims_of(w), max_batch=w.batch,
                         max_tokens=w.prefill_tokens + w.context_tokens + extra_steps,
                         max_prefill_tokens=w.prefill_tokens, dtype=w.dtype, ln_eps=w.ln_eps,
                         rope_theta=w.rope_theta)
-    h = M.mtla_create(cfg, {k: v.to(device) for k, v in weights.items()}, device=device)
+    dev_weights = {k: v.to(device) for k, v in weights.items()}
+    h = (M.mtla_create_paged(cfg, dev_weights, device=device) if paged
+         else M.mtla_create(cfg, dev_weights, device=device))
     return M, h
+
+
+def run_beam(args, bw: synth.BeamWorkload, device, local: int) -> None:
+    """Beam-search decoding on a paged handle: ragged contexts, one re-parenting per step.
+    A step is mtla_decode_step for all hypotheses followed by mtla_beam_reorder."""
+    from paper_2505_13544_b200 import binding as M
+    w = bw.layer
+    K, W = args.steps, max(args.warmup, 3)
+    contexts = bw.contexts()
+    e = 2 if w.dtype == "bf16" else 4
+    weights = synth.make_weights(w)
+    cfg = M.make_config(**dims_of(w), max_batch=bw.n_seq, max_tokens=max(contexts) + 2 * (K + W),
+                        max_prefill_tokens=0, dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    h = M.mtla_create_paged(cfg, {k: v.to(device) for k, v in weights.items()}, device=device)
+    for u, t in enumerate(contexts):
+        row = synth.context_cache_row(w, u, -(-t // w.stride))
+        M.mtla_cache_import_seqs(h, u, row[None].to(device), t)
+    M.mtla_beam_reorder(h, [u for u in range(bw.n_utt) for _ in range(bw.beam)])
+    dt = synth.torch_dtype(w.dtype)
+    xs = [synth.stored(synth.normal(w.seed, f"beam_x/{i}", (bw.n_seq, w.d_model)), w.dtype).to(device)
+          for i in range(8)]
+    y = torch.empty(bw.n_seq, w.d_model, dtype=dt, device=device)
+    parents = [synth.beam_parents(w.seed, i, bw.n_utt, bw.beam) for i in range(64)]
+
+    def logical_bytes():
+        return sum(-(-t // w.stride) for t in M.mtla_seq_positions(h)) * w.slot_width * e
+
+    def page_bytes():
+        return M.mtla_pages_in_use(h) * M.PAGE_SLOTS * w.slot_width * e
+
+    step = 0
+    for _ in range(W):
+        M.mtla_decode_step(h, xs[step % 8], y)
+        M.mtla_beam_reorder(h, parents[step % 64])
+        step += 1
+    torch.cuda.synchronize(device)
+    bytes0, launches0 = logical_bytes(), M.mtla_launch_count(h)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    M.mtla_profile_begin_attention(h, K)
+    host0 = time.perf_counter()
+    with ClockSampler(local) as clocks:
+        torch.cuda.synchronize(device)
+        ev0.record()
+        for _ in range(K):
+            M.mtla_decode_step(h, xs[step % 8], y)
+            M.mtla_beam_reorder(h, parents[step % 64])
+            step += 1
+        ev1.record()
+        host_issue_s = time.perf_counter() - host0
+        torch.cuda.synchronize(device)
+    ms = ev0.elapsed_time(ev1)
+    attn_ms, attn_steps = M.mtla_profile_end(h)
+    launches = M.mtla_launch_count(h) - launches0
+    bytes1, distinct = logical_bytes(), page_bytes()
+    M.mtla_check(h)
+    assert torch.isfinite(y.float()).all()
+
+    xh = [x.cpu().pin_memory() for x in xs]
+    yh = torch.empty(bw.n_seq, w.d_model, dtype=dt).pin_memory()
+    for _ in range(W):
+        M.mtla_decode_step_host(h, xh[step % 8], yh)
+        M.mtla_beam_reorder(h, parents[step % 64])
+        step += 1
+    torch.cuda.synchronize(device)
+    ev0.record()
+    for _ in range(K):
+        M.mtla_decode_step_host(h, xh[step % 8], yh)
+        M.mtla_beam_reorder(h, parents[step % 64])
+        step += 1
+    ev1.record()
+    torch.cuda.synchronize(device)
+    e2e_ms = ev0.elapsed_time(ev1)
+    M.mtla_check(h)
+
+    peaks = measured_peaks()
+    cache_bytes = 0.5 * (bytes0 + bytes1)
+    attn_s = attn_ms * 1e-3 / max(attn_steps, 1)
+    achieved = cache_bytes / attn_s / 1e9
+    line = {
+        "metric": METRIC, "value": bw.n_seq * K / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": bw.name, "utterances": bw.n_utt, "beam": bw.beam, "batch": bw.n_seq,
+                   "context_tokens": [min(contexts), max(contexts)], "d_model": w.d_model,
+                   "n_heads": w.n_heads, "head_dim": w.head_dim, "latent_rank": w.latent_rank,
+                   "rope_dim": w.rope_dim, "stride": w.stride, "storage": "paged, 64-slot pages",
+                   "step": "decode step + beam re-parenting",
+                   "l2": "logical cache read per step %.0f MB, distinct pages %.0f MB (L2 126 MB)"
+                         % (cache_bytes / 1e6, distinct / 1e6),
+                   "attention_variant": M.mtla_attention_variant(h)},
+        "roofline": {"bound": "hbm", "kernel": "decode attention (a7), ragged paged",
+                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                     "launch_ms": attn_s * 1e3, "traffic": None,
+                     "note": "achieved counts every hypothesis' slots (logical bytes); beams of one "
+                             "utterance share pages, so part of it is served by L2 and the fraction "
+                             "can exceed 1"},
+        "cache": {"logical_bytes": cache_bytes, "distinct_page_bytes": distinct},
+        "e2e": {"value": bw.n_seq * K / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": bw.n_seq * w.d_model * e + 4 * bw.n_seq,
+                "d2h_bytes_per_step": bw.n_seq * w.d_model * e},
+        "host_issue_us_per_step": host_issue_s / K * 1e6,
+        "gpu_launches": int(launches),
+        "clocks": clocks.summary(),
+    }
+    M.mtla_destroy(h)
+    del h
+    torch.cuda.empty_cache()
+    if not args.no_cpu_baseline:
+        from oracle import mtla_oracle as O
+        p = O.params_from_tensors(dims_of(w), {k: v.double().numpy() for k, v in weights.items()},
+                                  ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+        t = contexts[0]
+        row = synth.context_cache_row(w, 0, -(-t // w.stride)).double().numpy()
+        states = O.reorder_states([O.state_from_cache(row, t, p)], [0] * bw.beam)
+        n, t0 = 0, time.perf_counter()
+        while n < 64 and time.perf_counter() - t0 < 12.0:
+            x = xs[n % 8][: bw.beam].double().cpu().numpy()
+            for k in range(bw.beam):
+                O.decode_step(p, states[k], x[k])
+            states = O.reorder_states(states, [q for q in parents[n % 64][: bw.beam]])
+            n += 1
+        el = time.perf_counter() - t0
+        from threadpoolctl import threadpool_info
+        cores = max([int(i.get("num_threads", 1)) for i in threadpool_info()] + [1])
+        line["cpu_baseline"] = {"value": bw.beam * n / el, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"the {bw.beam} hypotheses of utterance 0 ({t} context tokens) x "
+                                          f"{n} steps with re-parenting, {el:.1f} s"}
+    print(json.dumps(line))
 
 
 def fill_context(M, h, w: synth.Workload, device) -> dict:
@@ -268,7 +399,10 @@ def main() -> None:
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=8)
-    ap.add_argument("--workload", default="large", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="large",
+                    choices=sorted(synth.WORKLOADS) + sorted(synth.BEAM_WORKLOADS))
+    ap.add_argument("--paged", action="store_true",
+                    help="keep the cache in 64-slot pages (mtla_create_paged) instead of contiguous rows")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0,
@@ -277,6 +411,8 @@ def main() -> None:
                     help="override the workload's imported context length")
     args = ap.parse_args()
     if args.impl == "reference":
+        if args.workload in synth.BEAM_WORKLOADS:
+            raise SystemExit("--impl reference covers the decode workloads")
         run_reference(args)
         return
 
@@ -296,9 +432,14 @@ def main() -> None:
             dist.barrier(device_ids=[local])
         torch.cuda.synchronize(device)
 
+    if args.workload in synth.BEAM_WORKLOADS:
+        if world > 1:
+            raise SystemExit("the beam workloads run on one GPU")
+        run_beam(args, synth.BEAM_WORKLOADS[args.workload], device, local)
+        return
     w = pick_workload(args)
     K, W = args.steps, max(args.warmup, 3)
-    M, h = build_layer(w, extra_steps=3 * (K + W), device=device)
+    M, h = build_layer(w, extra_steps=3 * (K + W), device=device, paged=args.paged)
     extras = fill_context(M, h, w, device)
     dt = synth.torch_dtype(w.dtype)
     xs = [synth.decode_input(w, i).to(device) for i in range(8)]
@@ -385,6 +526,7 @@ def main() -> None:
                          f"({work['cache_bytes'] / 1e6:.0f} MB) and the weights"
                          if work["cache_bytes"] > 126e6 else
                          "cache smaller than L2: bandwidth figures are effective, not DRAM",
+                   "storage": "paged, 64-slot pages" if args.paged else "contiguous",
                    "attention_variant": M.mtla_attention_variant(h)},
         "roofline": {"bound": "hbm", "kernel": "decode attention (a7)",
                      "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",

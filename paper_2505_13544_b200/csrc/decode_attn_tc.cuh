@@ -141,6 +141,15 @@ struct Misc {
   float fac[32];
   float comb_m[32];
   float comb_w[8][32];     // combine: weight of part p for head h (first 8 parts cached)
+  // Ragged batches: the tile list's length, and the segment the softmax warps are in (kept
+  // here, written by one thread per segment, so that no thread carries a list position).
+  long long total_tiles;
+  int seg_b, seg_tiles, seg_tps, seg_start, seg_tail_rows;
+  // Per-tile flags (1 = first of its segment, 2 = last) from the producer to the score issuers,
+  // and "first of its segment" from the softmax warps to the value issuers, so that the issuers
+  // carry no list position; both are written before the mbarrier arrival that the reader waits for.
+  int tile_flags[16];
+  int pv_first[2];
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
 
@@ -175,31 +184,33 @@ __host__ __device__ inline long long share_owner(long long g, long long total, l
 template <bool RAGGED>
 struct TileCursor {
   int b, t, tps;
+  // `prefix` is the shared-memory address of the prefix sums (ragged batches only).
   // List index of the sequence's first tile.
-  __device__ __forceinline__ long long start(const int* prefix) const {
-    if constexpr (RAGGED) return prefix[b];
+  __device__ __forceinline__ long long start(uint32_t prefix) const {
+    if constexpr (RAGGED) return ptx::lds_i32(prefix + 4 * b);
     else return (long long)b * tps;
   }
-  __device__ __forceinline__ void locate(long long g, int tps_uniform, const int* prefix, int batch) {
+  __device__ __forceinline__ void locate(long long g, int tps_uniform, uint32_t prefix, int batch) {
     if constexpr (RAGGED) {
       int lo = 0, hi = batch;               // largest b with prefix[b] <= g
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (prefix[mid] <= g) lo = mid; else hi = mid;
+        if (ptx::lds_i32(prefix + 4 * mid) <= g) lo = mid; else hi = mid;
       }
       b = lo;
-      tps = prefix[b + 1] - prefix[b];
+      tps = ptx::lds_i32(prefix + 4 * b + 4) - ptx::lds_i32(prefix + 4 * b);
     } else {
       b = (int)(g / tps_uniform);
       tps = tps_uniform;
     }
     t = (int)(g - start(prefix));
   }
-  __device__ __forceinline__ void next(const int* prefix) {
+  __device__ __forceinline__ void next(uint32_t prefix) {
     if (++t == tps) {
       t = 0;
       ++b;
-      if constexpr (RAGGED) tps = prefix[b + 1] - prefix[b];   // prefix has one entry to spare
+      if constexpr (RAGGED)                  // the array has one entry to spare past the batch
+        tps = ptx::lds_i32(prefix + 4 * b + 4) - ptx::lds_i32(prefix + 4 * b);
     }
   }
   __device__ __forceinline__ bool seq_first() const { return t == 0; }
@@ -268,11 +279,11 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   grid_dependency_wait();        // nothing before this line touches the previous kernel's data
 
   // This CTA's share of the tile list.
-  int* prefix = reinterpret_cast<int*>(sm + kOffPrefix);     // ragged only
-  int* staged = reinterpret_cast<int*>(sm + kOffStaged);     // ragged only
+  const uint32_t prefix_s = base + kOffPrefix, staged_s = base + kOffStaged;   // ragged only
   long long total = (long long)a.batch * a.tiles_per_seq;
   if constexpr (RAGGED) {
     // prefix[b] = tiles of the sequences before b; prefix[batch + 1] repeats the total.
+    int* prefix = reinterpret_cast<int*>(sm + kOffPrefix);
     for (int i = threadIdx.x; i < a.batch; i += kThreads)
       prefix[i + 1] = ceil_div(ceil_div(a.seq_tokens[i], a.stride), kTile);
     __syncthreads();
@@ -296,16 +307,20 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     }
     __syncthreads();
     total = prefix[a.batch];
-    if (threadIdx.x == 0) prefix[a.batch + 1] = (int)total;
+    if (threadIdx.x == 0) {
+      prefix[a.batch + 1] = (int)total;
+      misc->total_tiles = total;
+    }
   }
   const long long G = gridDim.x;
   const long long g0 = share_begin(blockIdx.x, total, G), g1 = share_begin(blockIdx.x + 1, total, G);
   const int n_tiles = (int)(g1 - g0);
   const int tps_u = a.tiles_per_seq;
   if constexpr (RAGGED) {
+    int* staged = reinterpret_cast<int*>(sm + kOffStaged);
     for (int n = threadIdx.x; n < min(n_tiles, kStagedPages); n += kThreads) {
       TileCursor<true> c;
-      c.locate(g0 + n, 0, prefix, a.batch);
+      c.locate(g0 + n, 0, prefix_s, a.batch);
       staged[n] = a.page_table[(long long)c.b * a.max_pages + c.t];
     }
     __syncthreads();
@@ -322,13 +337,14 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     bool ok = true;
     int pc = 0, seg = 0;
     TileCursor<RAGGED> cur, ahead;
-    cur.locate(g0, tps_u, prefix, a.batch);
+    cur.locate(g0, tps_u, prefix_s, a.batch);
     ahead = cur;
     // TMA coordinates (slot, plane) of a tile: its place in the sequence's row range, or its page.
     auto tile_coords = [&](const TileCursor<RAGGED>& c, int n, int& c_slot, int& c_plane) {
       if constexpr (RAGGED) {
         c_slot = 0;
-        c_plane = n < kStagedPages ? staged[n] : __ldg(a.page_table + (long long)c.b * a.max_pages + c.t);
+        c_plane = n < kStagedPages ? lds_i32(staged_s + 4 * n)
+                                   : __ldg(a.page_table + (long long)c.b * a.max_pages + c.t);
       } else {
         c_slot = c.t * kTile;
         c_plane = c.b;
@@ -343,10 +359,10 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       int slot, plane;
       tile_coords(ahead, n_ahead, slot, plane);
       for (int c = 0; c < 2 * RP + 1; ++c) tma_prefetch_l2_3d(&cache_map, c * 64, slot, plane);
-      ahead.next(prefix);
+      ahead.next(prefix_s);
     };
     for (int n = 0; n < kPrefetchAhead; ++n) prefetch_tile(n);
-    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix)) {
+    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix_s)) {
       const int b = cur.b;
       prefetch_tile(n + kPrefetchAhead);
       if (n == 0 || cur.seq_first()) {
@@ -363,6 +379,8 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       const int kb = n % kKrBufs;
       ok = mbar_wait(bar(&misc->empty_kr[kb]), ((n / kKrBufs) & 1) ^ 1, abort_word, a.error_word, 2);
       if (!ok) break;
+      misc->tile_flags[n & 15] = ((n == 0 || cur.seq_first()) ? 1 : 0) |
+                                 ((n + 1 == n_tiles || cur.seq_last()) ? 2 : 0);
       mbar_arrive_expect_tx(bar(&misc->full_kr[kb]), kSubBytes);
       tma_load_3d(kr_u32 + kb * kSubBytes, &cache_map, bar(&misc->full_kr[kb]), a.r, slot, plane);
       for (int c = 0; c < RP && ok; ++c, ++pc) {
@@ -382,24 +400,24 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     const int k = warp - 1;
     bool ok = true;
     int seg = 0;
-    TileCursor<RAGGED> cur;
-    cur.locate(g0, tps_u, prefix, a.batch);
-    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix)) {
+    for (int n = 0; n < n_tiles && ok; ++n) {
       const uint32_t d_tmem = tmem_base + kColS + (n & 1) * (kSParts * 32) + k * 32;
       auto qk = [&](uint32_t a_smem, int chunk, uint32_t accumulate) {
         const uint64_t ad = make_smem_desc(a_smem + k * 32, 16, 1024, kSwizzle128B);
         const uint64_t bd = make_smem_desc(q_u32 + chunk * QCHUNK + k * 32, 16, 1024, kSwizzle128B);
         mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, accumulate);
       };
-      if (n == 0 || cur.seq_first()) {
-        ok = mbar_wait(bar(&misc->q_full), seg & 1, abort_word, a.error_word, 4);
-        if (!ok) break;
-        ++seg;
-      }
       const int kb = n % kKrBufs;
       ok = mbar_wait(bar(&misc->s_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 9) &&
            mbar_wait(bar(&misc->full_kr[kb]), (n / kKrBufs) & 1, abort_word, a.error_word, 10);
       if (!ok) break;
+      const int flags = *reinterpret_cast<volatile int*>(&misc->tile_flags[n & 15]);
+      const bool seg_last = flags & 2;
+      if (flags & 1) {                   // a segment starts: its q~ must have landed
+        ok = mbar_wait(bar(&misc->q_full), seg & 1, abort_word, a.error_word, 4);
+        if (!ok) break;
+        ++seg;
+      }
       tc_fence_after_sync();
       qk(kr_u32 + kb * kSubBytes, 2 * RP, 0u);
       mma_commit(bar(&misc->empty_kr[kb]));
@@ -414,7 +432,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       }
       if (!ok) break;
       mma_commit(bar(&misc->s_full[n & 1]));
-      if (n + 1 == n_tiles || cur.seq_last()) mma_commit(bar(&misc->q_empty));   // segment's last tile
+      if (seg_last) mma_commit(bar(&misc->q_empty));
     }
   } else if (warp > kQkIssuers && warp <= kQkIssuers + kPvIssuers && lane == 0) {
     // ------------------------------------------------------------------ value issuer j
@@ -422,13 +440,11 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     // are published, and hands the pairs it read back to the producer.
     const int j = warp - 1 - kQkIssuers;
     bool ok = true;
-    TileCursor<RAGGED> cur;
-    cur.locate(g0, tps_u, prefix, a.batch);
-    for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix)) {
+    for (int n = 0; n < n_tiles && ok; ++n) {
       ok = mbar_wait(bar(&misc->p_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 12);
       if (!ok) break;
       tc_fence_after_sync();
-      const bool seg_first = n == 0 || cur.seq_first();
+      const bool seg_first = *reinterpret_cast<volatile int*>(&misc->pv_first[n & 1]) != 0;
       for (int mb = j; mb < RP; mb += kPvIssuers) {
         const int buf = (n * RP + mb) % kPairs;
         const uint32_t src = pairs_u32 + buf * kPairBytes;
@@ -487,20 +503,45 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       return is_max ? fmaxf(fmaxf(r0[0], r0[32]), fmaxf(r0[64], r0[96])) : r0[0] + r0[32] + r0[64] + r0[96];
     };
     float l_acc[NHH];
-    TileCursor<RAGGED> cur;
-    cur.locate(g0, tps_u, prefix, a.batch);
-    int n_slots = a.n_slots;
-    for (int n = 0; n < n_tiles; ++n, cur.next(prefix)) {
-      const int b = cur.b, t = cur.t;
-      const bool seg_first = n == 0 || cur.seq_first();
-      const bool seg_last = n + 1 == n_tiles || cur.seq_last();
+    TileCursor<false> cur;             // lock-step batches: every thread walks the list
+    if constexpr (!RAGGED) cur.locate(g0, tps_u, prefix_s, a.batch);
+    int seg_left = 0;                  // ragged batches: tiles left in the running segment
+    for (int n = 0; n < n_tiles; ++n) {
+      bool seg_first, seg_last;
+      if constexpr (RAGGED) {
+        seg_first = seg_left == 0;
+        if (seg_first && sidx == 0) {
+          // One thread finds the segment that starts at tile n and describes it in shared memory.
+          TileCursor<true> c;
+          c.locate(g0 + n, 0, prefix_s, a.batch);
+          const int tiles = min(n_tiles - n, c.tps - c.t);
+          const int seq_slots = ceil_div(__ldg(a.seq_tokens + c.b), a.stride);
+          misc->seg_b = c.b;
+          misc->seg_tiles = tiles;
+          misc->seg_tps = c.tps;
+          misc->seg_start = (int)c.start(prefix_s);
+          misc->seg_tail_rows = c.t + tiles == c.tps ? seq_slots - (c.tps - 1) * kTile : kTile;
+        }
+      } else {
+        seg_first = n == 0 || cur.seq_first();
+      }
       if (seg_first) {
-        if constexpr (RAGGED) n_slots = ceil_div(__ldg(a.seq_tokens + b), a.stride);
         // New sequence: empty references (shared by all threads) and denominators.
         if (sidx < 32) misc->m_used[sidx] = -INFINITY;
 #pragma unroll
         for (int i = 0; i < NHH; ++i) l_acc[i] = 0.f;
         group_sync();
+        if constexpr (RAGGED) seg_left = misc->seg_tiles;
+      }
+      int rows_valid;                  // slots of this tile that exist
+      if constexpr (RAGGED) {
+        seg_last = seg_left == 1;
+        --seg_left;
+        rows_valid = seg_last ? misc->seg_tail_rows : kTile;
+      } else {
+        seg_last = n + 1 == n_tiles || cur.seq_last();
+        rows_valid = a.n_slots - cur.t * kTile;
+        cur.next(prefix_s);
       }
       float s[NHH];
 #pragma unroll
@@ -520,7 +561,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
                  (__uint_as_float(sp[2][i]) + __uint_as_float(sp[3][i]));
         tc_fence_before_sync();
       }
-      const bool valid = ok && active && t * kTile + row < n_slots;
+      const bool valid = ok && active && row < rows_valid;
       float m_ref[NHH];
       bool exceed = false;
 #pragma unroll
@@ -559,6 +600,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       probabilities();
       // The probability buffer is free once the value MMAs of tile n - 2 have completed.
       if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 7);
+      if (ok && sidx == 0) misc->pv_first[n & 1] = seg_first;
       if (ok) store_probabilities();
       if (ok) ok = mbar_wait(bar(&misc->flag_bar[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 14);
       if (ok && misc->exceed_flag[n & 1]) {
@@ -621,6 +663,17 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (!seg_last) continue;
       // ---------------------------------------------------------------- end of a segment
       // Partial of sequence b: wait for the last value MMAs, read O^T from TMEM.
+      int b, seq_tiles;
+      long long seq_start;
+      if constexpr (RAGGED) {          // read before the first rendezvous below
+        b = misc->seg_b;
+        seq_tiles = misc->seg_tps;
+        seq_start = misc->seg_start;
+      } else {                         // cur has already moved on to the next tile
+        b = cur.t == 0 ? cur.b - 1 : cur.b;
+        seq_tiles = tps_u;
+        seq_start = (long long)b * tps_u;
+      }
       const long long part = blockIdx.x + b;      // unique per (CTA, sequence), increasing
       if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 8);
       ok = __all_sync(0xffffffffu, ok);
@@ -646,9 +699,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         __threadfence();
       }
       // Ticket: the CTA that delivers the sequence's last partial combines them.
-      const long long seq_start = cur.start(prefix);
-      const long long c_first = share_owner(seq_start, total, G);
-      const int n_parts = (int)(share_owner(seq_start + cur.tps - 1, total, G) - c_first) + 1;
+      const long long list_len = RAGGED ? misc->total_tiles : total;
+      const long long c_first = share_owner(seq_start, list_len, G);
+      const int n_parts = (int)(share_owner(seq_start + seq_tiles - 1, list_len, G) - c_first) + 1;
       group_sync();
       if (sidx == 0) {
         int last = 0;
