@@ -170,6 +170,35 @@ int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y
 #define MTLA_STATIC_SCRATCH_BYTES (4u << 20)
 int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, void* stream);
 
+/* ---- comparison layers: multi-head, grouped-query and multi-query attention (Section 3) ----
+ *
+ * The attentions the paper compares against, at the same boundary, so that its speed and
+ * cache-size ratios can be restated on this hardware: q = x W_Q (n_h heads), k = x W_K and
+ * v = x W_V (n_kv_heads heads, each shared by n_h / n_kv_heads query heads: n_kv_heads = n_h is
+ * MHA, 1 is MQA), standard rotary embedding of q and k at the token's position (Appendix:
+ * "Standard RoPE is used in MHA"), softmax(q K^T / sqrt(d_h)) V over the cached keys and values
+ * including the token's own, y = concat(heads) W_O.  bf16 only.  The cache keeps 2 n_kv_heads d_h
+ * elements per token, laid out [sequence][kv head][token][value | key].
+ * A handle made by mtla_baseline_create is used with mtla_decode_step, mtla_cache_bytes,
+ * mtla_cache_export / mtla_cache_import (layout [B][n_kv_heads][tokens][2 d_h]), mtla_position,
+ * mtla_reset, mtla_check, mtla_profile_* and mtla_destroy; every other call returns
+ * MTLA_ERR_STATE.  Weights: device, row-major [in][out], bf16. */
+typedef struct {
+  int32_t d_model, n_heads, n_kv_heads;
+  int32_t head_dim;           /* 64 or 128 */
+  int32_t max_batch, max_tokens;
+  float rope_theta;           /* 0 selects 10000 */
+} mtla_baseline_config;
+typedef struct {
+  const void* w_q;            /* [d][n_h*d_h] */
+  const void* w_k;            /* [d][n_kv_heads*d_h] */
+  const void* w_v;            /* [d][n_kv_heads*d_h] */
+  const void* w_o;            /* [n_h*d_h][d] */
+} mtla_baseline_weights;
+size_t mtla_baseline_arena_bytes(const mtla_baseline_config* cfg);
+int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_weights* weights,
+                         void* arena, size_t arena_bytes, void* stream, mtla_handle** out);
+
 /* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3);
  * with per-sequence token counts, the sum over the sequences. */
 size_t mtla_cache_bytes(const mtla_handle* h);

@@ -31,7 +31,8 @@ EXPORTED_SYMBOLS = (
     "mtla_arena_bytes_paged", "mtla_create_paged", "mtla_prefill_seqs", "mtla_beam_reorder",
     "mtla_seq_positions", "mtla_pages_in_use", "mtla_cache_export_seq", "mtla_cache_import_seqs",
     "mtla_page_pool_create", "mtla_page_pool_destroy", "mtla_page_pool_prepare",
-    "mtla_page_pool_reorder", "mtla_page_pool_row", "mtla_page_pool_in_use", "mtla_page_pool_ref")
+    "mtla_page_pool_reorder", "mtla_page_pool_row", "mtla_page_pool_in_use", "mtla_page_pool_ref",
+    "mtla_baseline_arena_bytes", "mtla_baseline_create")
 
 PAGE_SLOTS = 64
 
@@ -56,6 +57,16 @@ class mtla_paging(ctypes.Structure):
     _fields_ = [("page_slots", ctypes.c_int32), ("n_pages", ctypes.c_int32)]
 
 
+class mtla_baseline_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "d_model", "n_heads", "n_kv_heads", "head_dim", "max_batch", "max_tokens")] + [
+        ("rope_theta", ctypes.c_float)]
+
+
+class mtla_baseline_weights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w_q", "w_k", "w_v", "w_o")]
+
+
 class mtla_weights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES]
 
@@ -74,6 +85,10 @@ def load_library() -> ctypes.CDLL:
     cfg_p, w_p = ctypes.POINTER(mtla_config), ctypes.POINTER(mtla_weights)
     pg_p, i32_p = ctypes.POINTER(mtla_paging), ctypes.POINTER(ctypes.c_int32)
     sigs = {
+        "mtla_baseline_arena_bytes": (sz, [ctypes.POINTER(mtla_baseline_config)]),
+        "mtla_baseline_create": (ctypes.c_int, [ctypes.POINTER(mtla_baseline_config),
+                                                ctypes.POINTER(mtla_baseline_weights), vp, sz, vp,
+                                                ctypes.POINTER(vp)]),
         "mtla_arena_bytes_paged": (sz, [cfg_p, pg_p]),
         "mtla_create_paged": (ctypes.c_int, [cfg_p, pg_p, w_p, vp, sz, vp, ctypes.POINTER(vp)]),
         "mtla_prefill_seqs": (ctypes.c_int, [vp, i32, vp, i32, i32, vp, vp]),
@@ -142,6 +157,7 @@ class Handle:
     arena: torch.Tensor
     dtype: torch.dtype
     device: torch.device
+    kv_heads: int = 0      # comparison layers: key/value heads per sequence (0: an MTLA layer)
 
 
 def make_config(*, d_model, n_heads, head_dim, latent_rank, rope_dim, stride, hyper_dim=0,
@@ -214,6 +230,42 @@ def mtla_prefill(h: Handle, x: torch.Tensor, y: torch.Tensor | None = None, want
                                        y.data_ptr() if y is not None else None,
                                        _stream_ptr(stream)), "mtla_prefill")
     return y
+
+
+def mtla_baseline_create(*, d_model, n_heads, n_kv_heads, head_dim, max_batch, max_tokens,
+                         weights: dict, rope_theta=0.0, device="cuda:0", stream=None) -> Handle:
+    """A comparison layer (MHA: n_kv_heads = n_heads, MQA: 1, GQA in between), bf16.
+    weights: w_q, w_k, w_v, w_o as CUDA bf16 tensors, row-major [in][out]."""
+    lib = load_library()
+    cfg = mtla_baseline_config(d_model, n_heads, n_kv_heads, head_dim, max_batch, max_tokens,
+                               rope_theta)
+    nbytes = lib.mtla_baseline_arena_bytes(ctypes.byref(cfg))
+    if nbytes == 0:
+        raise MTLAError(-2, "mtla_baseline_arena_bytes")
+    device = torch.device(device)
+    with torch.cuda.device(device):
+        arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+        base = (arena.data_ptr() + 1023) // 1024 * 1024
+        w = mtla_baseline_weights()
+        keep = []
+        for name in ("w_q", "w_k", "w_v", "w_o"):
+            t = weights[name]
+            if t.dtype != torch.bfloat16 or not t.is_cuda:
+                raise TypeError(f"weight {name}: expected a bfloat16 CUDA tensor")
+            t = t.contiguous()
+            keep.append(t)
+            setattr(w, name, t.data_ptr())
+        out = ctypes.c_void_p()
+        _check(lib.mtla_baseline_create(ctypes.byref(cfg), ctypes.byref(w), base, nbytes,
+                                        _stream_ptr(stream), ctypes.byref(out)), "mtla_baseline_create")
+        torch.cuda.current_stream().synchronize()
+    # The generic calls read d_model / widths from an mtla_config: give them one that describes
+    # the cache rows of this layer (2 d_h elements per row, n_kv_heads planes per sequence).
+    shim = make_config(d_model=d_model, n_heads=n_heads, head_dim=head_dim, latent_rank=2 * head_dim,
+                       rope_dim=0, stride=1, max_batch=max_batch, max_tokens=max_tokens, dtype="bf16")
+    h = Handle(out.value, shim, arena, torch.bfloat16, device)
+    h.kv_heads = n_kv_heads
+    return h
 
 
 def mtla_create_paged(cfg: mtla_config, weights: dict, n_pages: int = 0, device="cuda:0",
@@ -387,7 +439,8 @@ def mtla_cache_export(h: Handle, stream=None) -> torch.Tensor:
     """The cache in use as a tensor [B][slots][r + d_R]."""
     _, slots, batch = mtla_position(h)
     width = h.config.latent_rank + h.config.rope_dim
-    out = torch.empty(batch, slots, width, dtype=h.dtype, device=h.device)
+    shape = (batch, slots, width) if h.kv_heads == 0 else (batch, h.kv_heads, slots, width)
+    out = torch.empty(*shape, dtype=h.dtype, device=h.device)
     if out.numel():
         _check(load_library().mtla_cache_export(h.ptr, out.data_ptr(),
                                                 out.numel() * out.element_size(),
@@ -399,7 +452,8 @@ def mtla_cache_import(h: Handle, cache: torch.Tensor, tokens: int, stream=None) 
     """cache [B][ceil(tokens/s)][r + d_R] on the device."""
     b = cache.shape[0]
     slots = -(-tokens // h.config.stride)
-    _expect(cache, h, (b, slots, h.config.latent_rank + h.config.rope_dim), "cache")
+    width = h.config.latent_rank + h.config.rope_dim
+    _expect(cache, h, (b, slots, width) if h.kv_heads == 0 else (b, h.kv_heads, slots, width), "cache")
     _check(load_library().mtla_cache_import(h.ptr, cache.data_ptr(), b, tokens,
                                             _stream_ptr(stream)), "mtla_cache_import")
 

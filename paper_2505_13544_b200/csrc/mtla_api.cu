@@ -20,6 +20,7 @@
 #include "prefill_kernels.cuh"
 #include "setup_kernels.cuh"
 #include "paging_kernels.cuh"
+#include "baseline_kernels.cuh"
 #include "page_pool.h"
 
 using namespace mtla;
@@ -183,6 +184,10 @@ struct mtla_handle {
   PagePool* pool;
   std::vector<int> seq_tokens;
   bool tokens_stale;
+  // Comparison layers (mtla_baseline_create): multi-head / grouped-query / multi-query attention
+  // over a key-value cache; g key/value heads per sequence, each a plane of the cache.
+  bool is_baseline;
+  int bl_groups;
   int64_t launches;
   bool attn_smem_ready, pf_smem_ready;
   // Tensor-core decode attention (bf16, r a multiple of 128): TMA view of the cache.
@@ -219,6 +224,7 @@ struct mtla_handle {
     return v;
   }
   int seq_len(int b) const { return pool ? seq_tokens[b] : tokens; }
+  int planes_per_seq() const { return is_baseline ? bl_groups : 1; }
 };
 
 namespace {
@@ -287,8 +293,9 @@ int make_cache_map(mtla_handle* h) {
   if (!fn) return MTLA_ERR_CUDA;
   const Dims& dm = h->dm;
   // Paged: the planes are the pool's 64-slot pages instead of the sequences' row ranges.
+  // Comparison layers: one plane per (sequence, key/value head).
   const cuuint64_t plane_rows = h->paged() ? kPageSlots : dm.max_slots;
-  const cuuint64_t planes = h->paged() ? dm.n_pages : h->cfg.max_batch;
+  const cuuint64_t planes = h->paged() ? dm.n_pages : (cuuint64_t)h->cfg.max_batch * h->planes_per_seq();
   const cuuint64_t dims[3] = {(cuuint64_t)dm.W, plane_rows, planes};
   const cuuint64_t strides[2] = {(cuuint64_t)dm.W * 2, plane_rows * dm.W * 2};
   const cuuint32_t box[3] = {64, (cuuint32_t)tc::kTile, 1};
@@ -298,7 +305,8 @@ int make_cache_map(mtla_handle* h) {
       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (rc != CUDA_SUCCESS) return MTLA_ERR_CUDA;
-  const cuuint64_t qdims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.nh, (cuuint64_t)h->cfg.max_batch};
+  const cuuint64_t qdims[3] = {(cuuint64_t)dm.W, (cuuint64_t)dm.nh,
+                               (cuuint64_t)h->cfg.max_batch * h->planes_per_seq()};
   const cuuint64_t qstrides[2] = {(cuuint64_t)dm.W * 2, (cuuint64_t)dm.nh * dm.W * 2};
   const cuuint32_t qbox[3] = {64, (cuuint32_t)(dm.nh <= 16 ? 16 : 32), 1};
   rc = fn(&h->q_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->at<void>(h->plan.qt), qdims, qstrides,
@@ -1004,8 +1012,16 @@ int dispatch_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t 
   return MTLA_OK;
 }
 
+int baseline_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st);
+
 int run_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
                const AttnScratch* scratch = nullptr) {
+  if (h->is_baseline) {
+    if (scratch) return MTLA_ERR_STATE;
+    MTLA_TRY(baseline_decode(h, x, B, y, st));
+    step_end(h, B);
+    return MTLA_OK;
+  }
   return h->cfg.dtype == MTLA_DTYPE_BF16 ? dispatch_decode<bf16>(h, x, B, y, st, scratch)
                                          : dispatch_decode<float>(h, x, B, y, st, scratch);
 }
@@ -1098,6 +1114,8 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
   h->gemm_attr_mask = 0;
   h->pool = nullptr;
   h->tokens_stale = false;
+  h->is_baseline = false;
+  h->bl_groups = 1;
   if (paging) {
     h->pool = new (std::nothrow) PagePool(dm.n_pages, c.max_batch, dm.max_pages);
     if (!h->pool) {
@@ -1122,12 +1140,212 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
   return MTLA_OK;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Comparison layers (Section 3): MHA / GQA / MQA decode over a key-value cache, bf16, built from
+// the same projection GEMM and the same decode attention kernel (see baseline_kernels.cuh).
+
+bool baseline_dims(const mtla_baseline_config* in, mtla_config* cfg, Dims* dm, int* groups) {
+  if (!in) return false;
+  if (in->d_model <= 0 || in->d_model % 8) return false;
+  if (in->head_dim != 64 && in->head_dim != 128) return false;
+  if (in->n_heads < 1 || in->n_kv_heads < 1 || in->n_heads % in->n_kv_heads) return false;
+  const int per = in->n_heads / in->n_kv_heads;
+  if (per > 32) return false;
+  if (in->max_batch < 1 || in->max_tokens < 1) return false;
+  if ((long long)in->max_batch * in->n_kv_heads * in->max_tokens > (1ll << 40)) return false;
+  memset(cfg, 0, sizeof(*cfg));
+  cfg->d_model = in->d_model; cfg->n_heads = in->n_heads; cfg->head_dim = in->head_dim;
+  cfg->max_batch = in->max_batch; cfg->max_tokens = in->max_tokens; cfg->stride = 1;
+  cfg->dtype = MTLA_DTYPE_BF16;
+  cfg->rope_theta = in->rope_theta == 0.f ? 10000.f : in->rope_theta;
+  memset(dm, 0, sizeof(*dm));
+  dm->d = in->d_model; dm->dh = in->head_dim; dm->s = 1; dm->elem = 2;
+  dm->nh = per;                       // heads the attention kernel sees per (sequence, group)
+  dm->W = 2 * in->head_dim;           // cache row: value, then key
+  dm->r = dm->W; dm->dr = 0;
+  dm->max_slots = in->max_tokens;
+  dm->ntot = (in->n_heads + 2 * in->n_kv_heads) * in->head_dim;
+  dm->max_units = kSmCount + in->max_batch * in->n_kv_heads;
+  *groups = in->n_kv_heads;
+  return true;
+}
+
+void plan_baseline(const mtla_config& c, const Dims& dm, int groups, ArenaPlan* p) {
+  memset(p, 0, sizeof(*p));
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes, 1024);
+    return at;
+  };
+  const size_t B = c.max_batch, hd = (size_t)c.n_heads * dm.dh, planes = B * groups;
+  p->wcat_t = take((size_t)dm.ntot * dm.d * 2);
+  p->w_o_t = take((size_t)dm.d * hd * 2);
+  p->rope_cos = take((size_t)c.max_tokens * (dm.dh / 2) * 4);
+  p->rope_sin = take((size_t)c.max_tokens * (dm.dh / 2) * 4);
+  p->cache = take(planes * dm.max_slots * dm.W * 2);
+  p->err_flag = take(16);
+  p->p1 = take(B * dm.ntot * 4);
+  p->qt = take(planes * dm.nh * dm.W * 2);
+  p->o_part = take((size_t)dm.max_units * dm.nh * dm.W * 4);
+  p->ml_part = take((size_t)dm.max_units * dm.nh * 2 * 4);
+  p->o = take(planes * 2 * dm.nh * dm.W * 2);
+  p->v = take(B * 2 * hd * 2);
+  p->gemm_part = take((size_t)kGemmSlots * gtc::kBM * act_box_rows(c.max_batch) * 4);
+  p->gemm_tickets = take((size_t)kGemmSlots * 4 * sizeof(int));
+  p->attn_tickets = take(planes * sizeof(int));
+  p->total = off;
+}
+
+int baseline_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st) {
+  const Dims& dm = h->dm;
+  const ArenaPlan& p = h->plan;
+  const int g = h->bl_groups, n_heads = dm.nh * g, hd = n_heads * dm.dh, pos = h->tokens;
+  const int bn = act_box_rows(B);
+  const bool prof = h->prof_used + MTLA_DECODE_STAGES + 1 <= (int)h->prof_events.size();
+  if (h->act_bn != bn) {
+    MTLA_TRY(make_map_2d(&h->map_v16, h->at<void>(p.v), h->cfg.max_batch, 2 * hd, 2 * hd, bn));
+    h->act_bn = bn;
+  }
+  MTLA_TRY(prof_mark(h, prof, 0, st));
+  CUtensorMap map_x;
+  MTLA_TRY(make_map_2d(&map_x, x, B, dm.d, dm.d, bn));
+  MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x,
+                          gemm_tc_args(h->at<float>(p.p1), 1, dm.ntot, dm.ntot, B, dm.d, 1.f), bn, 1,
+                          true, st));
+  MTLA_TRY(prof_mark(h, prof, 1, st));
+  KvPostArgs ka;
+  ka.p1 = h->at<float>(p.p1);
+  ka.rope_cos = h->at<float>(p.rope_cos);
+  ka.rope_sin = h->at<float>(p.rope_sin);
+  ka.cache = h->at<bf16>(p.cache);
+  ka.qt = h->at<bf16>(p.qt);
+  ka.n_heads = n_heads; ka.n_groups = g; ka.head_dim = dm.dh; ka.max_tokens = dm.max_slots;
+  ka.tokens = pos;
+  ka.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+  const bool pdl = !(prof && !h->prof_attention_only);
+  MTLA_CUDA(launch_kernel(kv_post_kernel, dim3(B), dim3(256), 0, st, pdl, ka));
+  h->launches++;
+  MTLA_TRY(prof_mark(h, prof, 2, st));
+  MTLA_TRY(prof_mark(h, prof, 3, st));
+  AttnTcArgs ta;
+  memset(&ta, 0, sizeof(ta));
+  ta.o_part = h->at<float>(p.o_part); ta.ml_part = h->at<float>(p.ml_part);
+  ta.o16 = h->at<bf16>(p.o);
+  ta.tickets = h->at<int>(p.attn_tickets);
+  ta.error_word = h->at<int>(p.err_flag);
+  ta.n_heads = dm.nh; ta.r = dm.W; ta.dr = 0; ta.n_slots = pos + 1; ta.batch = B * g;
+  ta.tiles_per_seq = ceil_div(pos + 1, tc::kTile);
+  const long long total = (long long)ta.batch * ta.tiles_per_seq;
+  const int grid = (int)(total < kSmCount ? total : kSmCount);
+  const bool attn_pdl = pdl && !prof;
+  if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, false>(h, ta, grid, st, attn_pdl)));
+  else MTLA_TRY((launch_attn_tc_rp<32, false>(h, ta, grid, st, attn_pdl)));
+  MTLA_TRY(prof_mark(h, prof, 4, st));
+  MTLA_TRY(prof_mark(h, prof, 5, st));
+  MTLA_CUDA(launch_kernel(kv_heads_gather_kernel, dim3(B), dim3(256), 0, st, pdl && !prof,
+                          (const bf16*)h->at<bf16>(p.o), h->at<bf16>(p.v), n_heads, g, dm.dh));
+  h->launches++;
+  MTLA_TRY(prof_mark(h, prof, 6, st));
+  GemmTcArgs ga = gemm_tc_args(y, 1, dm.d, dm.d, B, hd, 1.f);
+  ga.b_lo_col = hd;
+  MTLA_TRY(gemm_tc<bf16>(h, h->map_wot, h->map_v16, ga, bn, 1, true, st, pdl));
+  MTLA_TRY(prof_mark(h, prof, 7, st));
+  if (prof) h->prof_used += MTLA_DECODE_STAGES + 1;
+  return MTLA_OK;
+}
+
+int baseline_create(mtla_handle* h, const mtla_baseline_weights* w, cudaStream_t st) {
+  const Dims& dm = h->dm;
+  const ArenaPlan& p = h->plan;
+  const int g = h->bl_groups, n_heads = dm.nh * g, hd = n_heads * dm.dh, gd = g * dm.dh;
+  bf16* wcat = h->at<bf16>(p.wcat_t);
+  // Fused projection stored [out][in]: rows [ q | k | v ].
+  MTLA_TRY(launch_transpose<bf16>(h, w->w_q, wcat, dm.d, hd, hd, dm.d, st));
+  MTLA_TRY(launch_transpose<bf16>(h, w->w_k, wcat + (size_t)hd * dm.d, dm.d, gd, gd, dm.d, st));
+  MTLA_TRY(launch_transpose<bf16>(h, w->w_v, wcat + (size_t)(hd + gd) * dm.d, dm.d, gd, gd, dm.d, st));
+  MTLA_TRY(launch_transpose<bf16>(h, w->w_o, h->at<bf16>(p.w_o_t), hd, dm.d, dm.d, hd, st));
+  const long long n_rope = (long long)h->cfg.max_tokens * (dm.dh / 2);
+  rope_table_kernel<<<(unsigned)((n_rope + 255) / 256), 256, 0, st>>>(
+      h->at<float>(p.rope_cos), h->at<float>(p.rope_sin), h->cfg.max_tokens, dm.dh / 2,
+      (double)h->cfg.rope_theta);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  const size_t planes = (size_t)h->cfg.max_batch * g;
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.err_flag), 0, 16, st));
+  // Rows beyond the valid range are multiplied by probability 0 and must be finite; the zero
+  // halves of the query rows stay zero for the handle's life.
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.cache), 0, planes * dm.max_slots * dm.W * 2, st));
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.qt), 0, planes * dm.nh * dm.W * 2, st));
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.gemm_tickets), 0, (size_t)kGemmSlots * 4 * sizeof(int), st));
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(p.attn_tickets), 0, planes * sizeof(int), st));
+  MTLA_TRY(make_cache_map(h));
+  MTLA_TRY(make_map_2d(&h->map_wcat, h->at<void>(p.wcat_t), dm.ntot, dm.d, dm.d, gtc::kBM));
+  MTLA_TRY(make_map_2d(&h->map_wot, h->at<void>(p.w_o_t), dm.d, hd, hd, gtc::kBM));
+  return MTLA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mtla_baseline_arena_bytes(const mtla_baseline_config* cfg) {
+  mtla_config c;
+  Dims dm;
+  int groups;
+  if (!baseline_dims(cfg, &c, &dm, &groups)) return 0;
+  ArenaPlan p;
+  plan_baseline(c, dm, groups, &p);
+  return p.total;
+}
+
+int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_weights* w, void* arena,
+                         size_t arena_bytes, void* stream, mtla_handle** out) {
+  if (!cfg || !w || !arena || !out) return MTLA_ERR_INVALID_ARG;
+  mtla_config c;
+  Dims dm;
+  int groups;
+  if (!baseline_dims(cfg, &c, &dm, &groups)) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  for (const void* ptr : {w->w_q, w->w_k, w->w_v, w->w_o})
+    if (!ptr || !aligned16(ptr)) return MTLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(arena) & 1023) return MTLA_ERR_INVALID_ARG;
+  ArenaPlan p;
+  plan_baseline(c, dm, groups, &p);
+  if (arena_bytes < p.total) return MTLA_ERR_ARENA_TOO_SMALL;
+  mtla_handle* h = new (std::nothrow) mtla_handle();
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
+  h->tokens = 0; h->batch = 0; h->launches = 0;
+  h->attn_smem_ready = false; h->pf_smem_ready = false;
+  h->prof_used = 0;
+  h->prof_attention_only = false;
+  h->act_bn = 0;
+  h->gemm_attr_mask = 0;
+  h->pool = nullptr;
+  h->tokens_stale = false;
+  h->is_baseline = true;
+  h->bl_groups = groups;
+  h->use_tc = true;
+  const int rc = baseline_create(h, w, static_cast<cudaStream_t>(stream));
+  if (rc != MTLA_OK) {
+    delete h;
+    return rc;
+  }
+  *out = h;
+  return MTLA_OK;
+}
+
+}  // extern "C"
+
+namespace {
 }  // namespace
 
 extern "C" {
 
 int mtla_prefill(mtla_handle* h, const void* x, int32_t B, int32_t T, void* y, void* stream) {
   if (!h || !x || B <= 0 || T <= 0) return MTLA_ERR_INVALID_ARG;
+  if (h->is_baseline) return MTLA_ERR_STATE;
   if (!aligned16(x) || (y && !aligned16(y))) return MTLA_ERR_INVALID_ARG;
   if (h->tokens != 0 || h->batch != 0) return MTLA_ERR_STATE;
   if (B > h->cfg.max_batch || T > h->cfg.max_prefill_tokens || T > h->cfg.max_tokens)
@@ -1159,6 +1377,7 @@ int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y
                           void* stream) {
   const int chk = check_step_args(h, x_host, B, y_host);
   if (chk != MTLA_OK) return chk;
+  if (h->is_baseline) return MTLA_ERR_STATE;    // no staging rows in a comparison layer's arena
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t bytes = (size_t)B * h->dm.d * h->dm.elem;
   void* xs = h->at<void>(h->plan.x_stage);
@@ -1173,6 +1392,7 @@ int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, v
   const int chk = check_step_args(h, x, B, y);
   if (chk != MTLA_OK) return chk;
   if (!aligned16(x) || !aligned16(y)) return MTLA_ERR_INVALID_ARG;
+  if (h->is_baseline) return MTLA_ERR_STATE;
   // Same sizing as the arena's split workspace, for this call's batch.
   const Dims& dm = h->dm;
   const size_t units = (size_t)(h->use_tc ? kSmCount : kTargetCtas) + (size_t)B;
@@ -1204,7 +1424,7 @@ size_t mtla_cache_bytes(const mtla_handle* h) {
   if (!h) return 0;
   size_t slots = 0;
   for (int b = 0; b < h->batch; ++b) slots += ceil_div(h->seq_len(b), h->dm.s);
-  return slots * h->dm.W * h->dm.elem;
+  return slots * h->planes_per_seq() * h->dm.W * h->dm.elem;
 }
 
 int mtla_destroy(mtla_handle* h) {
@@ -1254,8 +1474,9 @@ int mtla_cache_export(mtla_handle* h, void* dst, size_t bytes, void* stream) {
   }
   const size_t row = (size_t)ceil_div(h->tokens, h->dm.s) * h->dm.W * h->dm.elem;
   const size_t pitch = (size_t)h->dm.max_slots * h->dm.W * h->dm.elem;
-  MTLA_CUDA(cudaMemcpy2DAsync(dst, row, h->at<char>(h->plan.cache), pitch, row, h->batch,
-                              cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+  MTLA_CUDA(cudaMemcpy2DAsync(dst, row, h->at<char>(h->plan.cache), pitch, row,
+                              (size_t)h->batch * h->planes_per_seq(), cudaMemcpyDeviceToDevice,
+                              static_cast<cudaStream_t>(stream)));
   return MTLA_OK;
 }
 
@@ -1284,8 +1505,8 @@ int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens
     for (int b = 0; b < B; ++b) h->seq_tokens[b] = tokens;
     h->tokens_stale = true;
   } else {
-    MTLA_CUDA(cudaMemcpy2DAsync(h->at<char>(h->plan.cache), pitch, src, row, row, B,
-                                cudaMemcpyDeviceToDevice, st));
+    MTLA_CUDA(cudaMemcpy2DAsync(h->at<char>(h->plan.cache), pitch, src, row, row,
+                                (size_t)B * h->planes_per_seq(), cudaMemcpyDeviceToDevice, st));
   }
   if (tokens % h->dm.s != 0) {
     if (h->cfg.dtype == MTLA_DTYPE_BF16)
@@ -1386,6 +1607,7 @@ int64_t mtla_pages_in_use(const mtla_handle* h) { return h && h->paged() ? h->po
 
 int mtla_cache_export_seq(mtla_handle* h, int32_t seq, void* dst, size_t bytes, void* stream) {
   if (!h || !dst || !aligned16(dst) || seq < 0 || seq >= h->batch) return MTLA_ERR_INVALID_ARG;
+  if (h->is_baseline) return MTLA_ERR_STATE;
   const int n_slots = ceil_div(h->seq_len(seq), h->dm.s);
   if (bytes < (size_t)n_slots * h->dm.W * h->dm.elem) return MTLA_ERR_CAPACITY;
   if (n_slots == 0) return MTLA_OK;

@@ -134,6 +134,25 @@ def make_weights(w: Workload) -> dict[str, torch.Tensor]:
     }
 
 
+def make_baseline_weights(w: Workload, n_kv_heads: int) -> dict[str, torch.Tensor]:
+    """Parameters of a comparison layer (MHA / GQA / MQA) of w's width: N(0,1)/sqrt(fan_in),
+    row-major [in][out], rounded to w.dtype."""
+    d, nh, dh = w.d_model, w.n_heads, w.head_dim
+
+    def mat(name, fan_in, fan_out):
+        return stored(normal(w.seed, f"baseline/{n_kv_heads}/{name}", (fan_in, fan_out),
+                             scale=fan_in ** -0.5), w.dtype)
+
+    return {"w_q": mat("w_q", d, nh * dh), "w_k": mat("w_k", d, n_kv_heads * dh),
+            "w_v": mat("w_v", d, n_kv_heads * dh), "w_o": mat("w_o", nh * dh, d)}
+
+
+def kv_cache_plane(w: Workload, seq: int, kv_head: int, tokens: int) -> torch.Tensor:
+    """A stand-in key-value cache [tokens][2 d_h] (value then key, unit normal) for one
+    (sequence, key/value head) of a comparison layer, where the context is too long to decode."""
+    return stored(normal(w.seed, f"kv/{seq}/{kv_head}", (tokens, 2 * w.head_dim)), w.dtype)
+
+
 def prompt(w: Workload, batch: int | None = None, tokens: int | None = None) -> torch.Tensor:
     """Prompt activations [B][T][d] ~ N(0,1), generated one sequence at a time."""
     b = w.batch if batch is None else batch
