@@ -394,6 +394,90 @@ def fill_context(M, h, w: synth.Workload, device) -> dict:
     return info
 
 
+def run_compare(args, device, local: int) -> None:
+    """The paper's comparison (Tables 1 and 5 are ratios against MHA, MQA, GQA and MLA), restated
+    on this GPU: the same layer width, batch and context for every method, decode steps timed
+    the same way; cache bytes per token from the library's own accounting."""
+    from paper_2505_13544_b200 import binding as M
+    base = synth.WORKLOADS[args.workload]
+    ctx = args.context_tokens or (8192 if base.name == "large" else 4096)
+    K, W = args.steps, max(args.warmup, 3)
+    dt = torch.bfloat16
+    rows = []
+
+    def time_steps(h, xs, y):
+        for i in range(W):
+            M.mtla_decode_step(h, xs[i % 8], y)
+        torch.cuda.synchronize(device)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        M.mtla_profile_begin_attention(h, K)
+        ev0.record()
+        for i in range(K):
+            M.mtla_decode_step(h, xs[i % 8], y)
+        ev1.record()
+        torch.cuda.synchronize(device)
+        attn_ms, n = M.mtla_profile_end(h)
+        M.mtla_check(h)
+        assert torch.isfinite(y.float()).all()
+        return ev0.elapsed_time(ev1) / K, attn_ms / max(n, 1)
+
+    xs = [synth.decode_input(base, i).to(device) for i in range(8)]
+    y = torch.empty(base.batch, base.d_model, dtype=dt, device=device)
+    kv_variants = [("MHA", base.n_heads)] + [("GQA", g) for g in sorted({max(base.n_heads // 4, 2), 2},
+                                                                          reverse=True)] + [("MQA", 1)]
+    for name, n_kv in kv_variants:
+        weights = synth.make_baseline_weights(base, n_kv)
+        h = M.mtla_baseline_create(d_model=base.d_model, n_heads=base.n_heads, n_kv_heads=n_kv,
+                                   head_dim=base.head_dim, max_batch=base.batch,
+                                   max_tokens=ctx + 2 * (K + W), device=device,
+                                   weights={k: v.to(device) for k, v in weights.items()})
+        # Four distinct seeded sequences, tiled over the batch (the values do not affect timing).
+        distinct = [torch.stack([synth.kv_cache_plane(base, b, g, ctx) for g in range(n_kv)]).to(device)
+                    for b in range(min(4, base.batch))]
+        cache = torch.empty(base.batch, n_kv, ctx, 2 * base.head_dim, dtype=dt, device=device)
+        for b in range(base.batch):
+            cache[b].copy_(distinct[b % len(distinct)])
+        M.mtla_cache_import(h, cache, ctx)
+        torch.cuda.synchronize(device)
+        del cache, distinct
+        torch.cuda.empty_cache()
+        per_token = M.mtla_cache_bytes(h) / (base.batch * ctx)
+        ms, attn = time_steps(h, xs, y)
+        rows.append({"method": name, "kv_heads": n_kv, "ms_per_step": ms, "attention_us": attn * 1e3,
+                     "tokens_per_s": base.batch / (ms * 1e-3), "cache_bytes_per_token": per_token})
+        M.mtla_destroy(h)
+        del h
+        torch.cuda.empty_cache()
+    for s in (1, 2, 3, 4):
+        w = base.scaled(stride=s, prefill_tokens=0, context_tokens=ctx, name=f"{base.name}[s={s}]")
+        Mx, h = build_layer(w, extra_steps=2 * (K + W), device=device)
+        fill_context(Mx, h, w, device)
+        per_token = M.mtla_cache_bytes(h) / (w.batch * ctx)
+        ms, attn = time_steps(h, xs, y)
+        rows.append({"method": "MLA" if s == 1 else "MTLA", "stride": s, "ms_per_step": ms,
+                     "attention_us": attn * 1e3, "tokens_per_s": w.batch / (ms * 1e-3),
+                     "cache_bytes_per_token": per_token})
+        M.mtla_destroy(h)
+        del h
+        torch.cuda.empty_cache()
+    mha = rows[0]
+    peaks = measured_peaks()
+    for r in rows:
+        r["speedup_vs_mha"] = mha["ms_per_step"] / r["ms_per_step"]
+        r["cache_reduction_vs_mha"] = mha["cache_bytes_per_token"] / r["cache_bytes_per_token"]
+        # The attention kernel's roofline: the cache read once per step against the copy peak.
+        r["attention_gbs"] = r["cache_bytes_per_token"] * base.batch * ctx / (r["attention_us"] * 1e-6) / 1e9
+        r["attention_frac_of_hbm_peak"] = r["attention_gbs"] / peaks["hbm_gbs"]
+    print(json.dumps({
+        "metric": METRIC, "unit": UNIT, "comparison": rows, "n_gpus": 1, "steps": K, "warmup": W,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"compare[{base.name}]", "batch": base.batch, "d_model": base.d_model,
+                   "n_heads": base.n_heads, "head_dim": base.head_dim, "latent_rank": base.latent_rank,
+                   "rope_dim": base.rope_dim, "context_tokens": ctx,
+                   "note": "same width, batch and context for every method; decode steps with inputs "
+                           "resident; attention_us from two events around the attention kernel"}}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -401,6 +485,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--workload", default="large",
                     choices=sorted(synth.WORKLOADS) + sorted(synth.BEAM_WORKLOADS))
+    ap.add_argument("--compare", action="store_true",
+                    help="time MHA / GQA / MQA / MLA / MTLA at the workload's width, batch and one context")
     ap.add_argument("--paged", action="store_true",
                     help="keep the cache in 64-slot pages (mtla_create_paged) instead of contiguous rows")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -432,6 +518,11 @@ def main() -> None:
             dist.barrier(device_ids=[local])
         torch.cuda.synchronize(device)
 
+    if args.compare:
+        if world > 1 or args.workload in synth.BEAM_WORKLOADS:
+            raise SystemExit("--compare runs a decode workload on one GPU")
+        run_compare(args, device, local)
+        return
     if args.workload in synth.BEAM_WORKLOADS:
         if world > 1:
             raise SystemExit("the beam workloads run on one GPU")
