@@ -86,3 +86,35 @@ def test_error_strings():
     with pytest.raises(M.MTLAError) as e:
         M._check(-4, "probe")
     assert "capacity" in str(e.value)
+
+
+def test_paged_arena_holds_the_pool_and_rejects_bad_paging():
+    lib = M.load_library()
+    cfg = good_config(max_tokens=1000)          # 500 slots -> 8 pages per sequence
+    page = 64 * (256 + 32) * 2
+    full = M.mtla_arena_bytes_paged(cfg)
+    small = M.mtla_arena_bytes_paged(cfg, n_pages=5)
+    assert full - small >= (4 * 8 - 5) * page - 4096
+    assert M.mtla_arena_bytes_paged(cfg, n_pages=4 * 8 + 1) == 0      # more pages than could ever be used
+    bad = M.mtla_paging(32, 0)                                        # pages are 64 slots
+    assert lib.mtla_arena_bytes_paged(ctypes.byref(cfg), ctypes.byref(bad)) == 0
+    assert lib.mtla_arena_bytes_paged(ctypes.byref(cfg), None) == 0
+
+
+def test_baseline_arena_follows_the_cache_formula():
+    """2 g d_h elements per token (Section 3), bf16."""
+    lib = M.load_library()
+
+    def arena(**kw):
+        base = dict(d_model=512, n_heads=8, n_kv_heads=8, head_dim=64, max_batch=2, max_tokens=100,
+                    rope_theta=0.0)
+        base.update(kw)
+        cfg = M.mtla_baseline_config(*[base[k] for k in ("d_model", "n_heads", "n_kv_heads", "head_dim",
+                                                         "max_batch", "max_tokens", "rope_theta")])
+        return lib.mtla_baseline_arena_bytes(ctypes.byref(cfg))
+
+    per_token = 2 * 8 * 64 * 2
+    assert arena(max_tokens=1100) - arena(max_tokens=100) >= 2 * 1000 * per_token
+    assert arena(n_kv_heads=1) < arena(n_kv_heads=8)
+    for bad in (dict(n_kv_heads=3), dict(head_dim=96), dict(n_heads=64, n_kv_heads=1), dict(max_batch=0)):
+        assert arena(**bad) == 0
