@@ -89,7 +89,9 @@ bool normalise(const mtla_config* in, const mtla_paging* pg, mtla_config* out, D
   dm->proj.off_u = -1;
   if (c.dtype == MTLA_DTYPE_BF16 && c.stride > 1) {
     dm->proj.off_u = dm->proj.width;
-    dm->proj.width += 2 * dm->dw;
+    // Rows of the projection output are read 16 bytes at a time by the CUDA-core GEMMs: an odd
+    // d_w would leave every other row misaligned, so the row is padded (zero weight rows).
+    dm->proj.width = (dm->proj.width + 2 * dm->dw + 3) / 4 * 4;
   }
   dm->ntot = dm->proj.width;
   dm->max_slots = ceil_div(c.max_tokens, c.stride);
@@ -508,6 +510,10 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
     MTLA_CUDA(cudaGetLastError());
     MTLA_TRY((gemm<float, T, float>(h, ga, w->w_r, wg, dm.dw, dm.d, dm.r, dm.r, dm.r, dm.d, 1.f, 1,
                                     0, 0, 0, st)));
+    const int pad_rows = dm.ntot - (dm.proj.off_u + 2 * dm.dw);
+    if (pad_rows > 0)
+      MTLA_CUDA(cudaMemsetAsync(h->at<bf16>(p.wcat_t) + (size_t)(dm.ntot - pad_rows) * dm.d, 0,
+                                (size_t)pad_rows * dm.d * sizeof(bf16), st));
     const long long n_wg = (long long)dm.dw * dm.d;
     gate_fold_pack_kernel<<<(unsigned)((n_wg + 255) / 256), 256, 0, st>>>(
         wg, h->at<bf16>(p.wcat_t) + (size_t)dm.proj.off_u * dm.d, dm.dw, dm.d);
@@ -968,11 +974,24 @@ int check_step_args(mtla_handle* h, const void* x, int32_t B, const void* y) {
   }
   if (!h->paged()) return h->tokens + 1 > h->cfg.max_tokens ? MTLA_ERR_CAPACITY : MTLA_OK;
   if (h->use_tc && B > tc::kMaxRaggedBatch) return MTLA_ERR_CAPACITY;
+  // Pages the step will take from the free list: new pages at page boundaries, and copies of
+  // shared newest pages.  Of the w sequences about to write a page that ref sequences hold, the
+  // last one to be served keeps the page if all holders write it: min(w, ref - 1) copies.
   int need = 0;
+  std::vector<int> shared;
   for (int b = 0; b < B; ++b) {
     if (h->seq_tokens[b] + 1 > h->cfg.max_tokens) return MTLA_ERR_CAPACITY;
-    const int slot = h->seq_tokens[b] / h->dm.s;
-    need += h->pool->pages_needed(b, slot + 1, slot);
+    const int slot = h->seq_tokens[b] / h->dm.s, k = slot / kPageSlots;
+    const int have = h->pool->pages_held(b);
+    need += std::max(0, PagePool::pages_for(slot + 1) - have);
+    if (k < have && h->pool->ref(h->pool->row(b)[k]) > 1) shared.push_back(h->pool->row(b)[k]);
+  }
+  std::sort(shared.begin(), shared.end());
+  for (size_t i = 0; i < shared.size();) {
+    size_t j = i;
+    while (j < shared.size() && shared[j] == shared[i]) ++j;
+    need += std::min((int)(j - i), h->pool->ref(shared[i]) - 1);
+    i = j;
   }
   return need > h->pool->pages_free() ? MTLA_ERR_CAPACITY : MTLA_OK;
 }
