@@ -90,3 +90,81 @@ def test_random_layer_and_call_sequence(seed):
             H.assert_cache_close(M.mtla_cache_export_seq(h, b), O.cache_array(states[b]), w.dtype)
     finally:
         M.mtla_destroy(h)
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_long_contexts_on_the_tensor_core_attention(seed):
+    """Imported contexts of up to 6000 tokens (ragged on paged handles), batches up to 24: tile
+    lists whose shares cut sequences at arbitrary places, sequences spread over many CTAs, CTAs
+    holding many short sequences.  Sampled sequences are followed by the oracle."""
+    g = np.random.Generator(np.random.Philox(key=[seed, 0xa77e]))
+    pick = lambda xs: xs[int(g.integers(len(xs)))]
+    batch = int(g.integers(1, 25))
+    w = synth.Workload(
+        name=f"fuzz_ctx{seed}", dtype="bf16", batch=batch, d_model=8 * int(g.integers(8, 33)),
+        n_heads=int(g.integers(1, 33)), head_dim=pick([64, 128]), latent_rank=pick([128, 256, 384, 512]),
+        rope_dim=pick([32, 64]), hyper_dim=int(g.integers(1, 65)), stride=int(g.integers(1, 5)),
+        prefill_tokens=0, context_tokens=0, decode_steps=3, seed=2000 + seed)
+    paged = bool(g.integers(2))
+    longest = int(g.integers(1, 6001))
+    lengths = [int(g.integers(1, longest + 1)) for _ in range(batch)] if paged else [longest] * batch
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    cfg = M.make_config(**H.dims_of(w), max_batch=batch, max_tokens=max(lengths) + w.decode_steps,
+                        max_prefill_tokens=0, dtype="bf16", ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    dev = {k: v.cuda() for k, v in weights.items()}
+    h = M.mtla_create_paged(cfg, dev) if paged else M.mtla_create(cfg, dev)
+    sampled = sorted({0, batch // 2, batch - 1})
+    try:
+        assert M.mtla_attention_variant(h) == "tcgen05"
+        rows = [synth.context_cache_row(w, b, -(-t // w.stride)) for b, t in enumerate(lengths)]
+        if paged:
+            for b, t in enumerate(lengths):
+                M.mtla_cache_import_seqs(h, b, rows[b][None].cuda(), t)
+        else:
+            M.mtla_cache_import(h, torch.stack(rows).cuda(), longest)
+        states = {b: O.state_from_cache(rows[b].double().numpy(), lengths[b], p) for b in sampled}
+        for i in range(w.decode_steps):
+            x = synth.stored(synth.normal(w.seed, f"x/{i}", (batch, w.d_model)), "bf16")
+            y = M.mtla_decode_step(h, x.cuda())
+            want = np.stack([O.decode_step(p, states[b], x[b].double().numpy()) for b in sampled])
+            assert_close_scaled(y[sampled], want, "bf16", f"step {i}")
+        M.mtla_check(h)
+        assert M.mtla_seq_positions(h) == [t + w.decode_steps for t in lengths]
+    finally:
+        M.mtla_destroy(h)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_comparison_layers(seed):
+    """MHA / GQA / MQA layers of random width and grouping with an imported context."""
+    from oracle import gqa_oracle as G
+    g = np.random.Generator(np.random.Philox(key=[seed, 0x69a]))
+    pick = lambda xs: xs[int(g.integers(len(xs)))]
+    n_kv = pick([1, 2, 3, 4, 8])
+    per = pick([1, 2, 4, 5, 8, 32]) if n_kv <= 2 else pick([1, 2, 4])
+    batch, ctx = int(g.integers(1, 9)), int(g.integers(1, 1500))
+    w = synth.Workload(
+        name=f"fuzz_kv{seed}", dtype="bf16", batch=batch, d_model=8 * int(g.integers(8, 49)),
+        n_heads=n_kv * per, head_dim=pick([64, 128]), latent_rank=128, rope_dim=32, hyper_dim=8, stride=1,
+        prefill_tokens=0, context_tokens=0, decode_steps=4, seed=3000 + seed)
+    weights = synth.make_baseline_weights(w, n_kv)
+    p = G.params_from_tensors(
+        dict(d_model=w.d_model, n_heads=w.n_heads, n_groups=n_kv, head_dim=w.head_dim),
+        {k: v.double().numpy() for k, v in weights.items()}, rope_theta=w.rope_theta)
+    h = M.mtla_baseline_create(d_model=w.d_model, n_heads=w.n_heads, n_kv_heads=n_kv, head_dim=w.head_dim,
+                               max_batch=batch, max_tokens=ctx + w.decode_steps,
+                               weights={k: v.cuda() for k, v in weights.items()}, rope_theta=w.rope_theta)
+    try:
+        cache = torch.stack([torch.stack([synth.kv_cache_plane(w, b, k, ctx) for k in range(n_kv)])
+                             for b in range(batch)])
+        M.mtla_cache_import(h, cache.cuda(), ctx)
+        states = [G.state_from_cache(cache[b].double().numpy()) for b in range(batch)]
+        for i in range(w.decode_steps):
+            x = synth.stored(synth.normal(w.seed, f"x/{i}", (batch, w.d_model)), "bf16")
+            y = M.mtla_decode_step(h, x.cuda())
+            want = np.stack([G.decode_step(p, states[b], x[b].double().numpy()) for b in range(batch)])
+            assert_close_scaled(y, want, "bf16", f"step {i}")
+        M.mtla_check(h)
+    finally:
+        M.mtla_destroy(h)
