@@ -79,6 +79,10 @@ struct AttnTcArgs {
   const int* seq_tokens;   // [B] tokens per sequence, this step's included
   const int* page_table;   // [B][max_pages] page of tile t of sequence b
   int max_pages, stride;
+  // 0: the partials are combined by decode_combine_parts_kernel afterwards (lock-step batches
+  // whose sequences are spread over many CTAs), 1: by the last CTA of each sequence.
+  int fused_combine;
+  int attn_grid;           // decode_combine_parts_kernel: grid size of the attention launch
 };
 
 namespace tc {
@@ -107,6 +111,7 @@ constexpr int kSParts = 4;                 // independent partial score accumula
 constexpr int kColS = 0;                   // score buffer b, partial k at column (b * 4 + k) * 32
 constexpr int kColO = 2 * kSParts * 32;    // output blocks at 256 + 32 * block
 constexpr float kRescaleThreshold = 8.f;
+constexpr int kSmCountMax = 256;           // upper bound on the attention grid (one CTA per SM)
 
 constexpr int kOffPairs = 0;
 constexpr int kOffKr = kPairs * kPairBytes;
@@ -703,6 +708,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       const long long c_first = share_owner(seq_start, list_len, G);
       const int n_parts = (int)(share_owner(seq_start + seq_tiles - 1, list_len, G) - c_first) + 1;
       group_sync();
+      if (!a.fused_combine) continue;        // a separate launch combines (uniform over the CTA)
       if (sidx == 0) {
         int last = 0;
         if (ok) {
@@ -716,37 +722,77 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (ok && misc->last_flag) {
         __threadfence();
         const long long part0 = c_first + b;
-        // Per head: global reference, each part's weight 2^(m_p - m) and the denominator.
+        // Per head: global reference, each part's weight 2^(m_p - m) and the denominator.  All
+        // loops over the parts keep kU loads in flight: a sequence spread over many CTAs (a small
+        // batch with a long context) has tens of parts, and one load at a time would make this
+        // the longest phase of the kernel.
+        constexpr int kU = 8;
         if (sidx < a.n_heads) {
+          const float* ml0 = a.ml_part + (part0 * a.n_heads + sidx) * 2;
+          const long long ml_step = 2ll * a.n_heads;
           float m = -INFINITY;
-          for (int pt = 0; pt < n_parts; ++pt)
-            m = fmaxf(m, __ldcg(a.ml_part + ((part0 + pt) * a.n_heads + sidx) * 2));
+          for (int p0 = 0; p0 < n_parts; p0 += kU) {
+            float mv[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) mv[u] = p0 + u < n_parts ? __ldcg(ml0 + (p0 + u) * ml_step) : -INFINITY;
+#pragma unroll
+            for (int u = 0; u < kU; ++u) m = fmaxf(m, mv[u]);
+          }
           float denom = 0.f;
-          for (int pt = 0; pt < n_parts; ++pt) {
-            const float* ml = a.ml_part + ((part0 + pt) * a.n_heads + sidx) * 2;
-            const float wgt = exp2f(__ldcg(ml) - m);
-            denom += wgt * __ldcg(ml + 1);
-            if (pt < 8) misc->comb_w[pt][sidx] = wgt;
+          for (int p0 = 0; p0 < n_parts; p0 += kU) {
+            float mv[kU], lv[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+              const bool in = p0 + u < n_parts;
+              mv[u] = in ? __ldcg(ml0 + (p0 + u) * ml_step) : -INFINITY;
+              lv[u] = in ? __ldcg(ml0 + (p0 + u) * ml_step + 1) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+              if (p0 + u >= n_parts) break;
+              const float wgt = exp2f(mv[u] - m);
+              denom += wgt * lv[u];
+              if (p0 + u < 8) misc->comb_w[p0 + u][sidx] = wgt;
+            }
           }
           misc->fac[sidx] = 1.f / denom;
           misc->comb_m[sidx] = m;
         }
         group_sync();
-        // Thread (cg, hh): latent columns 4*cg .. 4*cg+3 of the heads of parity hh.
-        const int cg = sidx & 127, hh = sidx >> 7;
-        if (ok && 4 * cg < a.r) {
+        // Thread (cg, hh): latent columns 4*cg .. 4*cg+3 of the heads hh, hh + lanes, ...
+        const int col_groups = a.r >> 2, lanes = kSoftmaxThreads / col_groups;
+        const int cg = sidx % col_groups, hh = sidx / col_groups;
+        if (ok && hh < lanes) {
           bf16* o_hi = a.o16 + (long long)b * 2 * a.n_heads * a.r + 4 * cg;
           bf16* o_lo = o_hi + (long long)a.n_heads * a.r;
-          for (int h = hh; h < a.n_heads; h += 2) {
+          const long long o_step = (long long)a.n_heads * a.r, ml_step = 2ll * a.n_heads;
+          for (int h = hh; h < a.n_heads; h += lanes) {
+            const float* o0 = a.o_part + (part0 * a.n_heads + h) * a.r + 4 * cg;
+            const float* ml0 = a.ml_part + (part0 * a.n_heads + h) * 2;
+            const float m = misc->comb_m[h];
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int pt = 0; pt < n_parts; ++pt) {
-              const float wgt = pt < 8 ? misc->comb_w[pt][h]
-                                       : exp2f(__ldcg(a.ml_part + ((part0 + pt) * a.n_heads + h) * 2) -
-                                               misc->comb_m[h]);
-              const float4 v = __ldcg(reinterpret_cast<const float4*>(
-                  a.o_part + ((part0 + pt) * a.n_heads + h) * a.r + 4 * cg));
-              acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
-              acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+            for (int p0 = 0; p0 < n_parts; p0 += kU) {
+              float4 v[kU];
+              float wg[kU];
+#pragma unroll
+              for (int u = 0; u < kU; ++u) {
+                const int pt = p0 + u;
+                if (pt < n_parts) {
+                  v[u] = __ldcg(reinterpret_cast<const float4*>(o0 + pt * o_step));
+                  wg[u] = pt < 8 ? misc->comb_w[pt][h] : __ldcg(ml0 + pt * ml_step);
+                } else {
+                  v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                  wg[u] = -INFINITY;
+                }
+              }
+#pragma unroll
+              for (int u = 0; u < kU; ++u) {
+                const int pt = p0 + u;
+                if (pt >= n_parts) break;
+                const float wgt = pt < 8 ? wg[u] : exp2f(wg[u] - m);
+                acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
+                acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
+              }
             }
             const float inv = misc->fac[h];
             const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
@@ -776,6 +822,70 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// Combine of the attention partials as a launch of its own, grid (n_h, B), 128 threads: used
+// for lock-step batches in which a sequence is spread over many CTAs (a small batch with a long
+// context), where one CTA reading every part of a sequence would be the kernel's longest phase.
+// Same arithmetic, in the same order, as the fused combine.
+__global__ void __launch_bounds__(128) decode_combine_parts_kernel(AttnTcArgs a) {
+  using namespace tc;
+  __shared__ float w_s[kSmCountMax];
+  __shared__ float red_s[33];
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+  const long long tps = a.tiles_per_seq, total = (long long)a.batch * tps, G = a.attn_grid;
+  const long long c_first = share_owner((long long)b * tps, total, G);
+  const int n_parts = (int)(share_owner((long long)(b + 1) * tps - 1, total, G) - c_first) + 1;
+  const long long part0 = c_first + b;
+  const float* ml0 = a.ml_part + (part0 * a.n_heads + h) * 2;
+  const long long ml_step = 2ll * a.n_heads, o_step = (long long)a.n_heads * a.r;
+  // Reference maximum, weights and denominator of head h (n_parts <= grid size <= kSmCountMax).
+  float m = -INFINITY;
+  for (int pt = tid; pt < n_parts; pt += 128) m = fmaxf(m, __ldcg(ml0 + pt * ml_step));
+  m = warp_max(m);
+  if ((tid & 31) == 0) red_s[tid >> 5] = m;
+  __syncthreads();
+  m = fmaxf(fmaxf(red_s[0], red_s[1]), fmaxf(red_s[2], red_s[3]));
+  for (int pt = tid; pt < n_parts; pt += 128) w_s[pt] = exp2f(__ldcg(ml0 + pt * ml_step) - m);
+  __syncthreads();
+  if (tid == 0) {
+    float denom = 0.f;
+    for (int pt = 0; pt < n_parts; ++pt) denom += w_s[pt] * __ldcg(ml0 + pt * ml_step + 1);   // part order
+    red_s[32] = 1.f / denom;
+  }
+  __syncthreads();
+  const float inv = red_s[32];
+  if (4 * tid >= a.r) return;
+  constexpr int kU = 8;
+  const float* o0 = a.o_part + (part0 * a.n_heads + h) * a.r + 4 * tid;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int p0 = 0; p0 < n_parts; p0 += kU) {
+    float4 v[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u)
+      v[u] = p0 + u < n_parts ? __ldcg(reinterpret_cast<const float4*>(o0 + (p0 + u) * o_step))
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      if (p0 + u >= n_parts) break;
+      const float wgt = w_s[p0 + u];
+      acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
+      acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
+    }
+  }
+  const float val[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+  const __nv_bfloat162 h0 = __floats2bfloat162_rn(val[0], val[1]);
+  const __nv_bfloat162 h1 = __floats2bfloat162_rn(val[2], val[3]);
+  const __nv_bfloat162 l0 = __floats2bfloat162_rn(val[0] - __low2float(h0), val[1] - __high2float(h0));
+  const __nv_bfloat162 l1 = __floats2bfloat162_rn(val[2] - __low2float(h1), val[3] - __high2float(h1));
+  bf16* o_hi = a.o16 + ((long long)b * 2 * a.n_heads + h) * a.r + 4 * tid;
+  bf16* o_lo = o_hi + (long long)a.n_heads * a.r;
+  *reinterpret_cast<uint2*>(o_hi) =
+      make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+  *reinterpret_cast<uint2*>(o_lo) =
+      make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
 }
 
 }  // namespace mtla

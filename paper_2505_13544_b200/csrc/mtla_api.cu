@@ -30,6 +30,7 @@ namespace {
 constexpr int kSmCount = 148;        // B200
 constexpr int kTargetCtas = 296;     // two CTAs per SM on a 148-SM part
 constexpr int kMinSlotsPerSplit = 64;
+constexpr int kFusedCombineMaxParts = 8;   // more parts per sequence: the combine gets its own launch
 constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill projections
 constexpr int kGemmSlots = 2 * kSmCount;   // CTAs a split-K GEMM may spread one product over
 
@@ -726,6 +727,11 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     const long long total = h->paged() ? ragged_tiles : (long long)B * ta.tiles_per_seq;
     const int grid = (int)(total < kSmCount ? total : kSmCount);
     aa.n_split = 0;
+    // A lock-step batch whose sequences are each spread over many CTAs hands the combine to a
+    // launch of its own, one CTA per (head, sequence), instead of one CTA per sequence.
+    const bool split_combine = !h->paged() && grid / B + 2 > kFusedCombineMaxParts;
+    ta.fused_combine = !split_combine;
+    ta.attn_grid = grid;
     const bool attn_pdl = pdl && !prof;     // the attention kernel is bracketed by events when timed
     if (h->paged()) {
       if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, true>(h, ta, grid, st, attn_pdl)));
@@ -734,6 +740,11 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
       if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, false>(h, ta, grid, st, attn_pdl)));
       else MTLA_TRY((launch_attn_tc_rp<32, false>(h, ta, grid, st, attn_pdl)));
     }
+    MTLA_TRY(prof_mark(h, prof, 4, st));
+    if (split_combine) {
+      MTLA_CUDA(launch_kernel(decode_combine_parts_kernel, dim3(dm.nh, B), dim3(128), 0, st, pdl && !prof, ta));
+      h->launches++;
+    }
   } else {
     int want = ceil_div(kTargetCtas, B);
     int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
@@ -741,8 +752,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
     aa.n_split = ceil_div(n_slots, aa.slots_per_split);
     MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st)));
+    MTLA_TRY(prof_mark(h, prof, 4, st));
   }
-  MTLA_TRY(prof_mark(h, prof, 4, st));
 
   CombineArgs ca;
   ca.o_part = aa.o_part; ca.ml_part = aa.ml_part; ca.o = h->at<void>(p.o);
@@ -1259,8 +1270,15 @@ int baseline_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t 
   const long long total = (long long)ta.batch * ta.tiles_per_seq;
   const int grid = (int)(total < kSmCount ? total : kSmCount);
   const bool attn_pdl = pdl && !prof;
+  const bool split_combine = grid / ta.batch + 2 > kFusedCombineMaxParts;
+  ta.fused_combine = !split_combine;
+  ta.attn_grid = grid;
   if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, false>(h, ta, grid, st, attn_pdl)));
   else MTLA_TRY((launch_attn_tc_rp<32, false>(h, ta, grid, st, attn_pdl)));
+  if (split_combine) {
+    MTLA_CUDA(launch_kernel(decode_combine_parts_kernel, dim3(dm.nh, ta.batch), dim3(128), 0, st, attn_pdl, ta));
+    h->launches++;
+  }
   MTLA_TRY(prof_mark(h, prof, 4, st));
   MTLA_TRY(prof_mark(h, prof, 5, st));
   MTLA_CUDA(launch_kernel(kv_heads_gather_kernel, dim3(B), dim3(256), 0, st, pdl && !prof,
