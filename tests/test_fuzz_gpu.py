@@ -168,3 +168,56 @@ def test_random_comparison_layers(seed):
         M.mtla_check(h)
     finally:
         M.mtla_destroy(h)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_large_batches(seed):
+    """Batches of 100-400 sequences (more sequences than CTAs, several activation tiles in the
+    projections) with short ragged contexts; the step is taken through the device, the static
+    scratch and the host entry points in turn."""
+    g = np.random.Generator(np.random.Philox(key=[seed, 0xb16]))
+    pick = lambda xs: xs[int(g.integers(len(xs)))]
+    batch = int(g.integers(100, 401))
+    w = synth.Workload(
+        name=f"fuzz_big{seed}", dtype="bf16", batch=batch, d_model=8 * int(g.integers(8, 25)),
+        n_heads=int(g.integers(1, 17)), head_dim=64, latent_rank=pick([128, 256]), rope_dim=pick([32, 64]),
+        hyper_dim=int(g.integers(1, 33)), stride=int(g.integers(1, 4)),
+        prefill_tokens=0, context_tokens=0, decode_steps=3, seed=4000 + seed)
+    paged = bool(g.integers(2))
+    longest = int(g.integers(1, 201))
+    lengths = [int(g.integers(1, longest + 1)) for _ in range(batch)] if paged else [longest] * batch
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    cfg = M.make_config(**H.dims_of(w), max_batch=batch, max_tokens=max(lengths) + w.decode_steps,
+                        max_prefill_tokens=0, dtype="bf16", ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    dev = {k: v.cuda() for k, v in weights.items()}
+    h = M.mtla_create_paged(cfg, dev) if paged else M.mtla_create(cfg, dev)
+    sampled = sorted({0, 1, batch // 3, batch // 2, batch - 2, batch - 1})
+    try:
+        rows = [synth.context_cache_row(w, b, -(-t // w.stride)) for b, t in enumerate(lengths)]
+        if paged:
+            for b, t in enumerate(lengths):
+                M.mtla_cache_import_seqs(h, b, rows[b][None].cuda(), t)
+        else:
+            M.mtla_cache_import(h, torch.stack(rows).cuda(), longest)
+        states = {b: O.state_from_cache(rows[b].double().numpy(), lengths[b], p) for b in sampled}
+        for i in range(w.decode_steps):
+            x = synth.stored(synth.normal(w.seed, f"x/{i}", (batch, w.d_model)), "bf16")
+            if i == 0:
+                y = M.mtla_decode_step(h, x.cuda())
+            elif i == 1:
+                try:
+                    y = M.mtla_decode_step_static(h, x.cuda())
+                except M.MTLAError as err:            # the workspace of a large batch may not fit
+                    assert err.status == -9
+                    y = M.mtla_decode_step(h, x.cuda())
+            else:
+                yh = torch.empty(batch, w.d_model, dtype=torch.bfloat16).pin_memory()
+                M.mtla_decode_step_host(h, x.pin_memory(), yh)
+                torch.cuda.synchronize()
+                y = yh
+            want = np.stack([O.decode_step(p, states[b], x[b].double().numpy()) for b in sampled])
+            assert_close_scaled(y[sampled], want, "bf16", f"step {i}")
+        M.mtla_check(h)
+    finally:
+        M.mtla_destroy(h)
