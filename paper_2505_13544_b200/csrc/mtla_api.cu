@@ -403,6 +403,11 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   int n_split = 1;
   // The partials are summed by the last CTA of a tile alone: at most four splits keep that short.
   if (allow_split && tiles < slots) n_split = max(1, min(min(kb_total / 4, (int)(slots / tiles)), 4));
+  // Short reductions with few activation rows (the paper's layer: K = 512, B <= 64): one CTA per
+  // tile with the whole K range in flight at once beats splitting it, which costs a trip of the
+  // partials through global memory on top of two load round trips.
+  const bool shallow = allow_split && kb_total <= 8 && bn <= 64;
+  if (shallow) n_split = 1;
   g.kb_per_split = ceil_div(kb_total, n_split);
   g.n_split = ceil_div(kb_total, g.kb_per_split);
   g.partial = h->at<float>(h->plan.gemm_part);
@@ -416,6 +421,21 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
               g.c_sn * osz % 16 == 0 && g.c_sz * osz % 16 == 0 && g.c_lo_off * osz % 8 == 0;
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
+  if (shallow && (sizeof(OutT) == 4 || hilo)) {
+    if constexpr (sizeof(OutT) == 4) {
+      switch (bn) {
+        case 16: return launch_gemm_tc_inst<16, 8, OutT, false>(h, 14, ma, mb, g, grid, st, dependent);
+        case 32: return launch_gemm_tc_inst<32, 8, OutT, false>(h, 15, ma, mb, g, grid, st, dependent);
+        default: return launch_gemm_tc_inst<64, 8, OutT, false>(h, 16, ma, mb, g, grid, st, dependent);
+      }
+    } else {
+      switch (bn) {
+        case 16: return launch_gemm_tc_inst<16, 8, OutT, true>(h, 17, ma, mb, g, grid, st, dependent);
+        case 32: return launch_gemm_tc_inst<32, 8, OutT, true>(h, 18, ma, mb, g, grid, st, dependent);
+        default: return launch_gemm_tc_inst<64, 6, OutT, true>(h, 19, ma, mb, g, grid, st, dependent);
+      }
+    }
+  }
   if constexpr (sizeof(OutT) == 2) {
     if (hilo) {
       switch (bn) {
