@@ -45,17 +45,23 @@ def measured_peaks() -> dict:
             "source": "fallback"}
 
 
+def code_hash(texts) -> str:
+    """sha256 of source texts with comments and blank space removed."""
+    out = ""
+    for text in texts:
+        for line in text.splitlines():
+            code = line.split("//")[0].strip()
+            if code:
+                out += " ".join(code.split()) + "\n"
+    return hashlib.sha256(out.encode()).hexdigest()
+
+
 def kernel_code_hash() -> str:
     """Hash of the decode-attention kernel's code (comments and blank space removed), to tell
     whether the committed ncu counters still describe the kernel that is being timed."""
     csrc = os.path.join(ROOT, "paper_2505_13544_b200", "csrc")
-    text = ""
-    for name in ("decode_attn_tc.cuh", "sm100_ptx.cuh"):
-        for line in open(os.path.join(csrc, name)):
-            code = line.split("//")[0].strip()
-            if code:
-                text += " ".join(code.split()) + "\n"
-    return hashlib.sha256(text.encode()).hexdigest()
+    return code_hash(open(os.path.join(csrc, name)).read()
+                     for name in ("decode_attn_tc.cuh", "sm100_ptx.cuh"))
 
 
 def algorithmic_work(w: synth.Workload, n_slots: float) -> dict:

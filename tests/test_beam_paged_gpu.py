@@ -147,3 +147,42 @@ def test_paging_calls_are_refused_without_paging():
         assert M.mtla_pages_in_use(h) == -1
     finally:
         M.mtla_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_prefill_of_several_sequences_behind_existing_ones(dtype):
+    """mtla_prefill_seqs with B > 1 and seq0 > 0, and a cache import in between."""
+    base = synth.WORKLOADS["tiny"] if dtype == "fp32" else synth.WORKLOADS["paper"]
+    w = base.scaled(stride=3, seed=77)
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    h = paged_handle(w, weights, 6, 400, 150)
+    try:
+        states = []
+
+        def prefill(seq0, n, t_len):
+            x = synth.stored(synth.normal(w.seed, f"pp/{seq0}", (n, t_len, w.d_model)), w.dtype)
+            y = M.mtla_prefill_seqs(h, seq0, x.cuda())
+            for b in range(n):
+                want, st = O.decode_sequence(p, x[b].double().numpy())
+                H.assert_close(y[b], want, w.dtype, f"prefill of sequence {seq0 + b}")
+                states.append(st)
+
+        prefill(0, 1, 100)
+        prefill(1, 3, 70)                     # three sequences behind the first
+        row = synth.context_cache_row(w, 4, 41)          # 122 tokens: the last slot is open
+        M.mtla_cache_import_seqs(h, 4, row[None].cuda(), 122)
+        states.append(O.state_from_cache(row.double().numpy(), 122, p))
+        prefill(5, 1, 150)
+        assert M.mtla_seq_positions(h) == [100, 70, 70, 70, 122, 150]
+        for i in range(8):
+            x = synth.stored(synth.normal(w.seed, f"px/{i}", (6, w.d_model)), w.dtype)
+            y = M.mtla_decode_step(h, x.cuda())
+            want = np.stack([O.decode_step(p, states[b], x[b].double().numpy()) for b in range(6)])
+            H.assert_close(y, want, w.dtype, f"decode step {i}")
+        M.mtla_check(h)
+        with pytest.raises(M.MTLAError) as err:       # sequence 2 is not empty
+            M.mtla_prefill_seqs(h, 2, synth.prompt(w, batch=1, tokens=8).cuda())
+        assert err.value.status == -7
+    finally:
+        M.mtla_destroy(h)
