@@ -82,6 +82,7 @@ class ClockSampler:
 
     def __init__(self, device_index: int):
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.mem_samples, self.power_samples = [], []
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -107,6 +108,8 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_SM))
+                self.mem_samples.append(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_MEM))
+                self.power_samples.append(n.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
                 try:
                     mask = n.nvmlDeviceGetCurrentClocksEventReasons(self._h)
                 except Exception:
@@ -132,7 +135,10 @@ class ClockSampler:
     def summary(self) -> dict:
         return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
                 "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
-                "reasons": sorted(self.reasons)}
+                "reasons": sorted(self.reasons),
+                "mem_mhz": float(np.median(self.mem_samples)) if self.mem_samples else None,
+                "power_w": float(np.median(self.power_samples)) if self.power_samples else None,
+                "power_w_max": float(max(self.power_samples)) if self.power_samples else None}
 
 
 def dims_of(w: synth.Workload) -> dict:
