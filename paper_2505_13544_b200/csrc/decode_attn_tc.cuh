@@ -16,7 +16,8 @@
 // Heads sit in the MMA's N dimension (16 or 32), so no padding of heads up to M is paid for.
 // Accumulators live in TMEM: two score buffers and r/128 output blocks.  With M = 64 the score
 // of slot i sits in TMEM lane 32*(i/16) + i%16, i.e. in the first 16 lanes of each warp's
-// quarter, so lanes 0-15 of each softmax warp own one slot each.
+// quarter; a softmax warp reads them with the two-half load shape (16x32bx2), so that its two
+// half-warps own the same 16 slots and different heads and no lane idles.
 //
 // A score buffer is four partial accumulators: k-step ks (16 columns) of every 64-column chunk
 // goes to partial ks, each partial has its own issuing thread (see below), and the softmax
@@ -42,9 +43,8 @@
 // small-N MMAs execute, so issue is spread over eight single-thread issuers in eight warps:
 // four for the scores (issuer k owns partial accumulator k) and four for the values (issuer j
 // owns output block j and returns its pair to the ring as soon as its four MMAs are in).
-// The softmax is instruction- and latency-bound too, so it runs on eight warps: with M = 64
-// only lanes 0-15 of a warp's TMEM quarter hold scores, and two warps per quarter split the
-// heads between them.  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
+// The softmax is instruction- and latency-bound too, so it runs on eight warps: two warps per
+// TMEM quarter split the heads between them, and each warp's halves split them again.  Warp roles: warp 0 = TMA producer, warps 1-4 = score issuers,
 // warps 5-8 = value issuers, warps 9-11 idle, warps 12-19 = softmax and epilogue.  The first
 // three warpgroups give most of their registers to the other two (setmaxnreg).
 //
@@ -157,23 +157,6 @@ struct Misc {
   int pv_first[2];
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc region too small");
-
-// Butterfly "transposed" reductions: every lane contributes 32 values; afterwards lane i
-// holds the reduction over all lanes of value i (31 shuffles instead of 160).
-template <typename Op>
-__device__ __forceinline__ float transposed_reduce(float (&v)[32], int lane, Op op) {
-#pragma unroll
-  for (int off = 16, n = 32; off >= 1; off >>= 1, n >>= 1) {
-    const bool upper = (lane & off) != 0;
-#pragma unroll
-    for (int i = 0; i < n / 2; ++i) {
-      const float keep = upper ? v[i + n / 2] : v[i];
-      const float send = upper ? v[i] : v[i + n / 2];
-      v[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, off));
-    }
-  }
-  return v[0];
-}
 
 // Share of the tile list owned by CTA c of G: [c * total / G, (c + 1) * total / G).
 __host__ __device__ inline long long share_begin(long long c, long long total, long long G) {
@@ -467,15 +450,17 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   } else {
     // ------------------------------------------------------------------ softmax / epilogue warps
     // Two groups of four warps; group g owns heads [g * NHH, (g + 1) * NHH) of every slot, i.e.
-    // TMEM columns g * NHH .. of each score partial and of each output block.
+    // TMEM columns g * NHH .. of each score partial and of each output block.  The scores of a
+    // tile sit in the first 16 lanes of each TMEM quarter (M = 64); the two halves of a warp
+    // read the same 16 slots and split the group's heads again (NQ each), so all lanes work.
     reg_alloc<kRegsSoftmax>();
-    constexpr int NHH = NHP / 2;
+    constexpr int NHH = NHP / 2, NQ = NHH / 2;
     const int sw = warp - kFirstSoftmaxWarp;                // 0..7
     const int g = sw >> 2, q = warp & 3;                    // head group; TMEM lane quarter
     const int HO = g * NHH;
+    const int HQ = HO + (lane >> 4) * NQ;                   // first head of this thread's scores
     const int sidx = sw * 32 + lane;                        // index among the 256
-    const bool active = lane < 16;                          // lanes that own a slot (M = 64 layout)
-    const int row = q * 16 + lane;                          // slot within the tile (active lanes)
+    const int row = q * 16 + (lane & 15);                   // slot within the tile
     const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16) + HO;
     bool ok = true;
     auto ld_cols = [&](uint32_t addr, uint32_t (&v)[16]) {
@@ -491,15 +476,19 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (ok) ok = mbar_wait(bar(&misc->group_sync), sync_phase & 1, abort_word, a.error_word, 13);
       ++sync_phase;
     };
-    // Per-warp reduction of one value per owned head over the warp's 32 lanes, left in
-    // misc->red[sw][i] for head HO + i.
-    auto reduce_heads = [&](const float (&v)[NHH], float fill, bool is_max) {
-      float red[32];
+    // Per-warp reduction of one value per owned head over the 16 slots of the warp (each half
+    // of the warp holds NQ heads), left in misc->red[sw][i] for head HO + i.
+    auto reduce_heads = [&](const float (&v)[NQ], bool is_max) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) red[i] = i < NHH ? v[i < NHH ? i : 0] : fill;
-      misc->red[sw][lane] = is_max
-          ? transposed_reduce(red, lane, [](float x, float y) { return fmaxf(x, y); })
-          : transposed_reduce(red, lane, [](float x, float y) { return x + y; });
+      for (int i = 0; i < NQ; ++i) {
+        float x = v[i];
+#pragma unroll
+        for (int o = 8; o >= 1; o >>= 1) {
+          const float y = __shfl_xor_sync(0xffffffffu, x, o);
+          x = is_max ? fmaxf(x, y) : x + y;
+        }
+        if ((lane & 15) == 0) misc->red[sw][(lane >> 4) * NQ + i] = x;
+      }
     };
     // Head h's value combined over the four warps of the group that owns it.
     auto reduced = [&](int h, bool is_max) {
@@ -507,7 +496,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       const float* r0 = &misc->red[gg * 4][i];
       return is_max ? fmaxf(fmaxf(r0[0], r0[32]), fmaxf(r0[64], r0[96])) : r0[0] + r0[32] + r0[64] + r0[96];
     };
-    float l_acc[NHH];
+    float l_acc[NQ];
     TileCursor<false> cur;             // lock-step batches: every thread walks the list
     if constexpr (!RAGGED) cur.locate(g0, tps_u, prefix_s, a.batch);
     int seg_left = 0;                  // ragged batches: tiles left in the running segment
@@ -534,7 +523,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         // New sequence: empty references (shared by all threads) and denominators.
         if (sidx < 32) misc->m_used[sidx] = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < NHH; ++i) l_acc[i] = 0.f;
+        for (int i = 0; i < NQ; ++i) l_acc[i] = 0.f;
         group_sync();
         if constexpr (RAGGED) seg_left = misc->seg_tiles;
       }
@@ -548,30 +537,33 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         rows_valid = a.n_slots - cur.t * kTile;
         cur.next(prefix_s);
       }
-      float s[NHH];
+      float s[NQ];
 #pragma unroll
-      for (int i = 0; i < NHH; ++i) s[i] = 0.f;
+      for (int i = 0; i < NQ; ++i) s[i] = 0.f;
       if (ok) ok = mbar_wait(bar(&misc->s_full[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 5);
       ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are whole-warp operations
       if (ok) {
         tc_fence_after_sync();
         const uint32_t s_addr = lane_base + kColS + (n & 1) * (kSParts * 32);
-        uint32_t sp[kSParts][16];
+        uint32_t sp[kSParts][8];
 #pragma unroll
-        for (int k = 0; k < kSParts; ++k) ld_cols(s_addr + k * 32, sp[k]);
+        for (int k = 0; k < kSParts; ++k) {
+          if (NQ == 8) tmem_ld_16x2_x8<NQ>(s_addr + k * 32, sp[k]);
+          else tmem_ld_16x2_x4<NQ>(s_addr + k * 32, sp[k]);
+        }
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < NHH; ++i)               // the score is the sum of the partials
+        for (int i = 0; i < NQ; ++i)                // the score is the sum of the partials
           s[i] = (__uint_as_float(sp[0][i]) + __uint_as_float(sp[1][i])) +
                  (__uint_as_float(sp[2][i]) + __uint_as_float(sp[3][i]));
         tc_fence_before_sync();
       }
-      const bool valid = ok && active && row < rows_valid;
-      float m_ref[NHH];
+      const bool valid = ok && row < rows_valid;
+      float m_ref[NQ];
       bool exceed = false;
 #pragma unroll
-      for (int i = 0; i < NHH; ++i) {
-        m_ref[i] = misc->m_used[HO + i];
+      for (int i = 0; i < NQ; ++i) {
+        m_ref[i] = misc->m_used[HQ + i];
         s[i] = valid ? s[i] : -INFINITY;
         exceed |= s[i] > m_ref[i] + kRescaleThreshold;
       }
@@ -581,10 +573,10 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       mbar_arrive(bar(&misc->flag_bar[n & 1]));
       if (ok) mbar_arrive(bar(&misc->s_empty[n & 1]));
 
-      uint32_t pb[NHH / 2];
+      uint32_t pb[NQ / 2];
       auto probabilities = [&]() {
 #pragma unroll
-        for (int i = 0; i < NHH; i += 2) {
+        for (int i = 0; i < NQ; i += 2) {
           const __nv_bfloat162 pk = __floats2bfloat162_rn(ex2_approx(s[i] - m_ref[i]),
                                                           ex2_approx(s[i + 1] - m_ref[i + 1]));
           pb[i / 2] = *reinterpret_cast<const uint32_t*>(&pk);
@@ -593,11 +585,10 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       // P^T as the K-major, un-swizzled B operand of the value MMA: element (head h, slot k)
       // at (h/8)*PSBO + (k/8)*128 + (h%8)*16 + (k%8)*2.
       auto store_probabilities = [&]() {
-        if (!active) return;
         uint8_t* prow = sm + kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
 #pragma unroll
-        for (int i = 0; i < NHH; ++i) {
-          const int h = HO + i;
+        for (int i = 0; i < NQ; ++i) {
+          const int h = HQ + i;
           const uint16_t bits = (i & 1) ? (uint16_t)(pb[i / 2] >> 16) : (uint16_t)(pb[i / 2] & 0xffffu);
           *reinterpret_cast<uint16_t*>(prow + (h >> 3) * PSBO + (h & 7) * 16) = bits;
         }
@@ -612,7 +603,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         // ---- rare: some head's scores rose more than 2^8 above its reference (always at
         // a sequence's first tile).  Everybody takes this branch: the flag is read after all
         // arrivals.  New references, rescaled denominators and accumulators, new P.
-        reduce_heads(s, -INFINITY, true);
+        reduce_heads(s, true);
         group_sync();
         if (sidx == 0) misc->exceed_flag[n & 1] = 0;
         if (sidx < NHP) {
@@ -624,9 +615,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         }
         group_sync();
 #pragma unroll
-        for (int i = 0; i < NHH; ++i) {
-          m_ref[i] = misc->m_used[HO + i];
-          l_acc[i] *= misc->fac[HO + i];
+        for (int i = 0; i < NQ; ++i) {
+          m_ref[i] = misc->m_used[HQ + i];
+          l_acc[i] *= misc->fac[HQ + i];
         }
         if (!seg_first) {
           // O holds contributions scaled to the old references: wait for the previous tile's
@@ -654,7 +645,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         group_sync();                         // fac / red may be rewritten by the next rare tile
       }
 #pragma unroll
-      for (int i = 0; i < NHH; i += 2) {
+      for (int i = 0; i < NQ; i += 2) {
         const __nv_bfloat162 pk = *reinterpret_cast<const __nv_bfloat162*>(&pb[i / 2]);
         l_acc[i] += __low2float(pk);
         l_acc[i + 1] += __high2float(pk);
@@ -695,7 +686,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         }
         tc_fence_before_sync();
       }
-      reduce_heads(l_acc, 0.f, false);
+      reduce_heads(l_acc, false);
       __threadfence();
       group_sync();
       if (ok && sidx < a.n_heads) {

@@ -249,6 +249,26 @@ __device__ __forceinline__ void tmem_st_x8(uint32_t taddr, const uint32_t (&v)[1
         "r"(taddr)
       : "memory");
 }
+// Warp-wide load of 16 TMEM lanes in two halves: thread t < 16 reads lane base + t, columns
+// c .. c + N - 1; thread t >= 16 reads lane base + t - 16, columns c + HALF .. c + HALF + N - 1
+// (HALF is an immediate).  With an M = 64 accumulator, whose rows sit in the first 16 lanes of
+// each quarter, this keeps all 32 threads of a warp busy.
+template <int HALF>
+__device__ __forceinline__ void tmem_ld_16x2_x8(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x32bx2.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8], %9;"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+        "=r"(v[7])
+      : "r"(taddr), "n"(HALF)
+      : "memory");
+}
+template <int HALF>
+__device__ __forceinline__ void tmem_ld_16x2_x4(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x32bx2.x4.b32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+               : "r"(taddr), "n"(HALF)
+               : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
