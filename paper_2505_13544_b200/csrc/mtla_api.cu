@@ -17,6 +17,7 @@
 #include "gemm_fma.cuh"
 #include "gemm_tc.cuh"
 #include "prefill_attn_tc.cuh"
+#include "prefill_attn_tc2.cuh"
 #include "prefill_kernels.cuh"
 #include "setup_kernels.cuh"
 #include "paging_kernels.cuh"
@@ -872,7 +873,9 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
     gkv.c_lo_off = 2 * hd;
     MTLA_TRY(gemm_tc<bf16>(h, h->map_wkvt, map_c, gkv, kPrefillBn, 1, false, st));
     // Attention on the tensor cores; the closed slots are a strided view of the token rows.
-    const int DQ = dm.dh + dm.dr, kt = pft::key_tile(dm.dh);
+    // d_h = 64: two query tiles per CTA over 64-slot key tiles (prefill_attn_tc2.cuh).
+    const bool two_tiles = dm.dh == 64;
+    const int DQ = dm.dh + dm.dr, kt = two_tiles ? pft2::KT : pft::key_tile(dm.dh);
     const int n_slots_closed = T_len / dm.s;
     const bf16* kv = h->at<bf16>(p.pf_kv);
     const bf16* kr = h->at<bf16>(p.pf_kr);
@@ -895,11 +898,12 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
     ta.error_word = h->at<int>(p.err_flag);
     ta.n_heads = dm.nh; ta.dr = dm.dr; ta.stride = dm.s; ta.T = T_len;
     dim3 grid(ceil_div(T_len, pft::kQTile), dm.nh, B);
-    if (dm.dh == 64) {
+    if (two_tiles) {
       if (!h->pf_smem_ready)
-        MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_tc_kernel<64>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, pft::smem_bytes(64)));
-      prefill_attn_tc_kernel<64><<<grid, pft::kThreads, pft::smem_bytes(64), st>>>(
+        MTLA_CUDA(cudaFuncSetAttribute(prefill_attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       pft2::kSmemBytes));
+      grid.x = ceil_div(T_len, pft2::kQTiles * pft2::kQTile);
+      prefill_attn_tc2_kernel<<<grid, pft2::kThreads, pft2::kSmemBytes, st>>>(
           q_map, kv_closed, kv_self, kr_closed, kr_self, ta);
     } else {
       if (!h->pf_smem_ready)
