@@ -15,6 +15,7 @@ from __future__ import annotations
 import argparse
 import hashlib
 import json
+import math
 import os
 import sys
 import threading
@@ -490,6 +491,157 @@ def run_compare(args, device, local: int) -> None:
                            "resident; attention_us from two events around the attention kernel"}}))
 
 
+def prefill_flop(w: synth.Workload) -> dict:
+    """FLOP the prefill must execute: un-absorbed attention over the pairs the stride-aware
+    mask admits (row m sees ceil(m/s) columns), the fused input projection, the key / value
+    up-projection of the running states and the output projection."""
+    B, T, s = w.batch, w.prefill_tokens, w.stride
+    d, nh, dh, r, dr = w.d_model, w.n_heads, w.head_dim, w.latent_rank, w.rope_dim
+    m = np.arange(1, T + 1, dtype=np.int64)
+    pairs = B * nh * int(((m + s - 1) // s).sum())
+    parts = {"attention": pairs * (2 * (dh + dr) + 2 * dh),
+             "input_proj": 2 * B * T * d * (nh * dh + nh * dr + r + dr),
+             "kv_up_proj": 2 * B * T * r * 2 * nh * dh,
+             "output_proj": 2 * B * T * nh * dh * d}
+    parts["total"] = sum(parts.values())
+    return parts
+
+
+def fill_prompt(w: synth.Workload, device, distinct: int = 4) -> torch.Tensor:
+    """Prompt activations [B][T][d]: `distinct` seeded sequences tiled over the batch (the values
+    do not affect the timing; the parity tests use one seeded prompt per sequence)."""
+    x = torch.empty(w.batch, w.prefill_tokens, w.d_model, dtype=synth.torch_dtype(w.dtype), device=device)
+    rows = [synth.stored(synth.normal(w.seed, f"prompt/{b}", (w.prefill_tokens, w.d_model)), w.dtype).to(device)
+            for b in range(min(distinct, w.batch))]
+    for b in range(w.batch):
+        x[b].copy_(rows[b % len(rows)])
+    return x
+
+
+def time_prefill(M, h, w: synth.Workload, x: torch.Tensor, device, runs: int = 3) -> dict:
+    """One warm-up prefill, then `runs` timed ones (each from an empty cache); the median."""
+    y = torch.empty_like(x)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    launches = 0
+    for i in range(runs + 1):
+        M.mtla_reset(h)
+        torch.cuda.synchronize(device)
+        l0 = M.mtla_launch_count(h)
+        ev0.record()
+        M.mtla_prefill(h, x, y)
+        ev1.record()
+        torch.cuda.synchronize(device)
+        launches = M.mtla_launch_count(h) - l0
+        times.append(ev0.elapsed_time(ev1))
+    M.mtla_check(h)
+    assert torch.isfinite(y[:, -1].float()).all()
+    ms = float(np.median(times[1:]))
+    peaks = measured_peaks()
+    flop = prefill_flop(w)
+    tensor_ms = flop["total"] / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+    return {"workload": w.name, "tokens_per_s": w.batch * w.prefill_tokens / (ms * 1e-3), "ms": ms,
+            "ms_min": float(min(times[1:])), "first_run_ms": times[0], "timed_runs": runs,
+            "batch": w.batch, "tokens": w.prefill_tokens, "algorithmic_tflop": flop["total"] / 1e12,
+            "achieved_tflops": flop["total"] / (ms * 1e-3) / 1e12,
+            "roofline": {"bound": "tensor", "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "peak_source": f"sustained bf16, of {peaks['source']}",
+                         "roofline_ms": tensor_ms, "frac": tensor_ms / ms},
+            "gpu_launches": int(launches)}
+
+
+def time_decode(M, h, w: synth.Workload, device, steps: int, warmup: int) -> dict:
+    """Decode steps with inputs resident, from the handle's current context."""
+    dt = synth.torch_dtype(w.dtype)
+    xs = [synth.decode_input(w, i).to(device) for i in range(8)]
+    y = torch.empty(w.batch, w.d_model, dtype=dt, device=device)
+    for i in range(warmup):
+        M.mtla_decode_step(h, xs[i % 8], y)
+    torch.cuda.synchronize(device)
+    slots0, l0 = M.mtla_position(h)[1], M.mtla_launch_count(h)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(steps):
+        M.mtla_decode_step(h, xs[i % 8], y)
+    ev1.record()
+    torch.cuda.synchronize(device)
+    ms = ev0.elapsed_time(ev1) / steps
+    slots1 = M.mtla_position(h)[1]
+    M.mtla_check(h)
+    assert torch.isfinite(y.float()).all()
+    peaks = measured_peaks()
+    work = algorithmic_work(w, 0.5 * (slots0 + 1 + slots1))
+    hbm_s = (work["weight_bytes"] + work["cache_bytes"]) / (peaks["hbm_gbs"] * 1e9)
+    tensor_s = (work["attn_flop"] + work["proj_flop"]) / (peaks["bf16_tflops_sustained"] * 1e12)
+    return {"workload": w.name, "batch": w.batch, "stride": w.stride, "context_slots": [slots0, slots1],
+            "decode_tokens_per_s": w.batch / (ms * 1e-3), "us_per_step": ms * 1e3,
+            "roofline_us": max(hbm_s, tensor_s) * 1e6,
+            "step_roofline_frac": max(hbm_s, tensor_s) / (ms * 1e-3),
+            "launches_per_step": (M.mtla_launch_count(h) - l0) / steps, "steps": steps,
+            "attention_variant": M.mtla_attention_variant(h)}
+
+
+def run_other_configs(device, steps: int = 64, warmup: int = 8):
+    """The other benchmark configurations, each for a fraction of a second: the parallel prefill
+    of the long-context workload against the tensor roofline, and decode steps of every
+    configuration at its full context."""
+    prefill, configs = None, []
+    for name in ("tiny", "paper", "sweep_s1", "sweep_s2", "sweep_s3", "sweep_s4", "longctx"):
+        w = synth.WORKLOADS[name]
+        M, h = build_layer(w, extra_steps=steps + warmup + 8, device=device)
+        x = fill_prompt(w, device)
+        pf = time_prefill(M, h, w, x, device, runs=3 if name == "longctx" else 1)
+        del x
+        torch.cuda.empty_cache()
+        if name == "longctx":
+            prefill = pf
+        row = time_decode(M, h, w, device, steps, warmup)
+        row["prefill_ms"] = pf["ms"]
+        row["prefill_tokens_per_s"] = pf["tokens_per_s"]
+        row["prefill_tensor_roofline_frac"] = pf["roofline"]["frac"] if w.dtype == "bf16" else None
+        configs.append(row)
+        M.mtla_destroy(h)
+        del h
+        torch.cuda.empty_cache()
+    return prefill, configs
+
+
+def run_sustained(M, h, w: synth.Workload, xs, y, local: int, device, seconds: float, step_ms: float,
+                  max_steps: int):
+    """The same decode loop for at least `seconds`, long enough for the board to settle under its
+    power limit; clocks and power are sampled (never set) while it runs."""
+    n = min(max_steps, int(math.ceil(seconds / (step_ms * 1e-3) * 1.1)))
+    slots0 = M.mtla_position(h)[1]
+    M.mtla_profile_begin_attention(h, n)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        torch.cuda.synchronize(device)
+        ev0.record()
+        for i in range(n):
+            M.mtla_decode_step(h, xs[i % 8], y)
+        ev1.record()
+        torch.cuda.synchronize(device)
+    ms = ev0.elapsed_time(ev1)
+    attn_ms, attn_steps = M.mtla_profile_end(h)
+    slots1 = M.mtla_position(h)[1]
+    M.mtla_check(h)
+    peaks = measured_peaks()
+    work = algorithmic_work(w, 0.5 * (slots0 + 1 + slots1))
+    attn_s = attn_ms * 1e-3 / max(attn_steps, 1)
+    step_s = ms * 1e-3 / n
+    hbm_s = (work["weight_bytes"] + work["cache_bytes"]) / (peaks["hbm_gbs"] * 1e9)
+    return {"steps": n, "seconds": ms * 1e-3, "ms_per_step": ms / n,
+            "tokens_per_s": w.batch * n / (ms * 1e-3), "context_slots": [slots0, slots1],
+            "attention_us": attn_s * 1e6,
+            "attention_gbs": work["cache_bytes"] / attn_s / 1e9,
+            "attention_frac": work["cache_bytes"] / attn_s / 1e9 / peaks["hbm_gbs"],
+            "attention_frac_of_nominal_8TBs": work["cache_bytes"] / attn_s / 1e9 / NOMINAL_HBM_GBS,
+            "step_roofline_frac": hbm_s / step_s,
+            "step_roofline_frac_of_nominal_8TBs":
+                (work["weight_bytes"] + work["cache_bytes"]) / (NOMINAL_HBM_GBS * 1e9) / step_s,
+            "clocks": clocks.summary()}
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -505,6 +657,10 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch (profiling-sized variants)")
+    ap.add_argument("--sustained-seconds", type=float, default=1.0,
+                    help="length of the second, sustained timing loop (0 skips it)")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the prefill / other-configuration blocks of the default run")
     ap.add_argument("--context-tokens", type=int, default=0,
                     help="override the workload's imported context length")
     args = ap.parse_args()
@@ -542,7 +698,13 @@ def main() -> None:
         return
     w = pick_workload(args)
     K, W = args.steps, max(args.warmup, 3)
-    M, h = build_layer(w, extra_steps=3 * (K + W), device=device, paged=args.paged)
+    # Room for the sustained loop: its step count follows the measured step time, bounded here by
+    # the step's time at the nominal 8 TB/s (and by 4096 steps for the small configurations).
+    floor_ms = algorithmic_work(w, (w.prefill_tokens + w.context_tokens) / w.stride)["cache_bytes"] / 8.0e9
+    sustained_steps = 0
+    if args.sustained_seconds > 0:
+        sustained_steps = min(4096, int(args.sustained_seconds / max(floor_ms * 1e-3, 1e-5) * 1.1) + 8)
+    M, h = build_layer(w, extra_steps=3 * (K + W) + sustained_steps, device=device, paged=args.paged)
     extras = fill_context(M, h, w, device)
     dt = synth.torch_dtype(w.dtype)
     xs = [synth.decode_input(w, i).to(device) for i in range(8)]
@@ -592,6 +754,11 @@ def main() -> None:
     assert torch.isfinite(yh.float()).all()
     M.mtla_check(h)
 
+    sustained = None
+    if sustained_steps > 0:
+        sustained = run_sustained(M, h, w, xs, y, local, device, args.sustained_seconds, local_ms / K,
+                                  sustained_steps)
+
     if rank != 0:
         M.mtla_destroy(h)
         if world > 1:
@@ -636,7 +803,9 @@ def main() -> None:
                      "frac": achieved_gbs / peaks["hbm_gbs"],
                      "peak_source": f"of {peaks['source']}",
                      "frac_of_nominal_8TBs": achieved_gbs / NOMINAL_HBM_GBS,
-                     "launch_ms": attn_launch_s * 1e3, "traffic": traffic},
+                     "launch_ms": attn_launch_s * 1e3, "traffic": traffic,
+                     "note": "burst figure of the K-step region; the `sustained` block repeats it over "
+                             "a loop of a second or more, under the board's power limit"},
         "step_roofline": {"hbm_time_ms": hbm_time * 1e3, "tensor_time_ms": tensor_time * 1e3,
                           "frac": max(hbm_time, tensor_time) / step_s,
                           "frac_of_nominal_8TBs": max(
@@ -650,11 +819,15 @@ def main() -> None:
         "gpu_launches": int(launches),
         "clocks": clocks.summary(),
     }
+    if sustained:
+        line["sustained"] = sustained
     if extras:
-        line["prefill"] = extras
+        line["prefill_of_this_workload"] = extras
     M.mtla_destroy(h)
-    del h
+    del h, xs, y
     torch.cuda.empty_cache()
+    if world == 1 and args.workload == "large" and not args.no_other_configs and not args.batch:
+        line["prefill"], line["configs"] = run_other_configs(device)
     if world == 1 and not args.no_cpu_baseline:
         n_seq = 1 if w.batch * w.latent_rank >= 8192 else min(w.batch, 4)
         res = oracle_decode_sample(w, n_seq, budget_s=12.0, max_steps=64)

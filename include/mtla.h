@@ -46,6 +46,9 @@ typedef enum {
 } mtla_status;
 
 enum { MTLA_DTYPE_FP32 = 0, MTLA_DTYPE_BF16 = 1 };
+/* mtla_config.kernel_path: which kernels a bf16 layer with r a multiple of 128 runs on.  Every
+ * other layer runs on the CUDA-core kernels whatever the setting. */
+enum { MTLA_PATH_AUTO = 0, MTLA_PATH_CUDA_CORE = 1 };
 
 /* Layer dimensions (paper's Section 4 and 4.3) and capacities. */
 typedef struct {
@@ -62,6 +65,7 @@ typedef struct {
   int32_t dtype;              /* MTLA_DTYPE_* */
   float ln_eps;               /* 0 selects 1e-5 */
   float rope_theta;           /* 0 selects 10000 */
+  int32_t kernel_path;        /* MTLA_PATH_*: AUTO takes the tensor-core kernels where they apply */
 } mtla_config;
 
 /* Device pointers to the parameters, row-major [in][out], element type config.dtype.
@@ -158,10 +162,12 @@ int mtla_decode_step_host(mtla_handle* h, const void* x_host, int32_t B, void* y
  * same within rounding (the partials are summed in the same order).
  *   - Limit: (B + 148) * n_h * (r + 2) * 4 bytes (B + 296 units on the CUDA-core path) plus
  *     the tickets must fit the array; otherwise MTLA_ERR_SCRATCH_LIMIT is returned and nothing
- *     is enqueued.  The paper's layer (8 heads, r 256) fits up to B = 350.
- *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress,
- *     checked); make that first call with the handle's device current and before starting
- *     any stream capture.
+ *     is enqueued.  The paper's layer (8 heads, r 256) fits up to B = 359.
+ *   - Every GPU has its own copy of the array, so the GPU that owns the handle's arena must be
+ *     the current device on every call (MTLA_ERR_STATE otherwise).  The first call on a device
+ *     resolves the array's device address (cudaGetSymbolAddress, checked); make that first
+ *     call before starting any stream capture.  The address cache is filled without a lock:
+ *     concurrent first calls store the same value.
  *   - All handles and all calls on a device share the one array, and it keeps the previous
  *     call's contents.  The tickets are cleared on `stream` at the start of every call; the
  *     partials are fully rewritten before they are read.  Two calls whose kernels may overlap
@@ -175,8 +181,8 @@ int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, v
  * The attentions the paper compares against, at the same boundary, so that its speed and
  * cache-size ratios can be restated on this hardware: q = x W_Q (n_h heads), k = x W_K and
  * v = x W_V (n_kv_heads heads, each shared by n_h / n_kv_heads query heads: n_kv_heads = n_h is
- * MHA, 1 is MQA), standard rotary embedding of q and k at the token's position (Appendix:
- * "Standard RoPE is used in MHA"), softmax(q K^T / sqrt(d_h)) V over the cached keys and values
+ * MHA, 1 is MQA), the ordinary rotary embedding of q and k at the token's position (what the
+ * appendix on the training set-up states for MHA), softmax(q K^T / sqrt(d_h)) V over the cached keys and values
  * including the token's own, y = concat(heads) W_O.  bf16 only.  The cache keeps 2 n_kv_heads d_h
  * elements per token, laid out [sequence][kv head][token][value | key].
  * A handle made by mtla_baseline_create is used with mtla_decode_step, mtla_cache_bytes,
@@ -273,6 +279,16 @@ int mtla_page_pool_ref(const mtla_page_pool* p, int32_t page);
 /* Synchronises `stream` and reports a sticky device-side status (MTLA_ERR_DEVICE_TIMEOUT if
  * a bounded wait inside a kernel gave up; MTLA_ERR_CUDA if the stream is in error). */
 int mtla_check(mtla_handle* h, void* stream);
+
+/* Diagnostics of the bounded device-side waits.  Every wait inside the tensor-core kernels
+ * gives up after a time budget, records a code and lets the kernel return, which is what
+ * mtla_check reports as MTLA_ERR_DEVICE_TIMEOUT.  mtla_selftest_wait_timeout exercises that path
+ * on purpose and harmlessly: it enqueues a one-CTA kernel whose only wait (on a barrier nobody
+ * arrives at) has a budget of budget_us microseconds (1 .. 1000000); the kernel returns by
+ * itself, and the next mtla_check on the stream reports the timeout.  The status is sticky
+ * until mtla_clear_error, which zeroes it on `stream`. */
+int mtla_selftest_wait_timeout(mtla_handle* h, int32_t budget_us, void* stream);
+int mtla_clear_error(mtla_handle* h, void* stream);
 
 /* Number of kernels the library has launched on behalf of this handle since creation. */
 int64_t mtla_launch_count(const mtla_handle* h);

@@ -15,6 +15,7 @@ import torch
 from .build import LIB_PATH, build_library
 
 MTLA_DTYPE_FP32, MTLA_DTYPE_BF16 = 0, 1
+MTLA_PATH_AUTO, MTLA_PATH_CUDA_CORE = 0, 1
 _DTYPES = {torch.float32: MTLA_DTYPE_FP32, torch.bfloat16: MTLA_DTYPE_BF16,
            "fp32": MTLA_DTYPE_FP32, "bf16": MTLA_DTYPE_BF16}
 _TORCH_DTYPES = {MTLA_DTYPE_FP32: torch.float32, MTLA_DTYPE_BF16: torch.bfloat16}
@@ -32,7 +33,8 @@ EXPORTED_SYMBOLS = (
     "mtla_seq_positions", "mtla_pages_in_use", "mtla_cache_export_seq", "mtla_cache_import_seqs",
     "mtla_page_pool_create", "mtla_page_pool_destroy", "mtla_page_pool_prepare",
     "mtla_page_pool_reorder", "mtla_page_pool_row", "mtla_page_pool_in_use", "mtla_page_pool_ref",
-    "mtla_baseline_arena_bytes", "mtla_baseline_create")
+    "mtla_baseline_arena_bytes", "mtla_baseline_create", "mtla_selftest_wait_timeout",
+    "mtla_clear_error")
 
 PAGE_SLOTS = 64
 
@@ -50,7 +52,8 @@ class mtla_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "d_model", "n_heads", "head_dim", "latent_rank", "rope_dim", "stride", "hyper_dim",
         "max_batch", "max_tokens", "max_prefill_tokens", "dtype")] + [
-        ("ln_eps", ctypes.c_float), ("rope_theta", ctypes.c_float)]
+        ("ln_eps", ctypes.c_float), ("rope_theta", ctypes.c_float),
+        ("kernel_path", ctypes.c_int32)]
 
 
 class mtla_paging(ctypes.Structure):
@@ -127,6 +130,8 @@ def load_library() -> ctypes.CDLL:
         "mtla_profile_end_stages": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
                                                    ctypes.POINTER(i32)]),
         "mtla_error_string": (ctypes.c_char_p, [ctypes.c_int]),
+        "mtla_selftest_wait_timeout": (ctypes.c_int, [vp, i32, vp]),
+        "mtla_clear_error": (ctypes.c_int, [vp, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -162,10 +167,10 @@ class Handle:
 
 def make_config(*, d_model, n_heads, head_dim, latent_rank, rope_dim, stride, hyper_dim=0,
                 max_batch, max_tokens, max_prefill_tokens=0, dtype="bf16", ln_eps=0.0,
-                rope_theta=0.0) -> mtla_config:
+                rope_theta=0.0, kernel_path=0) -> mtla_config:
     return mtla_config(d_model, n_heads, head_dim, latent_rank, rope_dim, stride, hyper_dim,
                        max_batch, max_tokens, max_prefill_tokens, _DTYPES[dtype], ln_eps,
-                       rope_theta)
+                       rope_theta, kernel_path)
 
 
 def mtla_arena_bytes(cfg: mtla_config) -> int:
@@ -460,6 +465,16 @@ def mtla_cache_import(h: Handle, cache: torch.Tensor, tokens: int, stream=None) 
 
 def mtla_check(h: Handle, stream=None) -> None:
     _check(load_library().mtla_check(h.ptr, _stream_ptr(stream)), "mtla_check")
+
+
+def mtla_selftest_wait_timeout(h: Handle, budget_us: int, stream=None) -> None:
+    """Enqueues the one-CTA kernel whose bounded wait runs out after budget_us microseconds."""
+    _check(load_library().mtla_selftest_wait_timeout(h.ptr, budget_us, _stream_ptr(stream)),
+           "mtla_selftest_wait_timeout")
+
+
+def mtla_clear_error(h: Handle, stream=None) -> None:
+    _check(load_library().mtla_clear_error(h.ptr, _stream_ptr(stream)), "mtla_clear_error")
 
 
 def mtla_launch_count(h: Handle) -> int:

@@ -259,11 +259,13 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     prefetch_tensormap(&q_map);
   }
   if (warp == 1) tmem_alloc(smem_u32(&misc->tmem_base), kTmemCols);
-  grid_launch_dependents();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = misc->tmem_base;
+  // Only now may the next kernel's CTAs start: this CTA owns its TMEM columns, so a successor
+  // that shares the SM cannot take them first and then sit in its dependency wait.
+  grid_launch_dependents();
   grid_dependency_wait();        // nothing before this line touches the previous kernel's data
 
   // This CTA's share of the tile list.

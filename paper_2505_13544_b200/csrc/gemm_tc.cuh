@@ -156,11 +156,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     prefetch_tensormap(&map_b);
   }
   if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), TMEM_COLS);
-  grid_launch_dependents();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
+  // Only now may the next kernel's CTAs start: this CTA owns its TMEM columns, so a successor
+  // that shares the SM cannot take them first and then sit in its dependency wait.
+  grid_launch_dependents();
   grid_dependency_wait();        // nothing before this line touches the previous kernel's data
 
   const int mt = blockIdx.x % g.m_tiles, ny = blockIdx.x / g.m_tiles;

@@ -22,18 +22,21 @@
 #include "setup_kernels.cuh"
 #include "paging_kernels.cuh"
 #include "baseline_kernels.cuh"
+#include "selftest_kernels.cuh"
 #include "page_pool.h"
 
 using namespace mtla;
 
 namespace {
 
-constexpr int kSmCount = 148;        // B200
-constexpr int kTargetCtas = 296;     // two CTAs per SM on a 148-SM part
+// The split workspaces are sized for persistent grids of up to kPlanSms CTAs (B200: 148 SMs);
+// the grids themselves follow the device's SM count read at create, capped at this bound.
+constexpr int kPlanSms = 148;
+constexpr int kTargetCtas = 2 * kPlanSms;   // CUDA-core attention: two CTAs per SM
 constexpr int kMinSlotsPerSplit = 64;
 constexpr int kFusedCombineMaxParts = 8;   // more parts per sequence: the combine gets its own launch
 constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill projections
-constexpr int kGemmSlots = 2 * kSmCount;   // CTAs a split-K GEMM may spread one product over
+constexpr int kGemmSlots = 2 * kPlanSms;   // CTAs a split-K GEMM may spread one product over
 
 // Rows of the activation-side TMA box (the MMA's N) for a decode batch of B sequences.
 int act_box_rows(int B) {
@@ -75,6 +78,7 @@ bool normalise(const mtla_config* in, const mtla_paging* pg, mtla_config* out, D
   if (c.hyper_dim < 1 || c.hyper_dim > 256) return false;
   if (c.max_batch < 1 || c.max_tokens < 1 || c.max_prefill_tokens < 0) return false;
   if (c.dtype != MTLA_DTYPE_FP32 && c.dtype != MTLA_DTYPE_BF16) return false;
+  if (c.kernel_path != MTLA_PATH_AUTO && c.kernel_path != MTLA_PATH_CUDA_CORE) return false;
   if (!(c.ln_eps > 0.f) || !(c.rope_theta > 0.f)) return false;
   if ((long long)c.max_batch * c.max_tokens > (1ll << 31)) return false;
   *out = c;
@@ -166,6 +170,19 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// The GPU that owns `arena` and its SM count (capped at the planning bound).
+int arena_device(const void* arena, int* device, int* sm_count) {
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, arena) != cudaSuccess) return MTLA_ERR_CUDA;
+  if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) return MTLA_ERR_INVALID_ARG;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, attr.device) != cudaSuccess || sms < 1)
+    return MTLA_ERR_CUDA;
+  *device = attr.device;
+  *sm_count = sms < kPlanSms ? sms : kPlanSms;
+  return MTLA_OK;
+}
+
 }  // namespace
 
 // Split workspace of mtla_decode_step_static: lives in every GPU that loads the library, for
@@ -193,6 +210,8 @@ struct mtla_handle {
   bool is_baseline;
   int bl_groups;
   int64_t launches;
+  int device;     // ordinal of the GPU that owns the arena
+  int sm_count;   // its SM count, capped at the bound the workspaces are sized for
   bool attn_smem_ready, pf_smem_ready;
   // Tensor-core decode attention (bf16, r a multiple of 128): TMA view of the cache.
   bool use_tc;
@@ -400,7 +419,7 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   const int kb_total = ceil_div(g.k, gtc::kBK);
   // Stacked hi / lo halves double the B tile: one CTA per SM then, two otherwise.
   const bool hilo = g.b_lo_col > 0 && bn <= 128 && sizeof(OutT) == 2;
-  const int slots = (hilo && bn == 128) || bn == 256 ? kSmCount : kGemmSlots;
+  const int slots = (hilo && bn == 128) || bn == 256 ? h->sm_count : 2 * h->sm_count;
   int n_split = 1;
   // The partials are summed by the last CTA of a tile alone: at most four splits keep that short.
   if (allow_split && tiles < slots) n_split = max(1, min(min(kb_total / 4, (int)(slots / tiles)), 4));
@@ -746,7 +765,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     ta.page_table = h->paged() ? h->d_page_table(buf) : nullptr;
     ta.max_pages = dm.max_pages; ta.stride = dm.s;
     const long long total = h->paged() ? ragged_tiles : (long long)B * ta.tiles_per_seq;
-    const int grid = (int)(total < kSmCount ? total : kSmCount);
+    const int grid = (int)(total < h->sm_count ? total : h->sm_count);
     aa.n_split = 0;
     // A lock-step batch whose sequences are each spread over many CTAs hands the combine to a
     // launch of its own, one CTA per (head, sequence), instead of one CTA per sequence.
@@ -767,7 +786,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
       h->launches++;
     }
   } else {
-    int want = ceil_div(kTargetCtas, B);
+    int want = ceil_div(2 * h->sm_count, B);
     int n_split = min(want, ceil_div(n_slots, kMinSlotsPerSplit));
     if (n_split < 1) n_split = 1;
     aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
@@ -1170,6 +1189,11 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
   h->tokens_stale = false;
   h->is_baseline = false;
   h->bl_groups = 1;
+  const int dev_rc = arena_device(arena, &h->device, &h->sm_count);
+  if (dev_rc != MTLA_OK) {
+    delete h;
+    return dev_rc;
+  }
   if (paging) {
     h->pool = new (std::nothrow) PagePool(dm.n_pages, c.max_batch, dm.max_pages);
     if (!h->pool) {
@@ -1179,10 +1203,9 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
     h->seq_tokens.assign(c.max_batch, 0);
     h->tokens_stale = true;
   }
-  // The tensor-core attention needs bf16 and whole 128-column latent blocks; the
-  // MTLA_ATTENTION=fma environment override keeps the CUDA-core kernel for comparisons.
-  const char* force = getenv("MTLA_ATTENTION");
-  h->use_tc = c.dtype == MTLA_DTYPE_BF16 && dm.r % 128 == 0 && !(force && !strcmp(force, "fma"));
+  // The tensor-core kernels need bf16 and whole 128-column latent blocks; config.kernel_path
+  // can keep such a layer on the CUDA-core kernels (for comparisons between the two).
+  h->use_tc = c.dtype == MTLA_DTYPE_BF16 && dm.r % 128 == 0 && c.kernel_path != MTLA_PATH_CUDA_CORE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int rc = c.dtype == MTLA_DTYPE_BF16 ? create_impl<bf16>(h, w, st) : create_impl<float>(h, w, st);
   if (rc != MTLA_OK) {
@@ -1220,7 +1243,7 @@ bool baseline_dims(const mtla_baseline_config* in, mtla_config* cfg, Dims* dm, i
   dm->r = dm->W; dm->dr = 0;
   dm->max_slots = in->max_tokens;
   dm->ntot = (in->n_heads + 2 * in->n_kv_heads) * in->head_dim;
-  dm->max_units = kSmCount + in->max_batch * in->n_kv_heads;
+  dm->max_units = kPlanSms + in->max_batch * in->n_kv_heads;
   *groups = in->n_kv_heads;
   return true;
 }
@@ -1292,7 +1315,7 @@ int baseline_decode(mtla_handle* h, const void* x, int B, void* y, cudaStream_t 
   ta.n_heads = dm.nh; ta.r = dm.W; ta.dr = 0; ta.n_slots = pos + 1; ta.batch = B * g;
   ta.tiles_per_seq = ceil_div(pos + 1, tc::kTile);
   const long long total = (long long)ta.batch * ta.tiles_per_seq;
-  const int grid = (int)(total < kSmCount ? total : kSmCount);
+  const int grid = (int)(total < h->sm_count ? total : h->sm_count);
   const bool attn_pdl = pdl && !prof;
   const bool split_combine = grid / ta.batch + 2 > kFusedCombineMaxParts;
   ta.fused_combine = !split_combine;
@@ -1388,6 +1411,11 @@ int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_we
   h->is_baseline = true;
   h->bl_groups = groups;
   h->use_tc = true;
+  const int dev_rc = arena_device(arena, &h->device, &h->sm_count);
+  if (dev_rc != MTLA_OK) {
+    delete h;
+    return dev_rc;
+  }
   const int rc = baseline_create(h, w, static_cast<cudaStream_t>(stream));
   if (rc != MTLA_OK) {
     delete h;
@@ -1456,15 +1484,19 @@ int mtla_decode_step_static(mtla_handle* h, const void* x, int32_t B, void* y, v
   if (h->is_baseline) return MTLA_ERR_STATE;
   // Same sizing as the arena's split workspace, for this call's batch.
   const Dims& dm = h->dm;
-  const size_t units = (size_t)(h->use_tc ? kSmCount : kTargetCtas) + (size_t)B;
+  const size_t units = (size_t)(h->use_tc ? kPlanSms : kTargetCtas) + (size_t)B;
   const size_t tickets_bytes = align_up((size_t)B * sizeof(int), 256);
   const size_t ml_bytes = align_up(units * dm.nh * 2 * sizeof(float), 256);
   const size_t o_bytes = units * dm.nh * dm.r * sizeof(float);
   if (tickets_bytes + ml_bytes + o_bytes > MTLA_STATIC_SCRATCH_BYTES) return MTLA_ERR_SCRATCH_LIMIT;
-  // First call on this device: turn the array's host-side name into its device address.
+  // The array exists once per GPU: the kernels must get the copy of the GPU that owns the
+  // handle's arena, so that GPU has to be the current one, on every call.
   int dev = -1;
   MTLA_CUDA(cudaGetDevice(&dev));
+  if (dev != h->device) return MTLA_ERR_STATE;
   if (dev < 0 || dev >= kMaxDevices) return MTLA_ERR_UNSUPPORTED_SHAPE;
+  // First call on this device: turn the array's host-side name into its device address.  Two
+  // threads that race here store the same address, so the slot needs no lock.
   if (!g_static_scratch_addr[dev]) {
     void* addr = nullptr;
     MTLA_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));
@@ -1727,6 +1759,22 @@ int mtla_check(mtla_handle* h, void* stream) {
   int flag[4] = {0, 0, 0, 0};
   MTLA_CUDA(cudaMemcpy(flag, h->at<char>(h->plan.err_flag), sizeof(flag), cudaMemcpyDeviceToHost));
   return flag[0] ? MTLA_ERR_DEVICE_TIMEOUT : MTLA_OK;
+}
+
+int mtla_selftest_wait_timeout(mtla_handle* h, int32_t budget_us, void* stream) {
+  if (!h || budget_us < 1 || budget_us > 1000000) return MTLA_ERR_INVALID_ARG;
+  int* flag = h->at<int>(h->plan.err_flag);
+  wait_timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(
+      flag, 99, (unsigned long long)budget_us * 1000ull, flag + 1);
+  h->launches++;
+  MTLA_CUDA(cudaGetLastError());
+  return MTLA_OK;
+}
+
+int mtla_clear_error(mtla_handle* h, void* stream) {
+  if (!h) return MTLA_ERR_INVALID_ARG;
+  MTLA_CUDA(cudaMemsetAsync(h->at<char>(h->plan.err_flag), 0, 16, static_cast<cudaStream_t>(stream)));
+  return MTLA_OK;
 }
 
 int64_t mtla_launch_count(const mtla_handle* h) { return h ? h->launches : 0; }

@@ -62,21 +62,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // records a code in the global error word.  Callers unwind without touching the barrier again.
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word,
-                                          int* error_word, int code) {
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int* abort_word,
+                                              int* error_word, int code, uint64_t budget_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
+    if ((it & 255u) == 0u || budget_ns < kWaitBudgetNs) {
       if (*abort_word) return false;
-      if (global_timer_ns() - t0 > kWaitBudgetNs) {
+      if (global_timer_ns() - t0 > budget_ns) {
         *abort_word = 1;
         atomicCAS(error_word, 0, code);
         return false;
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word,
+                                          int* error_word, int code) {
+  return mbar_wait_for(bar, parity, abort_word, error_word, code, kWaitBudgetNs);
 }
 
 // 2^x by the special-function unit (about 2 ulp; flushes denormals): enough for probabilities

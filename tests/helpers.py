@@ -26,13 +26,14 @@ def oracle_params(w: synth.Workload, weights: dict) -> O.Params:
 
 
 def gpu_handle(w: synth.Workload, weights: dict, max_batch=None, max_tokens=None,
-               max_prefill_tokens=None, device="cuda:0"):
+               max_prefill_tokens=None, device="cuda:0", kernel_path=0):
     from paper_2505_13544_b200 import binding as M
     cfg = M.make_config(**dims_of(w), max_batch=max_batch or w.batch,
                         max_tokens=max_tokens or w.max_tokens,
                         max_prefill_tokens=(w.prefill_tokens if max_prefill_tokens is None
                                             else max_prefill_tokens),
-                        dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+                        dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta,
+                        kernel_path=kernel_path)
     dev_weights = {k: v.to(device) for k, v in weights.items()}
     return M.mtla_create(cfg, dev_weights, device=device)
 

@@ -4,7 +4,6 @@ Shapes cover both head paddings (16 / 32), every latent block count r/128 in 1..
 RoPE widths, single-tile splits, multi-tile pipelines with ring wrap-around, and ragged tails.
 """
 import math
-import os
 
 import numpy as np
 import pytest
@@ -25,14 +24,13 @@ def workload(nh, dh, r, dr, batch, context, stride=2, d=256, seed=21):
                           decode_steps=3, seed=seed)
 
 
-def run(w, rows, monkeypatch=None, variant=None):
+def run(w, rows, variant=None):
     weights = synth.make_weights(w)
     p = H.oracle_params(w, weights)
     n_slots = math.ceil(w.context_tokens / w.stride)
     cache = torch.stack([synth.context_cache_row(w, b, n_slots) for b in range(w.batch)])
-    if variant:
-        monkeypatch.setenv("MTLA_ATTENTION", variant)
-    h = H.gpu_handle(w, weights, max_prefill_tokens=0)
+    h = H.gpu_handle(w, weights, max_prefill_tokens=0,
+                     kernel_path=M.MTLA_PATH_CUDA_CORE if variant == "fma" else M.MTLA_PATH_AUTO)
     outs = []
     try:
         assert M.mtla_attention_variant(h) == (variant or "tcgen05")
@@ -70,10 +68,10 @@ def test_tc_attention_matches_oracle(nh, dh, r, dr, batch, context):
     run(w, rows)
 
 
-def test_tc_and_fma_kernels_agree(monkeypatch):
+def test_tc_and_fma_kernels_agree():
     w = workload(32, 128, 512, 64, 5, 3000, stride=3)
     y_tc = run(w, [0, 4])
-    y_fma = run(w, [0, 4], monkeypatch, "fma")
+    y_fma = run(w, [0, 4], "fma")
     diff = (y_tc.float() - y_fma.float()).abs().max().item()
     assert diff <= 2e-2
 

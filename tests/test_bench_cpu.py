@@ -33,3 +33,14 @@ def test_traffic_capture_is_keyed_to_the_kernel_code():
     text = "int a = 1;   // one\n\n  int b = 2;\n"
     assert bench.code_hash([text]) == bench.code_hash(["int a = 1;\nint b = 2; // two\n// three\n"])
     assert bench.code_hash([text]) != bench.code_hash([text + "int c = 3;\n"])
+
+
+def test_prefill_flop_of_the_long_context_workload():
+    """Allowed pairs B n_h sum_m ceil(m/s) at 2 (d_h + d_R) + 2 d_h FLOP each, plus the three
+    projections: 2.90 TFLOP for 8 x 16384 tokens at s = 4."""
+    f = bench.prefill_flop(synth.WORKLOADS["longctx"])
+    assert abs(f["attention"] / 1e12 - 1.65) < 0.01
+    assert abs(f["total"] / 1e12 - 2.90) < 0.01
+    w = synth.WORKLOADS["tiny"].scaled(batch=1, prefill_tokens=5, stride=2)
+    pairs = 1 + 1 + 2 + 2 + 3                      # ceil(m/2) for m = 1..5
+    assert bench.prefill_flop(w)["attention"] == w.n_heads * pairs * (2 * (64 + 32) + 2 * 64)

@@ -30,8 +30,9 @@ def check_positions(h, w, tokens):
     assert M.mtla_cache_bytes(h) == w.batch * slots * w.slot_width * elem_bytes(w)
 
 
-def run_prefill_then_decode(w, seqs, prefill_rows, decode_steps_checked):
-    """Prefill the whole batch, then decode w.decode_steps steps; compare sampled outputs."""
+def run_prefill_then_decode(w, seqs, prefill_rows, decode_steps_checked, rows_by_seq=None):
+    """Prefill the whole batch, then decode w.decode_steps steps; compare sampled outputs.
+    rows_by_seq overrides the sampled prefill rows for individual sequences."""
     weights = synth.make_weights(w)
     p = H.oracle_params(w, weights)
     h = H.gpu_handle(w, weights)
@@ -50,8 +51,9 @@ def run_prefill_then_decode(w, seqs, prefill_rows, decode_steps_checked):
         check_positions(h, w, w.prefill_tokens)
         states = {}
         for b in seqs:
-            want, st = O.decode_sequence(p, prompts[b], rows=prefill_rows)
-            H.assert_close(y[b, prefill_rows], want, w.dtype, f"prefill seq {b}")
+            rows_b = (rows_by_seq or {}).get(b, prefill_rows)
+            want, st = O.decode_sequence(p, prompts[b], rows=rows_b)
+            H.assert_close(y[b, rows_b], want, w.dtype, f"prefill seq {b}")
             states[b] = st
         cache = M.mtla_cache_export(h)
         H.assert_cache_close(cache[seqs], np.stack([O.cache_array(states[b]) for b in seqs]), w.dtype)
@@ -95,9 +97,22 @@ def test_config_stride_sweep(s):
 
 
 def test_config_long_context_prefill():
+    """Sequence 0: every row of the first, a middle and the last pair of 128-row query tiles (one
+    CTA of the two-tile kernel each); sequence 7: scattered rows."""
     w = synth.WORKLOADS["longctx"]
     rows = [0, 3, 4, 255, 256, 8191, 16380, 16383]
-    run_prefill_then_decode(w, [0, 7], rows, {0, 1, 3, 4, 63})
+    pairs = sorted(set(range(0, 256)) | set(range(8192, 8448)) | set(range(16128, 16384)) | set(rows))
+    run_prefill_then_decode(w, [0, 7], rows, {0, 1, 3, 4, 63}, rows_by_seq={0: pairs})
+
+
+def test_large_layer_prefill_then_decode():
+    """The layer of the large workload (d 4096, 32 heads x 128, r 512, d_R 64, s 2) through the
+    prefill and into decoding: B 2, T 2048.  Whole first and last query tiles, the rows around the
+    middle, then six decode steps from the handed-over state."""
+    w = synth.WORKLOADS["large"].scaled(name="large_prefill", batch=2, prefill_tokens=2048,
+                                        context_tokens=0, decode_steps=6)
+    rows = sorted(set(range(0, 128)) | set(range(1016, 1032)) | set(range(1920, 2048)))
+    run_prefill_then_decode(w, [0, 1], rows, set(range(6)))
 
 
 def test_config_large_decode():
