@@ -71,7 +71,7 @@ def test_static_scratch_limit_is_reported_and_leaves_the_handle_untouched():
 
 def test_static_scratch_step_allocates_nothing():
     """With y preallocated, neither torch's allocator nor the driver hands out memory during the call."""
-    w = layer("bf16", 8, 256, batch=5, context=900)
+    w = layer("bf16", 8, 256, batch=5, context=900).scaled(decode_steps=8)
     weights = synth.make_weights(w)
     n_slots = math.ceil(w.context_tokens / w.stride)
     cache = torch.stack([synth.context_cache_row(w, b, n_slots) for b in range(w.batch)]).cuda()
