@@ -102,20 +102,20 @@ def stored(a: np.ndarray, dtype: str) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a)).to(torch_dtype(dtype))
 
 
-def make_weights(w: Workload) -> dict[str, torch.Tensor]:
+def make_weights(w: Workload, prefix: str = "") -> dict[str, torch.Tensor]:
     """All layer parameters, row-major [in][out], already rounded to w.dtype.
 
     Weight matrices are N(0,1)/sqrt(fan_in); LayerNorm gain 1 + 0.1 N(0,1), its bias and
-    the hyper-network biases 0.1 N(0,1).
+    the hyper-network biases 0.1 N(0,1).  `prefix` names the layer inside a stack.
     """
     d, nh, dh, r, dr, dw = (w.d_model, w.n_heads, w.head_dim, w.latent_rank, w.rope_dim,
                             w.hyper_dim)
 
     def mat(name, fan_in, fan_out):
-        return stored(normal(w.seed, name, (fan_in, fan_out), scale=fan_in ** -0.5), w.dtype)
+        return stored(normal(w.seed, prefix + name, (fan_in, fan_out), scale=fan_in ** -0.5), w.dtype)
 
     def vec(name, n, scale, shift=0.0):
-        return stored(normal(w.seed, name, (n,), scale=scale, shift=shift), w.dtype)
+        return stored(normal(w.seed, prefix + name, (n,), scale=scale, shift=shift), w.dtype)
 
     return {
         "w_q": mat("w_q", d, nh * dh),
@@ -132,6 +132,51 @@ def make_weights(w: Workload) -> dict[str, torch.Tensor]:
         "hyp_pe_w": mat("hyp_pe_w", r, dw),
         "hyp_pe_b": vec("hyp_pe_b", dw, 0.1),
     }
+
+
+@dataclass(frozen=True)
+class StackWorkload:
+    """The paper's decoder (Section 5.2, appendix on hyper-parameters): n_layers layers of MTLA
+    self-attention + feed-forward block of width d_ff, the encoder output being the first
+    prompt_tokens rows of the input sequence."""
+    name: str
+    layer: Workload       # attention dims, dtype, batch, prompt length (prefill_tokens), steps, seed
+    n_layers: int
+    d_ff: int
+
+
+STACK_WORKLOADS: dict[str, StackWorkload] = {
+    # 9 layers, d 512, feed-forward 2048, 8 heads, r 256, d_R 32, s 2; a 512-frame prompt.
+    "decoder_paper": StackWorkload("decoder_paper", WORKLOADS["paper"].scaled(
+        name="decoder_paper", prefill_tokens=512, decode_steps=256), n_layers=9, d_ff=2048),
+}
+
+
+def make_stack_weights(sw: StackWorkload) -> dict:
+    """Parameters of every layer of the stack plus the final LayerNorm, rounded to the storage
+    type: {"layers": [{attention weights..., ln1_gamma, ln1_beta, ln2_gamma, ln2_beta, w1, b1,
+    w2, b2}], "lnf_gamma", "lnf_beta"}.  Matrices N(0,1)/sqrt(fan_in), row-major [in][out];
+    LayerNorm gains 1 + 0.1 N(0,1); biases 0.1 N(0,1)."""
+    w = sw.layer
+    d = w.d_model
+
+    def vec(name, n, shift=0.0):
+        return stored(normal(w.seed, name, (n,), scale=0.1, shift=shift), w.dtype)
+
+    layers = []
+    for n in range(sw.n_layers):
+        pre = f"layer{n}/"
+        lw = make_weights(w, prefix=pre)
+        lw.update({
+            "ln1_gamma": vec(pre + "ln1_gamma", d, 1.0), "ln1_beta": vec(pre + "ln1_beta", d),
+            "ln2_gamma": vec(pre + "ln2_gamma", d, 1.0), "ln2_beta": vec(pre + "ln2_beta", d),
+            "w1": stored(normal(w.seed, pre + "w1", (d, sw.d_ff), scale=d ** -0.5), w.dtype),
+            "b1": vec(pre + "b1", sw.d_ff),
+            "w2": stored(normal(w.seed, pre + "w2", (sw.d_ff, d), scale=sw.d_ff ** -0.5), w.dtype),
+            "b2": vec(pre + "b2", d),
+        })
+        layers.append(lw)
+    return {"layers": layers, "lnf_gamma": vec("lnf_gamma", d, 1.0), "lnf_beta": vec("lnf_beta", d)}
 
 
 def make_baseline_weights(w: Workload, n_kv_heads: int) -> dict[str, torch.Tensor]:

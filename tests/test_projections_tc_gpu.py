@@ -106,3 +106,38 @@ def test_split_k_reduction_is_deterministic():
         finally:
             M.mtla_destroy(h)
     assert torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("batch", [2, 20, 40, 100, 200])
+def test_weight_streaming_schedule_matches_oracle(batch):
+    """The layer of the large workload (d 4096, 32 heads x 128, r 512): the input and output
+    projections have few 128-row weight tiles and a 64-block reduction, which the persistent GEMM
+    cuts into equal shares that end inside tiles (partials + ticketed sum).  One batch per
+    activation box height, 16 to 256 rows; all rows against the oracle, and twice for bit-equality."""
+    w = synth.WORKLOADS["large"].scaled(name="stream", batch=batch, context_tokens=200, decode_steps=3)
+    weights = synth.make_weights(w)
+    p = H.oracle_params(w, weights)
+    n_slots = math.ceil(w.context_tokens / w.stride)
+    cache = torch.stack([synth.context_cache_row(w, b, n_slots) for b in range(batch)])
+    rows = sorted({0, 1, batch // 2, batch - 1})
+    outs = []
+    for rep in range(2):
+        h = H.gpu_handle(w, weights, max_prefill_tokens=0)
+        try:
+            M.mtla_cache_import(h, cache.cuda(), w.context_tokens)
+            states = {b: O.state_from_cache(cache[b].double().numpy(), w.context_tokens, p)
+                      for b in rows}
+            ys = []
+            for i in range(w.decode_steps):
+                x = synth.decode_input(synth.WORKLOADS["large"], i, batch=batch) if batch <= 128 else \
+                    synth.stored(synth.normal(w.seed, f"x200/{i}", (batch, w.d_model)), "bf16")
+                y = M.mtla_decode_step(h, x.cuda())
+                M.mtla_check(h)
+                ys.append(y.cpu())
+                if rep == 0:
+                    want = np.stack([O.decode_step(p, states[b], x[b].double().numpy()) for b in rows])
+                    H.assert_close(y[rows], want, "bf16", f"step {i}")
+            outs.append(torch.stack(ys))
+        finally:
+            M.mtla_destroy(h)
+    assert torch.equal(outs[0], outs[1])
