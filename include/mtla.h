@@ -205,6 +205,57 @@ size_t mtla_baseline_arena_bytes(const mtla_baseline_config* cfg);
 int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_weights* weights,
                          void* arena, size_t arena_bytes, void* stream, mtla_handle** out);
 
+/* ---- decoder layers and stacks (Section 5.2; appendix on hyper-parameters) ----
+ *
+ * The paper's model is a Transformer decoder without cross-attention (the encoder output is
+ * simply the first part of the input sequence): 9 layers of width 512 with 8 heads and a
+ * feed-forward block of width 2048, every layer's self-attention being MTLA.  A stack is that
+ * model's hot path: n_layers layers, each
+ *     h = x + MTLA(LayerNorm_1(x));   y = h + W_2 relu(W_1 LayerNorm_2(h) + b_1) + b_2,
+ * followed by one final LayerNorm.  Pre-norm placement and ReLU are the usual settings of the
+ * toolkit the paper builds on (the paper states neither).  Every layer has the attention
+ * dimensions of `cfg` and its own weights and cache; the residual stream between sub-layers is
+ * kept in fp32, x and y are in cfg.dtype.  All layers advance in lock-step.
+ * Weights: device pointers, row-major [in][out], element type cfg.dtype, repacked at create and
+ * not referenced afterwards.  `layers` is a host array of n_layers entries. */
+typedef struct {
+  mtla_weights attn;                     /* the layer's self-attention (Section 4) */
+  const void *ln1_gamma, *ln1_beta;      /* [d]  LayerNorm in front of the attention */
+  const void *ln2_gamma, *ln2_beta;      /* [d]  LayerNorm in front of the feed-forward block */
+  const void *w1, *b1;                   /* [d][d_ff], [d_ff] */
+  const void *w2, *b2;                   /* [d_ff][d], [d] */
+} mtla_layer_weights;
+typedef struct {
+  int32_t n_layers;                      /* 1..256; the paper: 9 */
+  int32_t d_ff;                          /* feed-forward width, multiple of 8; the paper: 2048 */
+  float ln_eps;                          /* eps of the layers' LayerNorms; 0 selects 1e-5 */
+} mtla_stack_config;
+typedef struct mtla_stack mtla_stack;
+
+/* Device bytes mtla_stack_create needs (0 if the pair is invalid), and the constructor: arena
+ * device, 1024-byte aligned; lnf_gamma / lnf_beta [d] are the final LayerNorm. */
+size_t mtla_stack_arena_bytes(const mtla_config* cfg, const mtla_stack_config* scfg);
+int mtla_stack_create(const mtla_config* cfg, const mtla_stack_config* scfg,
+                      const mtla_layer_weights* layers, const void* lnf_gamma, const void* lnf_beta,
+                      void* arena, size_t arena_bytes, void* stream, mtla_stack** out);
+
+/* mtla_prefill / mtla_decode_step through every layer: x device [B][T][d] resp. [B][d], y the
+ * stack's output of the same shape (required).  Errors as for the single-layer calls. */
+int mtla_stack_prefill(mtla_stack* s, const void* x, int32_t B, int32_t T, void* y, void* stream);
+int mtla_stack_decode_step(mtla_stack* s, const void* x, int32_t B, void* y, void* stream);
+
+/* Cache bytes in use over all layers (n_layers times the per-layer count of Section 4.3). */
+size_t mtla_stack_cache_bytes(const mtla_stack* s);
+
+/* The attention handle of one layer, borrowed (valid until mtla_stack_destroy; do not destroy
+ * it): for mtla_position, mtla_cache_export and the other inspection calls. */
+mtla_handle* mtla_stack_layer(mtla_stack* s, int32_t layer);
+
+int mtla_stack_reset(mtla_stack* s);                       /* empties every layer's cache */
+int mtla_stack_check(mtla_stack* s, void* stream);          /* mtla_check over the layers */
+int64_t mtla_stack_launch_count(const mtla_stack* s);
+int mtla_stack_destroy(mtla_stack* s);
+
 /* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3);
  * with per-sequence token counts, the sum over the sequences. */
 size_t mtla_cache_bytes(const mtla_handle* h);

@@ -34,7 +34,9 @@ EXPORTED_SYMBOLS = (
     "mtla_page_pool_create", "mtla_page_pool_destroy", "mtla_page_pool_prepare",
     "mtla_page_pool_reorder", "mtla_page_pool_row", "mtla_page_pool_in_use", "mtla_page_pool_ref",
     "mtla_baseline_arena_bytes", "mtla_baseline_create", "mtla_selftest_wait_timeout",
-    "mtla_clear_error")
+    "mtla_clear_error", "mtla_stack_arena_bytes", "mtla_stack_create", "mtla_stack_prefill",
+    "mtla_stack_decode_step", "mtla_stack_cache_bytes", "mtla_stack_layer", "mtla_stack_reset",
+    "mtla_stack_check", "mtla_stack_launch_count", "mtla_stack_destroy")
 
 PAGE_SLOTS = 64
 
@@ -72,6 +74,17 @@ class mtla_baseline_weights(ctypes.Structure):
 
 class mtla_weights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES]
+
+
+LAYER_EXTRA_NAMES = ("ln1_gamma", "ln1_beta", "ln2_gamma", "ln2_beta", "w1", "b1", "w2", "b2")
+
+
+class mtla_layer_weights(ctypes.Structure):
+    _fields_ = [("attn", mtla_weights)] + [(n, ctypes.c_void_p) for n in LAYER_EXTRA_NAMES]
+
+
+class mtla_stack_config(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("ln_eps", ctypes.c_float)]
 
 
 _lib = None
@@ -130,6 +143,18 @@ def load_library() -> ctypes.CDLL:
         "mtla_profile_end_stages": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
                                                    ctypes.POINTER(i32)]),
         "mtla_error_string": (ctypes.c_char_p, [ctypes.c_int]),
+        "mtla_stack_arena_bytes": (sz, [cfg_p, ctypes.POINTER(mtla_stack_config)]),
+        "mtla_stack_create": (ctypes.c_int, [cfg_p, ctypes.POINTER(mtla_stack_config),
+                                             ctypes.POINTER(mtla_layer_weights), vp, vp, vp, sz, vp,
+                                             ctypes.POINTER(vp)]),
+        "mtla_stack_prefill": (ctypes.c_int, [vp, vp, i32, i32, vp, vp]),
+        "mtla_stack_decode_step": (ctypes.c_int, [vp, vp, i32, vp, vp]),
+        "mtla_stack_cache_bytes": (sz, [vp]),
+        "mtla_stack_layer": (vp, [vp, i32]),
+        "mtla_stack_reset": (ctypes.c_int, [vp]),
+        "mtla_stack_check": (ctypes.c_int, [vp, vp]),
+        "mtla_stack_launch_count": (ctypes.c_int64, [vp]),
+        "mtla_stack_destroy": (ctypes.c_int, [vp]),
         "mtla_selftest_wait_timeout": (ctypes.c_int, [vp, i32, vp]),
         "mtla_clear_error": (ctypes.c_int, [vp, vp]),
     }
@@ -508,3 +533,116 @@ def mtla_profile_end_stages(h: Handle) -> tuple[dict, int]:
     _check(load_library().mtla_profile_end_stages(h.ptr, ms, ctypes.byref(steps)),
            "mtla_profile_end_stages")
     return dict(zip(DECODE_STAGES, list(ms))), steps.value
+
+
+# --------------------------------------------------------------------------- decoder stacks
+
+@dataclass
+class Stack:
+    """A live decoder stack: the C object plus the arena that must outlive it."""
+    ptr: int
+    config: mtla_config
+    n_layers: int
+    d_ff: int
+    arena: torch.Tensor
+    dtype: torch.dtype
+    device: torch.device
+
+
+def mtla_stack_arena_bytes(cfg: mtla_config, n_layers: int, d_ff: int) -> int:
+    sc = mtla_stack_config(n_layers, d_ff, 0.0)
+    return load_library().mtla_stack_arena_bytes(ctypes.byref(cfg), ctypes.byref(sc))
+
+
+def mtla_stack_create(cfg: mtla_config, n_layers: int, d_ff: int, weights: dict, ln_eps: float = 0.0,
+                      device="cuda:0", stream=None) -> Stack:
+    """weights: {"layers": [per-layer dict of the attention weights plus ln1_gamma .. b2],
+    "lnf_gamma", "lnf_beta"}, CUDA tensors of cfg.dtype, matrices row-major [in][out]."""
+    lib = load_library()
+    sc = mtla_stack_config(n_layers, d_ff, ln_eps)
+    nbytes = lib.mtla_stack_arena_bytes(ctypes.byref(cfg), ctypes.byref(sc))
+    if nbytes == 0:
+        raise MTLAError(-2, "mtla_stack_arena_bytes")
+    device = torch.device(device)
+    dtype = _TORCH_DTYPES[cfg.dtype]
+    keep = []
+
+    def ptr(t, name):
+        if t is None:
+            return None
+        if t.dtype != dtype or not t.is_cuda:
+            raise TypeError(f"weight {name}: expected a {dtype} CUDA tensor")
+        t = t.contiguous()
+        keep.append(t)
+        return t.data_ptr()
+
+    with torch.cuda.device(device):
+        arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+        base = (arena.data_ptr() + 1023) // 1024 * 1024
+        arr = (mtla_layer_weights * n_layers)()
+        for n, lw in enumerate(weights["layers"]):
+            for name in WEIGHT_NAMES:
+                setattr(arr[n].attn, name, ptr(lw.get(name), name))
+            for name in LAYER_EXTRA_NAMES:
+                setattr(arr[n], name, ptr(lw[name], name))
+        out = ctypes.c_void_p()
+        _check(lib.mtla_stack_create(ctypes.byref(cfg), ctypes.byref(sc), arr,
+                                     ptr(weights["lnf_gamma"], "lnf_gamma"),
+                                     ptr(weights["lnf_beta"], "lnf_beta"), base, nbytes,
+                                     _stream_ptr(stream), ctypes.byref(out)), "mtla_stack_create")
+        torch.cuda.current_stream().synchronize()   # packing done: weight tensors may be freed
+    return Stack(out.value, cfg, n_layers, d_ff, arena, dtype, device)
+
+
+def mtla_stack_prefill(s: Stack, x: torch.Tensor, y: torch.Tensor | None = None, stream=None):
+    """x [B][T][d] on the device; returns the stack's output [B][T][d]."""
+    b, t, d = x.shape
+    _expect(x, s, (b, t, s.config.d_model), "x")
+    if y is None:
+        y = torch.empty_like(x)
+    _expect(y, s, x.shape, "y")
+    _check(load_library().mtla_stack_prefill(s.ptr, x.data_ptr(), b, t, y.data_ptr(),
+                                             _stream_ptr(stream)), "mtla_stack_prefill")
+    return y
+
+
+def mtla_stack_decode_step(s: Stack, x: torch.Tensor, y: torch.Tensor | None = None, stream=None):
+    """x [B][d] on the device; returns the stack's output [B][d]."""
+    b = x.shape[0]
+    _expect(x, s, (b, s.config.d_model), "x")
+    if y is None:
+        y = torch.empty_like(x)
+    _expect(y, s, x.shape, "y")
+    _check(load_library().mtla_stack_decode_step(s.ptr, x.data_ptr(), b, y.data_ptr(),
+                                                 _stream_ptr(stream)), "mtla_stack_decode_step")
+    return y
+
+
+def mtla_stack_cache_bytes(s: Stack) -> int:
+    return load_library().mtla_stack_cache_bytes(s.ptr)
+
+
+def mtla_stack_layer(s: Stack, layer: int) -> Handle:
+    """The attention handle of one layer, borrowed from the stack (never destroy it)."""
+    p = load_library().mtla_stack_layer(s.ptr, layer)
+    if not p:
+        raise MTLAError(-1, "mtla_stack_layer")
+    return Handle(p, s.config, s.arena, s.dtype, s.device)
+
+
+def mtla_stack_reset(s: Stack) -> None:
+    _check(load_library().mtla_stack_reset(s.ptr), "mtla_stack_reset")
+
+
+def mtla_stack_check(s: Stack, stream=None) -> None:
+    _check(load_library().mtla_stack_check(s.ptr, _stream_ptr(stream)), "mtla_stack_check")
+
+
+def mtla_stack_launch_count(s: Stack) -> int:
+    return load_library().mtla_stack_launch_count(s.ptr)
+
+
+def mtla_stack_destroy(s: Stack) -> None:
+    if s.ptr:
+        _check(load_library().mtla_stack_destroy(s.ptr), "mtla_stack_destroy")
+        s.ptr = 0

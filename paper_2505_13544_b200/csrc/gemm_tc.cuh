@@ -49,6 +49,13 @@ struct GemmTcArgs {
   int vec4_ok;                // 1: c_sm == 1, m % 4 == 0 and every column start is 16-byte aligned,
                               // so the split-K reduction may store four rows at once
   float alpha;
+  // Optional epilogue, applied to alpha * sum in this order (feed-forward block of a decoder
+  // layer): + bias[i] (one value per A row = output feature), ReLU, + residual[i * r_sm + j * r_sn]
+  // (fp32, may alias the output: every element is read and written by the same thread).
+  const float* bias;
+  const float* residual;
+  long long r_sm, r_sn;
+  int relu;
   float* partial;             // [tiles][n_split][BN][128] fp32 (split-K only)
   int* tickets;               // [tiles][4], zero between launches (split-K only)
   int* error_word;
@@ -117,6 +124,15 @@ __device__ __forceinline__ void store4(bf16* p, const float (&v)[4], long long l
     *reinterpret_cast<uint2*>(p + lo_off) = make_uint2(*reinterpret_cast<const uint32_t*>(&l0),
                                                        *reinterpret_cast<const uint32_t*>(&l1));
   }
+}
+
+// The finished value of output (i, j): scale, then the optional bias / ReLU / residual.
+__device__ __forceinline__ float finish(const GemmTcArgs& g, float acc, int i, int j) {
+  float v = g.alpha * acc;
+  if (g.bias) v += g.bias[i];
+  if (g.relu) v = fmaxf(v, 0.f);
+  if (g.residual) v += g.residual[(long long)i * g.r_sm + (long long)j * g.r_sn];
+  return v;
 }
 
 }  // namespace gtc
@@ -238,13 +254,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else {
 #pragma unroll
             for (int j = 0; j < CH; ++j)
-              if (j0 + j < g.n) put(p + j, g.alpha * __uint_as_float(v[j]));
+              if (j0 + j < g.n) put(p + j, finish(g, __uint_as_float(v[j]), i_row, j0 + j));
           }
         } else {
           OutT* p = c + (long long)i_row * g.c_sm;
 #pragma unroll
           for (int j = 0; j < CH; ++j)
-            if (j0 + j < g.n) put(p + (long long)(j0 + j) * g.c_sn, g.alpha * __uint_as_float(v[j]));
+            if (j0 + j < g.n)
+              put(p + (long long)(j0 + j) * g.c_sn, finish(g, __uint_as_float(v[j]), i_row, j0 + j));
         }
       };
       // Accumulator columns c0 .. c0 + CH of this thread's row (hi and lo products added).
@@ -324,15 +341,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int u = 0; u < U; ++u) {
               const int j = nt * BN + jb + u * 4 + cs;
               if (j >= g.n || i0 >= g.m) continue;
-              const float val[4] = {g.alpha * acc[u].x, g.alpha * acc[u].y, g.alpha * acc[u].z,
-                                    g.alpha * acc[u].w};
+              const float sum[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
               OutT* p = c + (long long)j * g.c_sn + (long long)i0 * g.c_sm;
               if (g.vec4_ok) {
+                const float val[4] = {g.alpha * sum[0], g.alpha * sum[1], g.alpha * sum[2], g.alpha * sum[3]};
                 store4(p, val, g.c_lo_off);
               } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                  if (i0 + e < g.m) put(p + (long long)e * g.c_sm, val[e]);
+                  if (i0 + e < g.m) put(p + (long long)e * g.c_sm, finish(g, sum[e], i0 + e, j));
               }
             }
           }

@@ -56,6 +56,7 @@ struct ArenaPlan {
   size_t page_table, seq_tokens;   // paged handles: two buffers each (beam reordering flips them)
   size_t p1, q16, qt, o_part, ml_part, o, v, x_stage, y_stage, gemm_part, gemm_tickets, attn_tickets;
   size_t pf_p1, pf_qcat, pf_cprime, pf_kr, pf_kv, pf_attn;
+  size_t scratch_begin;   // everything from here on is per-call scratch (nothing survives a call)
   size_t total;
 };
 
@@ -147,6 +148,7 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->page_table = take(paged * 2 * B * dm.max_pages * sizeof(int));
   p->seq_tokens = take(paged * 2 * B * sizeof(int));
   p->err_flag = take(16);
+  p->scratch_begin = off;
   p->p1 = take(B * dm.ntot * 4);
   p->q16 = take(B * 2 * hd * 2);
   p->qt = take(B * dm.nh * dm.W * 4);
@@ -200,6 +202,10 @@ struct mtla_handle {
   Dims dm;
   ArenaPlan plan;
   char* arena;
+  // Offsets at or beyond plan.scratch_begin resolve against this base instead of the arena
+  // (already shifted by -scratch_begin).  The layers of a stack share one scratch region:
+  // their calls are ordered on one stream and nothing in it survives a call.
+  char* scratch;
   int tokens;   // tokens consumed per sequence (paged handles: the longest sequence's)
   int batch;    // 0 while the cache is empty and no batch has been fixed
   // Paged handles (mtla_create_paged): per-sequence positions and the page pool.  The device
@@ -231,7 +237,9 @@ struct mtla_handle {
   int prof_used;
   bool prof_attention_only;   // record only the two events around the attention kernel
 
-  template <typename P> P* at(size_t off) const { return reinterpret_cast<P*>(arena + off); }
+  template <typename P> P* at(size_t off) const {
+    return reinterpret_cast<P*>((scratch && off >= plan.scratch_begin ? scratch : arena) + off);
+  }
   bool paged() const { return pool != nullptr; }
   int buf() const { return pool ? pool->current_buffer() : 0; }
   int* d_page_table(int which) const {
@@ -486,7 +494,9 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   // tile with the whole K range in flight at once beats splitting it, which costs a trip of the
   // partials through global memory on top of two load round trips.
   const bool shallow = allow_split && kb_total <= 8 && bn <= 64;
-  if (shallow) n_split = 1;
+  // Up to eight K blocks are never split, whatever the batch: the reduction's trip through
+  // global memory costs more than the shorter main loop saves.
+  if (shallow || kb_total <= 8) n_split = 1;
   g.kb_per_split = ceil_div(kb_total, n_split);
   g.n_split = ceil_div(kb_total, g.kb_per_split);
   g.partial = h->at<float>(h->plan.gemm_part);
@@ -498,6 +508,7 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   if ((long long)m_tiles * g.n_tiles * g.n_split > 0x7fffffffll) return MTLA_ERR_UNSUPPORTED_SHAPE;
   g.vec4_ok = g.c_sm == 1 && g.m % 4 == 0 && reinterpret_cast<uintptr_t>(g.c) % 16 == 0 &&
               g.c_sn * osz % 16 == 0 && g.c_sz * osz % 16 == 0 && g.c_lo_off * osz % 8 == 0;
+  if (g.bias || g.residual || g.relu) g.vec_ok = g.vec4_ok = 0;   // the epilogue extras are scalar
   // Enough work to fill the GPU: the persistent schedule.  Many tiles are dealt out whole; few
   // tiles with a long reduction (the decode step's weight streams) are cut anywhere.
   const long long total_kb = tiles * kb_total;
@@ -1189,7 +1200,7 @@ int run_prefill(mtla_handle* h, const void* x, int seq0, int B, int T, void* y, 
 }
 
 int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_weights* w, void* arena,
-                  size_t arena_bytes, void* stream, mtla_handle** out);
+                  size_t arena_bytes, void* stream, mtla_handle** out, void* shared_scratch = nullptr);
 
 }  // namespace
 
@@ -1228,8 +1239,10 @@ int mtla_create_paged(const mtla_config* cfg, const mtla_paging* paging, const m
 
 namespace {
 
+// With shared_scratch the arena holds only the persistent part (plan.scratch_begin bytes) and the
+// per-call scratch lives at shared_scratch (plan.total - plan.scratch_begin bytes, 1024-aligned).
 int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_weights* w, void* arena,
-                  size_t arena_bytes, void* stream, mtla_handle** out) {
+                  size_t arena_bytes, void* stream, mtla_handle** out, void* shared_scratch) {
   if (!cfg || !w || !arena || !out) return MTLA_ERR_INVALID_ARG;
   mtla_config c;
   Dims dm;
@@ -1241,10 +1254,11 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
   if (reinterpret_cast<uintptr_t>(arena) & 1023) return MTLA_ERR_INVALID_ARG;
   ArenaPlan p;
   plan_arena(c, dm, &p);
-  if (arena_bytes < p.total) return MTLA_ERR_ARENA_TOO_SMALL;
+  if (arena_bytes < (shared_scratch ? p.scratch_begin : p.total)) return MTLA_ERR_ARENA_TOO_SMALL;
   mtla_handle* h = new (std::nothrow) mtla_handle();
   if (!h) return MTLA_ERR_INVALID_ARG;
   h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
+  h->scratch = shared_scratch ? static_cast<char*>(shared_scratch) - p.scratch_begin : nullptr;
   h->tokens = 0; h->batch = 0; h->launches = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
@@ -1330,6 +1344,7 @@ void plan_baseline(const mtla_config& c, const Dims& dm, int groups, ArenaPlan* 
   p->rope_sin = take((size_t)c.max_tokens * (dm.dh / 2) * 4);
   p->cache = take(planes * dm.max_slots * dm.W * 2);
   p->err_flag = take(16);
+  p->scratch_begin = off;
   p->p1 = take(B * dm.ntot * 4);
   p->qt = take(planes * dm.nh * dm.W * 2);
   p->o_part = take((size_t)dm.max_units * dm.nh * dm.W * 4);
@@ -1467,6 +1482,7 @@ int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_we
   mtla_handle* h = new (std::nothrow) mtla_handle();
   if (!h) return MTLA_ERR_INVALID_ARG;
   h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
+  h->scratch = nullptr;
   h->tokens = 0; h->batch = 0; h->launches = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
@@ -1916,3 +1932,5 @@ const char* mtla_error_string(int status) {
 }
 
 }  // extern "C"
+
+#include "stack_api.inc"

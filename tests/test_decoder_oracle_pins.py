@@ -8,6 +8,7 @@ import torch
 from oracle import decoder_oracle as D
 from oracle import mtla_oracle as O
 from paper_2505_13544_b200 import synth
+from tests import helpers as H
 
 
 def small_stack(n_layers=3, stride=2, d_ff=96, seed=7):
@@ -19,18 +20,7 @@ def small_stack(n_layers=3, stride=2, d_ff=96, seed=7):
 
 
 def to_params(w, weights):
-    dims = dict(d_model=w.d_model, n_heads=w.n_heads, head_dim=w.head_dim, latent_rank=w.latent_rank,
-                rope_dim=w.rope_dim, hyper_dim=w.hyper_dim, stride=w.stride)
-    layers = []
-    for lw in weights["layers"]:
-        f = {k: v.double().numpy() for k, v in lw.items()}
-        attn = O.params_from_tensors(dims, {k: f[k] for k in (
-            "w_q", "w_qr", "w_r", "w_kr", "ln_gamma", "ln_beta", "w_k", "w_v", "w_o", "hyp_c_w",
-            "hyp_c_b", "hyp_pe_w", "hyp_pe_b")})
-        layers.append(D.LayerParams(attn=attn, **{k: f[k] for k in (
-            "ln1_gamma", "ln1_beta", "ln2_gamma", "ln2_beta", "w1", "b1", "w2", "b2")}))
-    return D.StackParams(layers=layers, lnf_gamma=weights["lnf_gamma"].double().numpy(),
-                         lnf_beta=weights["lnf_beta"].double().numpy())
+    return H.oracle_stack_params(synth.StackWorkload("pin", w, len(weights["layers"]), 0), weights)
 
 
 def torch_ln(x, gamma, beta):
