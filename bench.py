@@ -581,6 +581,103 @@ def time_decode(M, h, w: synth.Workload, device, steps: int, warmup: int) -> dic
             "attention_variant": M.mtla_attention_variant(h)}
 
 
+def stack_work(sw: synth.StackWorkload, n_slots: float) -> dict:
+    """Bytes and FLOP of one decode step of the stack: every layer's attention work plus its
+    feed-forward block (two d x d_ff matrices and their biases, the LayerNorm vectors)."""
+    w = sw.layer
+    e = 2 if w.dtype == "bf16" else 4
+    a = algorithmic_work(w, n_slots)
+    ffn_params = 2 * w.d_model * sw.d_ff + sw.d_ff + w.d_model + 4 * w.d_model
+    return {"weight_bytes": sw.n_layers * (a["weight_bytes"] + ffn_params * e),
+            "cache_bytes": sw.n_layers * a["cache_bytes"],
+            "flop": sw.n_layers * (a["attn_flop"] + a["proj_flop"] + 2 * w.batch * ffn_params)}
+
+
+def time_stack(sw: synth.StackWorkload, device, steps: int, warmup: int) -> dict:
+    """The decoder stack: parallel prefill of the prompt through every layer, then decode steps
+    (one token per sequence through all layers) with inputs resident."""
+    from paper_2505_13544_b200 import binding as M
+    w = sw.layer
+    weights = synth.make_stack_weights(sw)
+    cfg = M.make_config(**dims_of(w), max_batch=w.batch,
+                        max_tokens=w.prefill_tokens + steps + warmup + 8,
+                        max_prefill_tokens=w.prefill_tokens, dtype=w.dtype, ln_eps=w.ln_eps,
+                        rope_theta=w.rope_theta)
+    dev = {"layers": [{k: v.to(device) for k, v in lw.items()} for lw in weights["layers"]],
+           "lnf_gamma": weights["lnf_gamma"].to(device), "lnf_beta": weights["lnf_beta"].to(device)}
+    s = M.mtla_stack_create(cfg, sw.n_layers, sw.d_ff, dev, device=device)
+    x = fill_prompt(w, device)
+    y = torch.empty_like(x)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    for _ in range(3):
+        M.mtla_stack_reset(s)
+        torch.cuda.synchronize(device)
+        ev0.record()
+        M.mtla_stack_prefill(s, x, y)
+        ev1.record()
+        torch.cuda.synchronize(device)
+        times.append(ev0.elapsed_time(ev1))
+    M.mtla_stack_check(s)
+    assert torch.isfinite(y[:, -1].float()).all()
+    del x, y
+    prefill_ms = float(np.median(times[1:]))
+    dt = synth.torch_dtype(w.dtype)
+    xs = [synth.decode_input(w, i).to(device) for i in range(8)]
+    yd = torch.empty(w.batch, w.d_model, dtype=dt, device=device)
+    for i in range(warmup):
+        M.mtla_stack_decode_step(s, xs[i % 8], yd)
+    torch.cuda.synchronize(device)
+    l0 = M.mtla_stack_launch_count(s)
+    slots0 = M.mtla_position(M.mtla_stack_layer(s, 0))[1]
+    ev0.record()
+    for i in range(steps):
+        M.mtla_stack_decode_step(s, xs[i % 8], yd)
+    ev1.record()
+    torch.cuda.synchronize(device)
+    ms = ev0.elapsed_time(ev1) / steps
+    slots1 = M.mtla_position(M.mtla_stack_layer(s, 0))[1]
+    M.mtla_stack_check(s)
+    assert torch.isfinite(yd.float()).all()
+    launches = (M.mtla_stack_launch_count(s) - l0) / steps
+    cache_bytes = M.mtla_stack_cache_bytes(s)
+    M.mtla_stack_destroy(s)
+    peaks = measured_peaks()
+    work = stack_work(sw, 0.5 * (slots0 + 1 + slots1))
+    hbm_s = (work["weight_bytes"] + work["cache_bytes"]) / (peaks["hbm_gbs"] * 1e9)
+    tensor_s = work["flop"] / (peaks["bf16_tflops_sustained"] * 1e12)
+    return {"workload": sw.name, "n_layers": sw.n_layers, "d_ff": sw.d_ff, "batch": w.batch,
+            "d_model": w.d_model, "stride": w.stride, "prompt_tokens": w.prefill_tokens,
+            "prefill_ms": prefill_ms, "prefill_tokens_per_s": w.batch * w.prefill_tokens / (prefill_ms * 1e-3),
+            "decode_tokens_per_s": w.batch / (ms * 1e-3), "us_per_step": ms * 1e3,
+            "context_slots": [slots0, slots1], "launches_per_step": launches,
+            "roofline_us": max(hbm_s, tensor_s) * 1e6,
+            "step_roofline_frac": max(hbm_s, tensor_s) / (ms * 1e-3),
+            "cache_bytes": cache_bytes,
+            "note": "a step is one token per sequence through all layers; weights and caches of this "
+                    "model fit L2, so the step is bound by kernel latency, not by HBM"}
+
+
+def stack_cpu_baseline(sw: synth.StackWorkload, budget_s: float = 10.0) -> dict:
+    """The decoder oracle's decode step, as it stands, on one sequence after the full prompt."""
+    from oracle import decoder_oracle as D
+    from tests import helpers as H
+    from threadpoolctl import threadpool_info
+    w = sw.layer
+    sp = H.oracle_stack_params(sw, synth.make_stack_weights(sw))
+    prompt = synth.stored(synth.normal(w.seed, "prompt/0", (w.prefill_tokens, w.d_model)), w.dtype)
+    _, st = D.stack_forward_by_layers(sp, prompt.double().numpy(), rows=[])
+    n, t0 = 0, time.perf_counter()
+    while n < 64 and time.perf_counter() - t0 < budget_s:
+        D.stack_decode_step(sp, st, synth.decode_input(w, n, batch=1)[0].double().numpy())
+        n += 1
+    el = time.perf_counter() - t0
+    cores = max([int(i.get("num_threads", 1)) for i in threadpool_info()] + [1])
+    return {"value": n / el, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"1 of {w.batch} sequences x {n} decode steps through {sw.n_layers} layers after a "
+                      f"{w.prefill_tokens}-token prompt, {el:.1f} s"}
+
+
 def run_other_configs(device, steps: int = 64, warmup: int = 8):
     """The other benchmark configurations, each for a fraction of a second: the parallel prefill
     of the long-context workload against the tensor roofline, and decode steps of every
@@ -648,7 +745,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--workload", default="large",
-                    choices=sorted(synth.WORKLOADS) + sorted(synth.BEAM_WORKLOADS))
+                    choices=sorted(synth.WORKLOADS) + sorted(synth.BEAM_WORKLOADS)
+                    + sorted(synth.STACK_WORKLOADS))
     ap.add_argument("--compare", action="store_true",
                     help="time MHA / GQA / MQA / MLA / MTLA at the workload's width, batch and one context")
     ap.add_argument("--paged", action="store_true",
@@ -665,7 +763,7 @@ def main() -> None:
                     help="override the workload's imported context length")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload in synth.BEAM_WORKLOADS:
+        if args.workload in synth.BEAM_WORKLOADS or args.workload in synth.STACK_WORKLOADS:
             raise SystemExit("--impl reference covers the decode workloads")
         run_reference(args)
         return
@@ -695,6 +793,25 @@ def main() -> None:
         if world > 1:
             raise SystemExit("the beam workloads run on one GPU")
         run_beam(args, synth.BEAM_WORKLOADS[args.workload], device, local)
+        return
+    if args.workload in synth.STACK_WORKLOADS:
+        if world > 1:
+            raise SystemExit("the decoder-stack workload runs on one GPU")
+        sw = synth.STACK_WORKLOADS[args.workload]
+        with ClockSampler(local) as clocks:
+            res = time_stack(sw, device, steps=args.steps, warmup=max(args.warmup, 3))
+        line = {"metric": METRIC, "value": res["decode_tokens_per_s"], "unit": UNIT, "n_gpus": 1,
+                "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": res["us_per_step"] * 1e-3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if sw.layer.dtype == "bf16" else "f32", "data": "synthetic",
+                "config": {"workload": sw.name, "batch": sw.layer.batch, "n_layers": sw.n_layers,
+                           "d_model": sw.layer.d_model, "d_ff": sw.d_ff, "stride": sw.layer.stride,
+                           "l2": "weights and caches fit L2: latency-bound, bandwidth figures are effective"},
+                "decoder": res, "gpu_launches": int(round(res["launches_per_step"] * args.steps)),
+                "clocks": clocks.summary()}
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = stack_cpu_baseline(sw)
+        print(json.dumps(line))
         return
     w = pick_workload(args)
     K, W = args.steps, max(args.warmup, 3)
@@ -828,6 +945,7 @@ def main() -> None:
     torch.cuda.empty_cache()
     if world == 1 and args.workload == "large" and not args.no_other_configs and not args.batch:
         line["prefill"], line["configs"] = run_other_configs(device)
+        line["decoder"] = time_stack(synth.STACK_WORKLOADS["decoder_paper"], device, steps=64, warmup=8)
     if world == 1 and not args.no_cpu_baseline:
         n_seq = 1 if w.batch * w.latent_rank >= 8192 else min(w.batch, 4)
         res = oracle_decode_sample(w, n_seq, budget_s=12.0, max_steps=64)

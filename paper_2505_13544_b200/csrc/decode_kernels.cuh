@@ -201,6 +201,143 @@ __global__ void __launch_bounds__(256) decode_post_kernel(PostArgs a) {
   if (a.seq_tokens && tid == 0) a.seq_tokens[b] = i0 + 1;
 }
 
+// The same step for layers whose gate needs no matrix (the folded form, or s = 1 where w = 1),
+// laid out for latency: warp 0 alone carries the dependent chain of a sequence (latent row ->
+// LayerNorm by shuffles -> gate -> slot row), everything it touches moving as 16-byte vectors,
+// while warps 1-7 convert the queries (bf16 hi / lo halves for the tensor-core absorption) and
+// rotate the RoPE queries, which depend on nothing but the projection row.  No block-wide
+// barrier is needed.  One CTA of 256 threads per sequence; r <= 512.
+template <typename T, typename TQ>
+__global__ void __launch_bounds__(256) decode_post_fast_kernel(PostArgs a) {
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* row = a.p1 + (long long)b * a.proj.width;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();   // the projection kernel's output is read from here on
+  const int i0 = a.seq_tokens ? a.seq_tokens[b] : a.tokens;
+  const int slot = i0 / a.stride;
+  const bool new_slot = i0 % a.stride == 0;
+  const int half = a.dr / 2, W = a.r + a.dr;
+  const float* rope_cos = a.rope_cos + (long long)i0 * half;
+  const float* rope_sin = a.rope_sin + (long long)i0 * half;
+  if (warp == 0) {
+    // Latent: lane l holds elements 128 v + 4 l .. + 3 of the row, v < ceil(r / 128).
+    float c[4][4];
+    float sum = 0.f;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const int i = v * 128 + lane * 4;
+      const float4 x4 = i < a.r ? *reinterpret_cast<const float4*>(row + a.proj.off_c + i)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+      c[v][0] = x4.x; c[v][1] = x4.y; c[v][2] = x4.z; c[v][3] = x4.w;
+      sum += (x4.x + x4.y) + (x4.z + x4.w);
+    }
+    // The other inputs of the chain are requested before the first reduction.
+    float uu[8], gss[8], gtt[8], gpp[8];
+    const float* gate_pe = a.gate_pe + (long long)slot * a.dw;
+    if (a.use_gate) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int n = k * 32 + lane;
+        const bool in = n < a.dw;
+        uu[k] = in ? row[a.proj.off_u + n] + row[a.proj.off_u + a.dw + n] : 0.f;
+        gss[k] = in ? a.gate_s[n] : 0.f;
+        gtt[k] = in ? a.gate_t[n] : 0.f;
+        gpp[k] = in ? gate_pe[n] : 0.f;
+      }
+    }
+    float acc_old[4][4];
+    float* acc = a.open_acc + (long long)b * a.r;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const int i = v * 128 + lane * 4;
+      const float4 o4 = (!new_slot && i < a.r) ? *reinterpret_cast<const float4*>(acc + i)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+      acc_old[v][0] = o4.x; acc_old[v][1] = o4.y; acc_old[v][2] = o4.z; acc_old[v][3] = o4.w;
+    }
+    const float mean = warp_sum(sum) / a.r;
+    float sq = 0.f;
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float d = (v * 128 + lane * 4 + e < a.r) ? c[v][e] - mean : 0.f;
+        sq += d * d;
+      }
+    const float rstd = rsqrtf(warp_sum(sq) / a.r + a.ln_eps);
+    float w = 1.f;
+    if (a.use_gate) {
+      float prod = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) prod += (rstd * (uu[k] - mean * gss[k]) + gtt[k]) * gpp[k];
+      w = 1.f / (1.f + expf(-warp_sum(prod)));
+    }
+    T* slot_row = static_cast<T*>(a.cache.base) + cache_row(a.cache, b, slot) * W;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const int i = v * 128 + lane * 4;
+      if (i >= a.r) continue;
+      const float4 g4 = *reinterpret_cast<const float4*>(a.gamma + i);
+      const float4 b4 = *reinterpret_cast<const float4*>(a.beta + i);
+      const float gam[4] = {g4.x, g4.y, g4.z, g4.w}, bet[4] = {b4.x, b4.y, b4.z, b4.w};
+      float val[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        val[e] = acc_old[v][e] + w * ((c[v][e] - mean) * rstd * gam[e] + bet[e]);
+      *reinterpret_cast<float4*>(acc + i) = make_float4(val[0], val[1], val[2], val[3]);
+      if (sizeof(T) == 2) {
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(val[0], val[1]), h1 = __floats2bfloat162_rn(val[2], val[3]);
+        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(slot_row) + i) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+      } else {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(slot_row) + i) =
+            make_float4(val[0], val[1], val[2], val[3]);
+      }
+    }
+    // RoPE key of this token replaces the slot's key (pairs 2k, 2k + 1; d_R / 2 <= 32 pairs).
+    if (lane < half) {
+      const float2 x2 = *reinterpret_cast<const float2*>(row + a.proj.off_kr + 2 * lane);
+      const float cs = rope_cos[lane], sn = rope_sin[lane];
+      const float y0 = x2.x * cs - x2.y * sn, y1 = x2.x * sn + x2.y * cs;
+      if (sizeof(T) == 2)
+        *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<bf16*>(slot_row) + a.r + 2 * lane) =
+            __floats2bfloat162_rn(y0, y1);
+      else
+        *reinterpret_cast<float2*>(reinterpret_cast<float*>(slot_row) + a.r + 2 * lane) = make_float2(y0, y1);
+    }
+    if (a.seq_tokens && lane == 0) a.seq_tokens[b] = i0 + 1;
+    return;
+  }
+  // Warps 1-7: queries.  bf16 [hi | lo] halves of q, four elements per thread and step.
+  const int t = tid - 32;
+  if (a.q16) {
+    const int hd = a.n_heads * a.head_dim;
+    bf16* dst = a.q16 + (long long)b * 2 * hd;
+    for (int i = t * 4; i < hd; i += 224 * 4) {
+      const float4 q4 = *reinterpret_cast<const float4*>(row + a.proj.off_q + i);
+      const __nv_bfloat162 h0 = __floats2bfloat162_rn(q4.x, q4.y), h1 = __floats2bfloat162_rn(q4.z, q4.w);
+      const __nv_bfloat162 l0 = __floats2bfloat162_rn(q4.x - __low2float(h0), q4.y - __high2float(h0));
+      const __nv_bfloat162 l1 = __floats2bfloat162_rn(q4.z - __low2float(h1), q4.w - __high2float(h1));
+      *reinterpret_cast<uint2*>(dst + i) =
+          make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+      *reinterpret_cast<uint2*>(dst + hd + i) =
+          make_uint2(*reinterpret_cast<const uint32_t*>(&l0), *reinterpret_cast<const uint32_t*>(&l1));
+    }
+  }
+  // Rotated, pre-scaled RoPE queries behind the (separately computed) absorbed query.
+  TQ* qt = static_cast<TQ*>(a.qt) + (long long)b * a.n_heads * W;
+  for (int i = t; i < a.n_heads * half; i += 224) {
+    const int h = i / half, k = i % half;
+    const float2 x2 = *reinterpret_cast<const float2*>(row + a.proj.off_qr + h * a.dr + 2 * k);
+    const float cs = rope_cos[k], sn = rope_sin[k];
+    const float y0 = (x2.x * cs - x2.y * sn) * a.q_scale, y1 = (x2.x * sn + x2.y * cs) * a.q_scale;
+    if (sizeof(TQ) == 2)
+      *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<bf16*>(qt) + h * W + a.r + 2 * k) =
+          __floats2bfloat162_rn(y0, y1);
+    else
+      *reinterpret_cast<float2*>(reinterpret_cast<float*>(qt) + h * W + a.r + 2 * k) = make_float2(y0, y1);
+  }
+}
+
 struct AttnArgs {
   const void* qt;      // [B][n_h][r + d_R], pre-scaled by log2(e)/sqrt(d_h)
   CacheView cache;

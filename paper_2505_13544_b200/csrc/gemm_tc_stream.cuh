@@ -10,8 +10,7 @@
 //     deep TMA ring that never drains between tiles.  A share that ends inside a tile leaves a
 //     partial accumulator in a workspace; the CTA that delivers a tile's last partial sums them
 //     in share order (an atomic ticket per 32-row quarter, never a wait), so the result does
-//     not depend on arrival order.  A CTA that finds all other parts delivered keeps its own
-//     part in tensor memory and sums straight away;
+//     not depend on arrival order;
 //   * many tiles (the prefill's projections): shares are cut at tile boundaries, nothing is
 //     partial, and the CTA simply runs tile after tile.
 //
@@ -275,85 +274,84 @@ gemm_tc_stream_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(&bars->acc_empty[acc]));
       } else {
-        // A partial.  Slots of one tile's parts are consecutive in the workspace and in share
-        // order (first owner + tile, ...); each 32-row quarter has its own ticket, so the four
-        // epilogue warps go their own ways.
+        // A partial: to the workspace slot of (this CTA, this tile), then a ticket.  Slots of one
+        // tile's parts are consecutive and in share order: first owner + tile, ...
+        float* part = s.parts + ((long long)blockIdx.x + tile) * (long long)(BN * kBM);
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += CH) {
+          uint32_t v[32];
+          load_acc(c0, v);
+#pragma unroll
+          for (int j = 0; j < CH; ++j) part[(c0 + j) * kBM + row_local] = __uint_as_float(v[j]);
+        }
+        // The accumulator is in the workspace: the issuer may reuse the buffer while this warp
+        // goes on to the ticket and, if it is the last, the sum.
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(&bars->acc_empty[acc]));
         const long long k_first = tile * kb_total;
         const long long c_first = share_owner(k_first, total, G);
         const int n_parts = (int)(share_owner(k_first + kb_total - 1, total, G) - c_first) + 1;
-        const int mine = (int)(blockIdx.x - c_first);
-        int* ticket = g.tickets + tile * 4 + q;
-        // If every other part has been delivered already, this warp is the one that sums: its
-        // own part then never leaves tensor memory.
-        int state = 0;                                  // 1: last, own part still in TMEM
-        if (lane == 0) state = *reinterpret_cast<volatile int*>(ticket) == n_parts - 1 ? 1 : 0;
-        state = __shfl_sync(0xffffffffu, state, 0);
-        if (!state) {
-          float* part = s.parts + ((long long)blockIdx.x + tile) * (long long)(BN * kBM);
-#pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += CH) {
-            uint32_t v[32];
-            load_acc(c0, v);
-#pragma unroll
-            for (int j = 0; j < CH; ++j) part[(c0 + j) * kBM + row_local] = __uint_as_float(v[j]);
-          }
-          // The accumulator is in the workspace: the issuer may reuse the buffer.
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(&bars->acc_empty[acc]));
-          __threadfence();
-          __syncwarp();
-          if (lane == 0) state = atomicAdd(ticket, 1) == n_parts - 1 ? 2 : 0;   // 2: last after all
-          state = __shfl_sync(0xffffffffu, state, 0);
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+          int* ticket = g.tickets + tile * 4 + q;
+          last = atomicAdd(ticket, 1) == n_parts - 1;
+          if (last) *ticket = 0;               // every other part has already arrived
         }
-        if (state) {
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
           __threadfence();
-          // Sum over the parts in share order, 32 columns at a time in the accumulator's own
-          // layout (thread = row, so a warp's load of one column of one part is 128 contiguous
-          // bytes), three parts' loads in flight per thread, then the ordinary epilogue.
-          const float* all = s.parts + (c_first + tile) * (long long)(BN * kBM) + row_local;
-          constexpr int P = 3;
+          // This warp sums its 32-row quarter over the parts, in share order.  Lane l owns rows
+          // 4*(l%8)..+3 of column (l/8) in each group of four columns: every load is a 16-byte
+          // vector and a warp instruction covers 512 contiguous bytes.  The sum is bound by the
+          // L2 round trip, so as many loads as the registers hold are in flight: U column groups
+          // of up to four parts at a time.
+          const float* all = s.parts + (c_first + tile) * (long long)(BN * kBM) + q * 32;
+          const int r4 = 4 * (lane & 7), cs = lane >> 3;
+          constexpr int U = BN >= 32 ? 8 : 4;           // column groups per step (BN / 4 >= U)
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += CH) {
-            uint32_t own[32];
-            if (state == 1) load_acc(c0, own);
-            float sum[32];
+          for (int jb = 0; jb < BN; jb += 4 * U) {
+            float4 accv[U];
 #pragma unroll
-            for (int j = 0; j < CH; ++j) sum[j] = 0.f;
+            for (int u = 0; u < U; ++u) accv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-            for (int p0 = 0; p0 < n_parts; p0 += P) {
-              float t[P][32];
+            for (int sp0 = 0; sp0 < n_parts; sp0 += 4) {
+              float4 t[4][U];
 #pragma unroll
-              for (int u = 0; u < P; ++u) {
-                const int pt = p0 + u;
-                const bool from_mem = pt < n_parts && !(state == 1 && pt == mine);
+              for (int s4 = 0; s4 < 4; ++s4)
 #pragma unroll
-                for (int j = 0; j < CH; ++j)
-                  t[u][j] = from_mem ? __ldcg(all + (long long)pt * (BN * kBM) + (c0 + j) * kBM) : 0.f;
-              }
+                for (int u = 0; u < U; ++u)
+                  t[s4][u] = sp0 + s4 < n_parts
+                                 ? __ldcg(reinterpret_cast<const float4*>(
+                                       all + (long long)(sp0 + s4) * (BN * kBM) +
+                                       (jb + u * 4 + cs) * kBM + r4))
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-              for (int u = 0; u < P; ++u) {
-                const int pt = p0 + u;
-                if (pt >= n_parts) break;
-                if (state == 1 && pt == mine) {
+              for (int s4 = 0; s4 < 4; ++s4)
 #pragma unroll
-                  for (int j = 0; j < CH; ++j) sum[j] += __uint_as_float(own[j]);
-                } else {
-#pragma unroll
-                  for (int j = 0; j < CH; ++j) sum[j] += t[u][j];
+                for (int u = 0; u < U; ++u) {
+                  accv[u].x += t[s4][u].x; accv[u].y += t[s4][u].y;
+                  accv[u].z += t[s4][u].z; accv[u].w += t[s4][u].w;
                 }
+            }
+            const int i0 = mt * kBM + q * 32 + r4;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              const int j = nt * BN + jb + u * 4 + cs;
+              if (j >= g.n || i0 >= g.m) continue;
+              const float sum[4] = {accv[u].x, accv[u].y, accv[u].z, accv[u].w};
+              OutT* p = c + (long long)j * g.c_sn + (long long)i0 * g.c_sm;
+              if (g.vec4_ok) {
+                const float val[4] = {g.alpha * sum[0], g.alpha * sum[1], g.alpha * sum[2], g.alpha * sum[3]};
+                gtc::store4(p, val, g.c_lo_off);
+              } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (i0 + e < g.m) put(p + (long long)e * g.c_sm, gtc::finish(g, sum[e], i0 + e, j));
               }
             }
-            uint32_t v[32];
-#pragma unroll
-            for (int j = 0; j < CH; ++j) v[j] = __float_as_uint(sum[j]);
-            emit(v, c0);
-          }
-          if (lane == 0) *ticket = 0;                   // every part has arrived: ready for the next launch
-          if (state == 1) {
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(&bars->acc_empty[acc]));
           }
         }
       }

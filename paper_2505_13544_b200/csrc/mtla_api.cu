@@ -494,9 +494,7 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   // tile with the whole K range in flight at once beats splitting it, which costs a trip of the
   // partials through global memory on top of two load round trips.
   const bool shallow = allow_split && kb_total <= 8 && bn <= 64;
-  // Up to eight K blocks are never split, whatever the batch: the reduction's trip through
-  // global memory costs more than the shorter main loop saves.
-  if (shallow || kb_total <= 8) n_split = 1;
+  if (shallow) n_split = 1;
   g.kb_per_split = ceil_div(kb_total, n_split);
   g.n_split = ceil_div(kb_total, g.kb_per_split);
   g.partial = h->at<float>(h->plan.gemm_part);
@@ -514,8 +512,14 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   const long long total_kb = tiles * kb_total;
   if (tiles >= 2ll * h->sm_count)
     return gemm_tc_stream<OutT>(h, ma, mb, g, bn, batches, true, hilo, h->sm_count, st, dependent);
-  if (allow_split && total_kb >= 4ll * h->sm_count)
-    return gemm_tc_stream<OutT>(h, ma, mb, g, bn, batches, false, hilo, h->sm_count, st, dependent);
+  if (allow_split && total_kb >= 4ll * h->sm_count) {
+    // Few tiles: every tile is cut into the same number of parts, so that no share crosses a
+    // tile boundary and the sum at the end reads as few partials as possible.  More tiles than
+    // SMs: equal shares that end wherever they end.
+    int grid = h->sm_count;
+    if (tiles <= h->sm_count) grid = (int)tiles * max(1, min((int)(h->sm_count / tiles), kb_total / 4));
+    return gemm_tc_stream<OutT>(h, ma, mb, g, bn, batches, false, hilo, grid, st, dependent);
+  }
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
   if (shallow && (sizeof(OutT) == 4 || hilo)) {
@@ -799,10 +803,16 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   // On the tensor-core path every kernel after the first is a programmatic dependent launch:
   // its prologue overlaps the tail of its predecessor (not while events sit between them).
   const bool pdl = h->use_tc && !(prof && !h->prof_attention_only);
+  // Layers whose gate needs no matrix (folded form, or s = 1) take the latency-oriented kernel.
+  const bool post_fast = dm.proj.off_u >= 0 || !pa.use_gate;
   if (h->use_tc) {
-    MTLA_CUDA(launch_kernel(decode_post_kernel<T, bf16>, dim3(B), dim3(256), 0, st, pdl, pa));
+    if (post_fast)
+      MTLA_CUDA(launch_kernel(decode_post_fast_kernel<T, bf16>, dim3(B), dim3(256), 0, st, pdl, pa));
+    else
+      MTLA_CUDA(launch_kernel(decode_post_kernel<T, bf16>, dim3(B), dim3(256), 0, st, pdl, pa));
   } else {
-    decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
+    if (post_fast) decode_post_fast_kernel<T, float><<<B, 256, 0, st>>>(pa);
+    else decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
     MTLA_CUDA(cudaGetLastError());
   }
   h->launches++;

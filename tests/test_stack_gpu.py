@@ -40,7 +40,7 @@ def run_stack(sw, seqs=None, prefill_rows=None, steps_checked=None):
         for b in seqs:
             want, st = D.stack_forward_by_layers(sp, prompts[b].double().numpy(), rows=prefill_rows)
             got = y[b] if prefill_rows is None else y[b, prefill_rows]
-            H.assert_close(got, want, w.dtype, f"prefill seq {b}")
+            H.assert_close_stack(got, want, w.dtype, sw.n_layers, f"prefill seq {b}")
             states[b] = st
         slots = math.ceil(w.prefill_tokens / w.stride)
         elem = 4 if w.dtype == "fp32" else 2
@@ -51,7 +51,7 @@ def run_stack(sw, seqs=None, prefill_rows=None, steps_checked=None):
             check = steps_checked is None or i in steps_checked
             want = [D.stack_decode_step(sp, states[b], x[b].double().numpy()) for b in seqs]
             if check:
-                H.assert_close(yd[seqs], np.stack(want), w.dtype, f"decode step {i}")
+                H.assert_close_stack(yd[seqs], np.stack(want), w.dtype, sw.n_layers, f"decode step {i}")
         M.mtla_stack_check(s)
         tokens = w.prefill_tokens + w.decode_steps
         for n in range(sw.n_layers):
@@ -59,7 +59,7 @@ def run_stack(sw, seqs=None, prefill_rows=None, steps_checked=None):
             assert M.mtla_position(layer) == (tokens, math.ceil(tokens / w.stride), w.batch)
             cache = M.mtla_cache_export(layer)
             H.assert_cache_close(cache[seqs], np.stack([O.cache_array(states[b].layers[n]) for b in seqs]),
-                                 w.dtype)
+                                 w.dtype, scale=math.sqrt(n + 1))
     finally:
         M.mtla_stack_destroy(s)
 
@@ -104,7 +104,7 @@ def test_decode_from_empty_and_errors():
             y = M.mtla_stack_decode_step(s, x.cuda())
             want = np.stack([D.stack_decode_step(sp, states[b], x[b].double().numpy())
                              for b in range(w.batch)])
-            H.assert_close(y, want, "bf16", f"step {i}")
+            H.assert_close_stack(y, want, "bf16", 2, f"step {i}")
         with pytest.raises(M.MTLAError) as e:
             M.mtla_stack_decode_step(s, synth.decode_input(w, 0).cuda())   # max_tokens reached
         assert e.value.status == -4
