@@ -16,7 +16,6 @@
 #include "decode_kernels.cuh"
 #include "gemm_fma.cuh"
 #include "gemm_tc.cuh"
-#include "gemm_tc_stream.cuh"
 #include "prefill_attn_tc.cuh"
 #include "prefill_attn_tc2.cuh"
 #include "prefill_kernels.cuh"
@@ -38,8 +37,7 @@ constexpr int kMinSlotsPerSplit = 64;
 constexpr int kFusedCombineMaxParts = 8;   // more parts per sequence: the combine gets its own launch
 constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill projections
 constexpr int kGemmSlots = 2 * kPlanSms;   // CTAs a split-K GEMM may spread one product over
-constexpr int kGemmParts = 3 * kPlanSms;   // partial accumulators of the persistent GEMM: one per
-                                           // CTA plus one per tile, at most 2 * SMs tiles
+
 
 // Rows of the activation-side TMA box (the MMA's N) for a decode batch of B sequences.
 int act_box_rows(int B) {
@@ -160,7 +158,7 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->y_stage = take(B * dm.d * e);
   // Split-K workspace of the tensor-core GEMMs: at most kGemmSlots CTAs hold a partial tile.
   p->gemm_part = take(c.dtype == MTLA_DTYPE_BF16
-                          ? (size_t)kGemmParts * gtc::kBM * act_box_rows(c.max_batch) * 4 : 0);
+                          ? (size_t)kGemmSlots * gtc::kBM * act_box_rows(c.max_batch) * 4 : 0);
   p->gemm_tickets = take((size_t)kGemmSlots * 4 * sizeof(int));
   p->attn_tickets = take(B * sizeof(int));
   const size_t rows = B * (size_t)c.max_prefill_tokens;
@@ -231,7 +229,6 @@ struct mtla_handle {
   CUtensorMap map_q16, map_o16, map_v16;
   int act_bn;               // box rows the three activation maps were encoded with (0: none yet)
   unsigned gemm_attr_mask;  // kernel instances whose shared-memory limit has been raised
-  unsigned stream_attr_mask;
   // Optional timing of the decode step's kernels: MTLA_DECODE_STAGES + 1 events per profiled step.
   std::vector<cudaEvent_t> prof_events;
   int prof_used;
@@ -418,61 +415,6 @@ int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const C
   return MTLA_OK;
 }
 
-template <int BN, typename OutT, bool HILO>
-int launch_gemm_stream_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
-                            const GemmStreamArgs& s, int grid, cudaStream_t st, bool dependent) {
-  constexpr int smem = gts::smem_bytes(HILO ? 2 * BN : BN);
-  if (!(h->stream_attr_mask & (1u << inst))) {
-    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_stream_kernel<BN, OutT, HILO>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    h->stream_attr_mask |= 1u << inst;
-  }
-  MTLA_CUDA(launch_kernel(gemm_tc_stream_kernel<BN, OutT, HILO>, dim3(grid), dim3(192), smem, st,
-                          dependent, ma, mb, s));
-  h->launches++;
-  return MTLA_OK;
-}
-
-// The persistent schedule (gemm_tc_stream.cuh) for products with enough work to fill the GPU.
-template <typename OutT>
-int gemm_tc_stream(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, const GemmTcArgs& g,
-                   int bn, int batches, bool whole_tiles, bool hilo, int grid, cudaStream_t st,
-                   bool dependent) {
-  GemmStreamArgs s;
-  s.g = g;
-  s.batches = batches;
-  s.whole_tiles = whole_tiles ? 1 : 0;
-  s.parts = h->at<float>(h->plan.gemm_part);
-  if constexpr (sizeof(OutT) == 4) {
-    switch (bn) {
-      case 16: return launch_gemm_stream_inst<16, OutT, false>(h, 0, ma, mb, s, grid, st, dependent);
-      case 32: return launch_gemm_stream_inst<32, OutT, false>(h, 1, ma, mb, s, grid, st, dependent);
-      case 64: return launch_gemm_stream_inst<64, OutT, false>(h, 2, ma, mb, s, grid, st, dependent);
-      case 128: return launch_gemm_stream_inst<128, OutT, false>(h, 3, ma, mb, s, grid, st, dependent);
-      case 256: return launch_gemm_stream_inst<256, OutT, false>(h, 4, ma, mb, s, grid, st, dependent);
-      default: return MTLA_ERR_UNSUPPORTED_SHAPE;
-    }
-  } else {
-    if (hilo) {
-      switch (bn) {
-        case 16: return launch_gemm_stream_inst<16, OutT, true>(h, 5, ma, mb, s, grid, st, dependent);
-        case 32: return launch_gemm_stream_inst<32, OutT, true>(h, 6, ma, mb, s, grid, st, dependent);
-        case 64: return launch_gemm_stream_inst<64, OutT, true>(h, 7, ma, mb, s, grid, st, dependent);
-        case 128: return launch_gemm_stream_inst<128, OutT, true>(h, 8, ma, mb, s, grid, st, dependent);
-        default: return MTLA_ERR_UNSUPPORTED_SHAPE;
-      }
-    }
-    switch (bn) {
-      case 16: return launch_gemm_stream_inst<16, OutT, false>(h, 9, ma, mb, s, grid, st, dependent);
-      case 32: return launch_gemm_stream_inst<32, OutT, false>(h, 10, ma, mb, s, grid, st, dependent);
-      case 64: return launch_gemm_stream_inst<64, OutT, false>(h, 11, ma, mb, s, grid, st, dependent);
-      case 128: return launch_gemm_stream_inst<128, OutT, false>(h, 12, ma, mb, s, grid, st, dependent);
-      case 256: return launch_gemm_stream_inst<256, OutT, false>(h, 13, ma, mb, s, grid, st, dependent);
-      default: return MTLA_ERR_UNSUPPORTED_SHAPE;
-    }
-  }
-}
-
 // D[z][i][j] = alpha * sum_k A[z][i][k] B[z][j][k] on the tensor cores (see gemm_tc.cuh).
 // `bn` is the row count of map_b's box.  With allow_split the reduction is spread over
 // several CTAs when the tile count alone would leave most SMs idle.
@@ -507,19 +449,6 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   g.vec4_ok = g.c_sm == 1 && g.m % 4 == 0 && reinterpret_cast<uintptr_t>(g.c) % 16 == 0 &&
               g.c_sn * osz % 16 == 0 && g.c_sz * osz % 16 == 0 && g.c_lo_off * osz % 8 == 0;
   if (g.bias || g.residual || g.relu) g.vec_ok = g.vec4_ok = 0;   // the epilogue extras are scalar
-  // Enough work to fill the GPU: the persistent schedule.  Many tiles are dealt out whole; few
-  // tiles with a long reduction (the decode step's weight streams) are cut anywhere.
-  const long long total_kb = tiles * kb_total;
-  if (tiles >= 2ll * h->sm_count)
-    return gemm_tc_stream<OutT>(h, ma, mb, g, bn, batches, true, hilo, h->sm_count, st, dependent);
-  if (allow_split && total_kb >= 4ll * h->sm_count) {
-    // Few tiles: every tile is cut into the same number of parts, so that no share crosses a
-    // tile boundary and the sum at the end reads as few partials as possible.  More tiles than
-    // SMs: equal shares that end wherever they end.
-    int grid = h->sm_count;
-    if (tiles <= h->sm_count) grid = (int)tiles * max(1, min((int)(h->sm_count / tiles), kb_total / 4));
-    return gemm_tc_stream<OutT>(h, ma, mb, g, bn, batches, false, hilo, grid, st, dependent);
-  }
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
   if (shallow && (sizeof(OutT) == 4 || hilo)) {
@@ -1275,7 +1204,6 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
   h->prof_attention_only = false;
   h->act_bn = 0;
   h->gemm_attr_mask = 0;
-  h->stream_attr_mask = 0;
   h->pool = nullptr;
   h->tokens_stale = false;
   h->is_baseline = false;
@@ -1361,7 +1289,7 @@ void plan_baseline(const mtla_config& c, const Dims& dm, int groups, ArenaPlan* 
   p->ml_part = take((size_t)dm.max_units * dm.nh * 2 * 4);
   p->o = take(planes * 2 * dm.nh * dm.W * 2);
   p->v = take(B * 2 * hd * 2);
-  p->gemm_part = take((size_t)kGemmParts * gtc::kBM * act_box_rows(c.max_batch) * 4);
+  p->gemm_part = take((size_t)kGemmSlots * gtc::kBM * act_box_rows(c.max_batch) * 4);
   p->gemm_tickets = take((size_t)kGemmSlots * 4 * sizeof(int));
   p->attn_tickets = take(planes * sizeof(int));
   p->total = off;
@@ -1499,7 +1427,6 @@ int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_we
   h->prof_attention_only = false;
   h->act_bn = 0;
   h->gemm_attr_mask = 0;
-  h->stream_attr_mask = 0;
   h->pool = nullptr;
   h->tokens_stale = false;
   h->is_baseline = true;

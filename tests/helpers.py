@@ -89,3 +89,36 @@ def assert_cache_close(got: torch.Tensor, want: np.ndarray, dtype: str, scale: f
         assert np.abs(g - want).max() <= FP32_MAX_ABS * scale
     else:
         assert (np.abs(g - want) <= scale * 2.0 ** -7 * (1.0 + np.abs(want))).all()
+
+
+ATTN_WEIGHT_NAMES = ("w_q", "w_qr", "w_r", "w_kr", "ln_gamma", "ln_beta", "w_k", "w_v", "w_o",
+                     "hyp_c_w", "hyp_c_b", "hyp_pe_w", "hyp_pe_b")
+LAYER_EXTRA_NAMES = ("ln1_gamma", "ln1_beta", "ln2_gamma", "ln2_beta", "w1", "b1", "w2", "b2")
+
+
+def oracle_stack_params(sw: synth.StackWorkload, weights: dict):
+    """The decoder oracle's parameters from a stack's stored weights."""
+    from oracle import decoder_oracle as D
+    w = sw.layer
+    layers = []
+    for lw in weights["layers"]:
+        f = {k: v.double().numpy() for k, v in lw.items()}
+        attn = O.params_from_tensors(dims_of(w), {k: f[k] for k in ATTN_WEIGHT_NAMES},
+                                     ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+        layers.append(D.LayerParams(attn=attn, **{k: f[k] for k in LAYER_EXTRA_NAMES}))
+    return D.StackParams(layers=layers, lnf_gamma=weights["lnf_gamma"].double().numpy(),
+                         lnf_beta=weights["lnf_beta"].double().numpy())
+
+
+def gpu_stack(sw: synth.StackWorkload, weights: dict, max_batch=None, max_tokens=None,
+              max_prefill_tokens=None, device="cuda:0"):
+    from paper_2505_13544_b200 import binding as M
+    w = sw.layer
+    cfg = M.make_config(**dims_of(w), max_batch=max_batch or w.batch,
+                        max_tokens=max_tokens or w.max_tokens,
+                        max_prefill_tokens=(w.prefill_tokens if max_prefill_tokens is None
+                                            else max_prefill_tokens),
+                        dtype=w.dtype, ln_eps=w.ln_eps, rope_theta=w.rope_theta)
+    dev = {"layers": [{k: v.to(device) for k, v in lw.items()} for lw in weights["layers"]],
+           "lnf_gamma": weights["lnf_gamma"].to(device), "lnf_beta": weights["lnf_beta"].to(device)}
+    return M.mtla_stack_create(cfg, sw.n_layers, sw.d_ff, dev, device=device)

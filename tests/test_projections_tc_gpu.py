@@ -109,11 +109,11 @@ def test_split_k_reduction_is_deterministic():
 
 
 @pytest.mark.parametrize("batch", [2, 20, 40, 100, 200])
-def test_weight_streaming_schedule_matches_oracle(batch):
+def test_large_layer_projections_match_oracle(batch):
     """The layer of the large workload (d 4096, 32 heads x 128, r 512): the input and output
-    projections have few 128-row weight tiles and a 64-block reduction, which the persistent GEMM
-    cuts into equal shares that end inside tiles (partials + ticketed sum).  One batch per
-    activation box height, 16 to 256 rows; all rows against the oracle, and twice for bit-equality."""
+    projections have few 128-row weight tiles and a 64-block reduction, so they run split over
+    K with the ticketed sum of the partials.  One batch per activation box height, 16 to 256
+    rows; sampled rows against the oracle, and the whole run twice for bit-equality."""
     w = synth.WORKLOADS["large"].scaled(name="stream", batch=batch, context_tokens=200, decode_steps=3)
     weights = synth.make_weights(w)
     p = H.oracle_params(w, weights)
