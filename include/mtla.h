@@ -256,6 +256,35 @@ int mtla_stack_check(mtla_stack* s, void* stream);          /* mtla_check over t
 int64_t mtla_stack_launch_count(const mtla_stack* s);
 int mtla_stack_destroy(mtla_stack* s);
 
+/* ---- training path (Section 4.2, Eq. 14-16) ----
+ *
+ * The paper trains with the parallel form: the merge weights of every chunk at once (Eq. 16 with
+ * the chunk mask), the sequence of running states C' (Eq. 14), attention over C' and the
+ * un-compressed RoPE keys under the stride-aware causal mask.  mtla_prefill computes exactly
+ * that form (as per-chunk running sums and a mask predicate instead of T x T matrices), so it IS
+ * the training forward pass; mtla_train_backward is its reverse.  Given dL/dY it returns dL/dX
+ * and the gradient of every parameter, through the softmax and the mask, the key / value
+ * up-projections, the running sums and their sigmoid gates (including both Linear layers of
+ * the hyper-network), the LayerNorm, the rotations and the fused input projection.
+ *
+ * fp32 layers on contiguous storage only (MTLA_ERR_UNSUPPORTED_SHAPE otherwise).  The call must
+ * follow mtla_prefill(h, x, B, T, y != NULL) on the same handle with nothing in between
+ * (MTLA_ERR_STATE otherwise): it reads what that call left in the handle's prefill workspace.
+ * x, dy, dx device [B][T][d] fp32; x is the prefill's input again.  The gradient buffers are
+ * device fp32 arrays shaped like the weights of mtla_weights (row-major [in][out]); they are
+ * overwritten, not accumulated, and hold sums over the batch.  At s = 1 the hyper-network's
+ * gradients are zero.  `workspace` is device memory of at least
+ * mtla_train_workspace_bytes(h, B, T) bytes, 256-byte aligned, owned by the caller; it holds,
+ * among others, two T x T matrices per (sequence, head).  Results do not depend on the launch
+ * configuration (every reduction runs in index order). */
+typedef struct {
+  void *w_q, *w_qr, *w_r, *w_kr, *ln_gamma, *ln_beta, *w_k, *w_v, *w_o;
+  void *hyp_c_w, *hyp_c_b, *hyp_pe_w, *hyp_pe_b;
+} mtla_grads;
+size_t mtla_train_workspace_bytes(const mtla_handle* h, int32_t B, int32_t T);
+int mtla_train_backward(mtla_handle* h, const void* x, const void* dy, int32_t B, int32_t T, void* dx,
+                        const mtla_grads* grads, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of cache in use: B * ceil(tokens/s) * (r + d_R) * sizeof(element)  (Sections 4, 4.3);
  * with per-sequence token counts, the sum over the sequences. */
 size_t mtla_cache_bytes(const mtla_handle* h);

@@ -36,7 +36,8 @@ EXPORTED_SYMBOLS = (
     "mtla_baseline_arena_bytes", "mtla_baseline_create", "mtla_selftest_wait_timeout",
     "mtla_clear_error", "mtla_stack_arena_bytes", "mtla_stack_create", "mtla_stack_prefill",
     "mtla_stack_decode_step", "mtla_stack_cache_bytes", "mtla_stack_layer", "mtla_stack_reset",
-    "mtla_stack_check", "mtla_stack_launch_count", "mtla_stack_destroy")
+    "mtla_stack_check", "mtla_stack_launch_count", "mtla_stack_destroy",
+    "mtla_train_workspace_bytes", "mtla_train_backward")
 
 PAGE_SLOTS = 64
 
@@ -81,6 +82,10 @@ LAYER_EXTRA_NAMES = ("ln1_gamma", "ln1_beta", "ln2_gamma", "ln2_beta", "w1", "b1
 
 class mtla_layer_weights(ctypes.Structure):
     _fields_ = [("attn", mtla_weights)] + [(n, ctypes.c_void_p) for n in LAYER_EXTRA_NAMES]
+
+
+class mtla_grads(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in WEIGHT_NAMES]
 
 
 class mtla_stack_config(ctypes.Structure):
@@ -155,6 +160,9 @@ def load_library() -> ctypes.CDLL:
         "mtla_stack_check": (ctypes.c_int, [vp, vp]),
         "mtla_stack_launch_count": (ctypes.c_int64, [vp]),
         "mtla_stack_destroy": (ctypes.c_int, [vp]),
+        "mtla_train_workspace_bytes": (sz, [vp, i32, i32]),
+        "mtla_train_backward": (ctypes.c_int, [vp, vp, vp, i32, i32, vp, ctypes.POINTER(mtla_grads), vp,
+                                               sz, vp]),
         "mtla_selftest_wait_timeout": (ctypes.c_int, [vp, i32, vp]),
         "mtla_clear_error": (ctypes.c_int, [vp, vp]),
     }
@@ -646,3 +654,39 @@ def mtla_stack_destroy(s: Stack) -> None:
     if s.ptr:
         _check(load_library().mtla_stack_destroy(s.ptr), "mtla_stack_destroy")
         s.ptr = 0
+
+
+# --------------------------------------------------------------------------- training path
+
+def weight_shapes(cfg: mtla_config) -> dict:
+    """Shapes of the parameters (and of their gradients), row-major [in][out]."""
+    d, nh, dh, r, dr = cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.latent_rank, cfg.rope_dim
+    dw = cfg.hyper_dim or r // 4
+    return {"w_q": (d, nh * dh), "w_qr": (d, nh * dr), "w_r": (d, r), "w_kr": (d, dr),
+            "ln_gamma": (r,), "ln_beta": (r,), "w_k": (r, nh * dh), "w_v": (r, nh * dh),
+            "w_o": (nh * dh, d), "hyp_c_w": (r, dw), "hyp_c_b": (dw,), "hyp_pe_w": (r, dw),
+            "hyp_pe_b": (dw,)}
+
+
+def mtla_train_backward(h: Handle, x: torch.Tensor, dy: torch.Tensor, stream=None):
+    """The reverse of the mtla_prefill(h, x) that must directly precede this call.
+    x, dy [B][T][d] fp32 on the device.  Returns (dx, {parameter name: gradient})."""
+    b, t, d = x.shape
+    _expect(x, h, (b, t, h.config.d_model), "x")
+    _expect(dy, h, x.shape, "dy")
+    lib = load_library()
+    nbytes = lib.mtla_train_workspace_bytes(h.ptr, b, t)
+    if nbytes == 0:
+        raise MTLAError(-2, "mtla_train_workspace_bytes")
+    with torch.cuda.device(h.device):
+        ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=h.device)
+        base = (ws.data_ptr() + 255) // 256 * 256
+        dx = torch.empty_like(x)
+        grads = {n: torch.empty(*shape, dtype=torch.float32, device=h.device)
+                 for n, shape in weight_shapes(h.config).items()}
+        g = mtla_grads(*[grads[n].data_ptr() for n in WEIGHT_NAMES])
+        _check(lib.mtla_train_backward(h.ptr, x.data_ptr(), dy.data_ptr(), b, t, dx.data_ptr(),
+                                       ctypes.byref(g), base, nbytes, _stream_ptr(stream)),
+               "mtla_train_backward")
+        torch.cuda.current_stream().synchronize()     # the workspace is released on return
+    return dx, grads

@@ -217,6 +217,7 @@ struct mtla_handle {
   bool is_baseline;
   int bl_groups;
   int64_t launches;
+  int train_B, train_T;   // shape of the prefill whose workspace mtla_train_backward may read (0: none)
   int device;     // ordinal of the GPU that owns the arena
   int sm_count;   // its SM count, capped at the bound the workspaces are sized for
   bool attn_smem_ready, pf_smem_ready;
@@ -1081,6 +1082,7 @@ int step_begin(mtla_handle* h, int B, cudaStream_t st) {
 }
 
 void step_end(mtla_handle* h, int B) {
+  h->train_B = h->train_T = 0;      // the decode step reuses the prefill's scratch
   if (h->paged()) {
     for (int b = 0; b < B; ++b) {
       h->seq_tokens[b] += 1;
@@ -1199,6 +1201,7 @@ int create_handle(const mtla_config* cfg, const mtla_paging* paging, const mtla_
   h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
   h->scratch = shared_scratch ? static_cast<char*>(shared_scratch) - p.scratch_begin : nullptr;
   h->tokens = 0; h->batch = 0; h->launches = 0;
+  h->train_B = h->train_T = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
   h->prof_attention_only = false;
@@ -1422,6 +1425,7 @@ int mtla_baseline_create(const mtla_baseline_config* cfg, const mtla_baseline_we
   h->cfg = c; h->dm = dm; h->plan = p; h->arena = static_cast<char*>(arena);
   h->scratch = nullptr;
   h->tokens = 0; h->batch = 0; h->launches = 0;
+  h->train_B = h->train_T = 0;
   h->attn_smem_ready = false; h->pf_smem_ready = false;
   h->prof_used = 0;
   h->prof_attention_only = false;
@@ -1460,7 +1464,12 @@ int mtla_prefill(mtla_handle* h, const void* x, int32_t B, int32_t T, void* y, v
   if (h->tokens != 0 || h->batch != 0) return MTLA_ERR_STATE;
   if (B > h->cfg.max_batch || T > h->cfg.max_prefill_tokens || T > h->cfg.max_tokens)
     return MTLA_ERR_CAPACITY;
-  return run_prefill(h, x, 0, B, T, y, static_cast<cudaStream_t>(stream));
+  const int rc = run_prefill(h, x, 0, B, T, y, static_cast<cudaStream_t>(stream));
+  if (rc == MTLA_OK && y) {
+    h->train_B = B;
+    h->train_T = T;
+  }
+  return rc;
 }
 
 int mtla_prefill_seqs(mtla_handle* h, int32_t seq0, const void* x, int32_t B, int32_t T, void* y,
@@ -1553,6 +1562,7 @@ int mtla_reset(mtla_handle* h) {
   if (!h) return MTLA_ERR_INVALID_ARG;
   h->tokens = 0;
   h->batch = 0;
+  h->train_B = h->train_T = 0;
   if (h->paged()) {
     h->pool->reset();
     h->seq_tokens.assign(h->cfg.max_batch, 0);
@@ -1634,6 +1644,7 @@ int mtla_cache_import(mtla_handle* h, const void* src, int32_t B, int32_t tokens
   }
   h->tokens = tokens;
   h->batch = B;
+  h->train_B = h->train_T = 0;
   return MTLA_OK;
 }
 
@@ -1871,3 +1882,4 @@ const char* mtla_error_string(int status) {
 }  // extern "C"
 
 #include "stack_api.inc"
+#include "train_api.inc"
