@@ -88,7 +88,8 @@ def assert_cache_close(got: torch.Tensor, want: np.ndarray, dtype: str, scale: f
     if dtype == "fp32":
         assert np.abs(g - want).max() <= FP32_MAX_ABS * scale
     else:
-        assert (np.abs(g - want) <= scale * 2.0 ** -7 * (1.0 + np.abs(want))).all()
+        ratio = float((np.abs(g - want) / (2.0 ** -7 * (1.0 + np.abs(want)))).max())
+        assert ratio <= scale, f"cache rows: worst error {ratio:.2f} x the bf16 bound (allowed {scale:.2f})"
 
 
 ATTN_WEIGHT_NAMES = ("w_q", "w_qr", "w_r", "w_kr", "ln_gamma", "ln_beta", "w_k", "w_v", "w_o",

@@ -54,12 +54,16 @@ def run_stack(sw, seqs=None, prefill_rows=None, steps_checked=None):
                 H.assert_close_stack(yd[seqs], np.stack(want), w.dtype, sw.n_layers, f"decode step {i}")
         M.mtla_stack_check(s)
         tokens = w.prefill_tokens + w.decode_steps
+        # Cache rows: a layer inside a stack reads the bf16 rounding of LayerNorm_1(stream), which
+        # the oracle does not round, and from the second layer on also the error the stream has
+        # accumulated; the single-layer bound (a few storage ulps) is therefore taken three times
+        # wider at the first layer and grows like the outputs' bound, with sqrt(layer).
         for n in range(sw.n_layers):
             layer = M.mtla_stack_layer(s, n)
             assert M.mtla_position(layer) == (tokens, math.ceil(tokens / w.stride), w.batch)
             cache = M.mtla_cache_export(layer)
             H.assert_cache_close(cache[seqs], np.stack([O.cache_array(states[b].layers[n]) for b in seqs]),
-                                 w.dtype, scale=math.sqrt(n + 1))
+                                 w.dtype, scale=3.0 * math.sqrt(n + 1))
     finally:
         M.mtla_stack_destroy(s)
 
