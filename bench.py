@@ -678,6 +678,67 @@ def stack_cpu_baseline(sw: synth.StackWorkload, budget_s: float = 10.0) -> dict:
                       f"{w.prefill_tokens}-token prompt, {el:.1f} s"}
 
 
+FP32_FMA_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # SMs x fp32 lanes x 2 FLOP x max SM clock
+
+
+def time_training(device, batch: int = 8, tokens: int = 512, runs: int = 3,
+                  cpu_baseline: bool = True) -> dict:
+    """The training path on the paper's layer in fp32: mtla_prefill as the forward pass of the
+    parallel form and mtla_train_backward as its reverse.  A step is forward + backward over
+    `batch` sequences of `tokens` tokens; the roofline is plain fp32 FMA arithmetic (both passes
+    run on the CUDA cores; TF32 would not hold the fp32 tolerance)."""
+    from paper_2505_13544_b200 import binding as M
+    w = synth.WORKLOADS["paper"].scaled(name="train_paper_fp32", dtype="fp32", batch=batch,
+                                        prefill_tokens=tokens, decode_steps=2)
+    Mx, h = build_layer(w, extra_steps=4, device=device)
+    x = fill_prompt(w, device)
+    dy = torch.randn(x.shape, device=device, generator=torch.Generator(device=device).manual_seed(w.seed))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    fwd, bwd = [], []
+    launches = 0
+    for _ in range(runs + 1):
+        M.mtla_reset(h)
+        torch.cuda.synchronize(device)
+        l0 = M.mtla_launch_count(h)
+        ev[0].record()
+        M.mtla_prefill(h, x)
+        ev[1].record()
+        dx, grads = M.mtla_train_backward(h, x, dy)
+        ev[2].record()
+        torch.cuda.synchronize(device)
+        launches = M.mtla_launch_count(h) - l0
+        fwd.append(ev[0].elapsed_time(ev[1]))
+        bwd.append(ev[1].elapsed_time(ev[2]))
+    M.mtla_check(h)
+    assert torch.isfinite(dx).all() and all(torch.isfinite(g).all() for g in grads.values())
+    M.mtla_destroy(h)
+    f_ms, b_ms = float(np.median(fwd[1:])), float(np.median(bwd[1:]))
+    flop = prefill_flop(w)["total"]
+    # The reverse pass costs two products per forward product; its attention works on dense
+    # T x T matrices (all pairs, not only the s-th of them the mask admits).
+    res = {"workload": w.name, "batch": batch, "tokens": tokens, "stride": w.stride, "dtype": "f32",
+           "forward_ms": f_ms, "backward_ms": b_ms,
+           "tokens_per_s": batch * tokens / ((f_ms + b_ms) * 1e-3),
+           "algorithmic_tflop": 3 * flop / 1e12,
+           "roofline": {"bound": "alu", "peak": FP32_FMA_TFLOPS, "unit": "TFLOP/s",
+                        "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                        "achieved": 3 * flop / ((f_ms + b_ms) * 1e-3) / 1e12,
+                        "frac": 3 * flop / ((f_ms + b_ms) * 1e-3) / 1e12 / FP32_FMA_TFLOPS},
+           "gpu_launches": int(launches)}
+    if cpu_baseline:
+        from oracle import train_oracle as TR
+        from tests import helpers as H
+        p = H.oracle_params(w, synth.make_weights(w))
+        xs = x[0].double().cpu().numpy()
+        t0 = time.perf_counter()
+        y, sv = TR.forward(p, xs)
+        TR.backward(p, sv, dy[0].double().cpu().numpy())
+        el = time.perf_counter() - t0
+        res["cpu_baseline"] = {"value": tokens / el, "unit": "tokens/s", "kind": "oracle",
+                               "sample": f"1 of {batch} sequences, forward + backward, {el:.1f} s"}
+    return res
+
+
 def run_other_configs(device, steps: int = 64, warmup: int = 8):
     """The other benchmark configurations, each for a fraction of a second: the parallel prefill
     of the long-context workload against the tensor roofline, and decode steps of every
@@ -946,6 +1007,7 @@ def main() -> None:
     if world == 1 and args.workload == "large" and not args.no_other_configs and not args.batch:
         line["prefill"], line["configs"] = run_other_configs(device)
         line["decoder"] = time_stack(synth.STACK_WORKLOADS["decoder_paper"], device, steps=64, warmup=8)
+        line["training"] = time_training(device, cpu_baseline=not args.no_cpu_baseline)
     if world == 1 and not args.no_cpu_baseline:
         n_seq = 1 if w.batch * w.latent_rank >= 8192 else min(w.batch, 4)
         res = oracle_decode_sample(w, n_seq, budget_s=12.0, max_steps=64)

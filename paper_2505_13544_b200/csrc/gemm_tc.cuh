@@ -126,18 +126,23 @@ __device__ __forceinline__ void store4(bf16* p, const float (&v)[4], long long l
   }
 }
 
-// The finished value of output (i, j): scale, then the optional bias / ReLU / residual.
+// The finished value of output (i, j): scale, then - in the instantiations that carry them - the
+// optional bias / ReLU / residual.  (Run-time flags instead of the template parameter slowed
+// the plain products' epilogue by a third.)
+template <bool EXTRAS>
 __device__ __forceinline__ float finish(const GemmTcArgs& g, float acc, int i, int j) {
   float v = g.alpha * acc;
-  if (g.bias) v += g.bias[i];
-  if (g.relu) v = fmaxf(v, 0.f);
-  if (g.residual) v += g.residual[(long long)i * g.r_sm + (long long)j * g.r_sn];
+  if constexpr (EXTRAS) {
+    if (g.bias) v += g.bias[i];
+    if (g.relu) v = fmaxf(v, 0.f);
+    if (g.residual) v += g.residual[(long long)i * g.r_sm + (long long)j * g.r_sn];
+  }
   return v;
 }
 
 }  // namespace gtc
 
-template <int BN, int STAGES, typename OutT, bool HILO>
+template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                GemmTcArgs g) {
@@ -254,14 +259,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else {
 #pragma unroll
             for (int j = 0; j < CH; ++j)
-              if (j0 + j < g.n) put(p + j, finish(g, __uint_as_float(v[j]), i_row, j0 + j));
+              if (j0 + j < g.n) put(p + j, finish<EXTRAS>(g, __uint_as_float(v[j]), i_row, j0 + j));
           }
         } else {
           OutT* p = c + (long long)i_row * g.c_sm;
 #pragma unroll
           for (int j = 0; j < CH; ++j)
             if (j0 + j < g.n)
-              put(p + (long long)(j0 + j) * g.c_sn, finish(g, __uint_as_float(v[j]), i_row, j0 + j));
+              put(p + (long long)(j0 + j) * g.c_sn, finish<EXTRAS>(g, __uint_as_float(v[j]), i_row, j0 + j));
         }
       };
       // Accumulator columns c0 .. c0 + CH of this thread's row (hi and lo products added).
@@ -349,7 +354,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                  if (i0 + e < g.m) put(p + (long long)e * g.c_sm, finish(g, sum[e], i0 + e, j));
+                  if (i0 + e < g.m) put(p + (long long)e * g.c_sm, finish<EXTRAS>(g, sum[e], i0 + e, j));
               }
             }
           }

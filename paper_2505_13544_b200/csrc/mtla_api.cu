@@ -401,16 +401,16 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
-template <int BN, int STAGES, typename OutT, bool HILO>
+template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false>
 int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
                         const GemmTcArgs& g, dim3 grid, cudaStream_t st, bool dependent) {
   constexpr int smem = gtc::smem_bytes(HILO ? 2 * BN : BN, STAGES);
   if (!(h->gemm_attr_mask & (1u << inst))) {
-    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO>,
+    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     h->gemm_attr_mask |= 1u << inst;
   }
-  MTLA_CUDA(launch_kernel(gemm_tc_kernel<BN, STAGES, OutT, HILO>, grid, dim3(192), smem, st,
+  MTLA_CUDA(launch_kernel(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS>, grid, dim3(192), smem, st,
                           dependent, ma, mb, g));
   h->launches++;
   return MTLA_OK;
@@ -452,6 +452,19 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   if (g.bias || g.residual || g.relu) g.vec_ok = g.vec4_ok = 0;   // the epilogue extras are scalar
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
+  if (g.bias || g.residual || g.relu) {
+    // The feed-forward products of a decoder layer: the instantiations with the fused
+    // bias / ReLU / residual epilogue (single bf16 activations, no hi / lo halves).
+    if (hilo || g.b_lo_col > 0) return MTLA_ERR_UNSUPPORTED_SHAPE;
+    switch (bn) {
+      case 16: return launch_gemm_tc_inst<16, 4, OutT, false, true>(h, 21 + o, ma, mb, g, grid, st, dependent);
+      case 32: return launch_gemm_tc_inst<32, 4, OutT, false, true>(h, 23 + o, ma, mb, g, grid, st, dependent);
+      case 64: return launch_gemm_tc_inst<64, 4, OutT, false, true>(h, 25 + o, ma, mb, g, grid, st, dependent);
+      case 128: return launch_gemm_tc_inst<128, 3, OutT, false, true>(h, 27 + o, ma, mb, g, grid, st, dependent);
+      case 256: return launch_gemm_tc_inst<256, 4, OutT, false, true>(h, 29 + o, ma, mb, g, grid, st, dependent);
+      default: return MTLA_ERR_UNSUPPORTED_SHAPE;
+    }
+  }
   if (shallow && (sizeof(OutT) == 4 || hilo)) {
     if constexpr (sizeof(OutT) == 4) {
       switch (bn) {
