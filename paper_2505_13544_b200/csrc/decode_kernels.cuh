@@ -22,6 +22,9 @@ struct ProjLayout {
 struct PostArgs {
   const float* p1;        // [B][proj.width] fused projection of this step's tokens (fp32)
   ProjLayout proj;
+  int absorbed;           // 1: the query block of p1 is the absorbed, pre-scaled query (layers that keep
+                          // W_Q W_K^T pre-multiplied): n_h r columns from the weight's bf16 hi half,
+                          // then n_h r from its lo half; their sum goes to qt
   const float* gamma;     // [r]
   const float* beta;      // [r]
   const float* hyp_c_w;   // [r][d_w] fp32
@@ -309,7 +312,23 @@ __global__ void __launch_bounds__(256) decode_post_fast_kernel(PostArgs a) {
   }
   // Warps 1-7: queries.  bf16 [hi | lo] halves of q, four elements per thread and step.
   const int t = tid - 32;
-  if (a.q16) {
+  if (a.absorbed) {
+    // The projection already holds q~ (Eq. 12) in two parts: add them, narrow into the attention kernel's rows.
+    TQ* qrow = static_cast<TQ*>(a.qt) + (long long)b * a.n_heads * W;
+    for (int i = t * 4; i < a.n_heads * a.r; i += 224 * 4) {
+      const int h = i / a.r, j = i % a.r;
+      float4 q4 = *reinterpret_cast<const float4*>(row + a.proj.off_q + i);
+      const float4 ql = *reinterpret_cast<const float4*>(row + a.proj.off_q + a.n_heads * a.r + i);
+      q4.x += ql.x; q4.y += ql.y; q4.z += ql.z; q4.w += ql.w;
+      if (sizeof(TQ) == 2) {
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(q4.x, q4.y), h1 = __floats2bfloat162_rn(q4.z, q4.w);
+        *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(qrow) + h * W + j) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+      } else {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(qrow) + h * W + j) = q4;
+      }
+    }
+  } else if (a.q16) {
     const int hd = a.n_heads * a.head_dim;
     bf16* dst = a.q16 + (long long)b * 2 * hd;
     for (int i = t * 4; i < hd; i += 224 * 4) {

@@ -40,6 +40,9 @@ struct GemmTcArgs {
   int b_lo_col;               // > 0: B rows hold [hi | lo] bf16 halves of an fp32 activation, lo
                               // starting at this column; both halves are multiplied (2 passes
                               // over each K block), which keeps ~16 mantissa bits of B
+  int b_k_wrap;               // K blocks after which B's K index starts over (A holds [hi | lo]
+                              // halves of a weight along K, both multiplied by the same B columns);
+                              // a value >= the K blocks of the product leaves B unwrapped
   long long c_lo_off;         // > 0 (bf16 output only): also store the rounding remainder
                               // bf16(val - bf16(val)) this many elements after each output
   int kb_per_split, n_split;  // K blocks (of 64) per split; number of splits
@@ -206,11 +209,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t dst = base + st * stage_bytes(NB);
       mbar_arrive_expect_tx(bar(&bars->full[st]), stage_bytes(NB));
       tma_load_2d(dst, &map_a, bar(&bars->full[st]), a_col + kb * kBK, a_row);
-      tma_load_2d(dst + kABytes, &map_b, bar(&bars->full[st]), b_col + lo * g.b_lo_col + kb * kBK,
+      const int kbb = kb - (kb >= g.b_k_wrap ? g.b_k_wrap : 0);
+      tma_load_2d(dst + kABytes, &map_b, bar(&bars->full[st]), b_col + lo * g.b_lo_col + kbb * kBK,
                   b_row);
       if (HILO)
         tma_load_2d(dst + kABytes + b_bytes(BN), &map_b, bar(&bars->full[st]),
-                    b_col + g.b_lo_col + kb * kBK, b_row);
+                    b_col + g.b_lo_col + kbb * kBK, b_row);
     }
   } else if (warp == 1 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer

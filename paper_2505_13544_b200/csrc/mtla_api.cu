@@ -36,6 +36,11 @@ constexpr int kTargetCtas = 2 * kPlanSms;   // CUDA-core attention: two CTAs per
 constexpr int kMinSlotsPerSplit = 64;
 constexpr int kFusedCombineMaxParts = 8;   // more parts per sequence: the combine gets its own launch
 constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill projections
+// Layers whose pre-multiplied matrices W_Q W_K^T and W_V W_O (Eq. 12, taken literally) stay below
+// this size each keep them for the decode step: two launches fewer per step, which is what counts
+// where the whole layer lives in L2.  Larger layers keep the two-step form (the pre-multiplied
+// matrices have n_h r / (n_h d_h) times the bytes of the factors, and decode streams the weights).
+constexpr size_t kFoldMaxBytes = 8u << 20;
 constexpr int kGemmSlots = 2 * kPlanSms;   // CTAs a split-K GEMM may spread one product over
 
 
@@ -48,6 +53,9 @@ int act_box_rows(int B) {
 
 struct ArenaPlan {
   size_t wcat_t, w_k, w_kv_t, w_o_t;
+  size_t wcat_dec_t, w_vo_t;   // folded decode weights (Dims::fold): [q~ hi | q~ lo | q^R | c | k^R | u][d],
+                               // [d][hi | lo of n_h r]
+  size_t fold_tmp;             // [r][d] fp32: one head's product before it is split (create only)
   size_t gamma, beta, hyp_c_w, hyp_c_b, hyp_pe_w, hyp_pe_b, gate_pe, rope_cos, rope_sin;
   size_t gate_s, gate_t, gate_tmp;
   size_t cache, open_acc, err_flag;
@@ -63,6 +71,11 @@ struct Dims {
   int n_pages, max_pages;   // paged handles: pool size, pages per sequence; 0 otherwise
   size_t elem;
   ProjLayout proj;
+  // Decode with pre-multiplied weights: the input projection emits the absorbed query directly
+  // (columns [0, n_h r) of proj_dec, its off_q), the attention output goes through W_V W_O at once.
+  bool fold;
+  ProjLayout proj_dec;
+  int ntot_dec;
 };
 
 bool normalise(const mtla_config* in, const mtla_paging* pg, mtla_config* out, Dims* dm) {
@@ -102,6 +115,21 @@ bool normalise(const mtla_config* in, const mtla_paging* pg, mtla_config* out, D
     dm->proj.width = (dm->proj.width + 2 * dm->dw + 3) / 4 * 4;
   }
   dm->ntot = dm->proj.width;
+  dm->fold = c.dtype == MTLA_DTYPE_BF16 && c.latent_rank % 128 == 0 && c.kernel_path != MTLA_PATH_CUDA_CORE &&
+             (size_t)dm->nh * dm->r * dm->d * 2 <= kFoldMaxBytes;
+  dm->proj_dec = dm->proj;
+  dm->ntot_dec = dm->ntot;
+  if (dm->fold) {
+    // The query block widens from d_h to r columns per head, twice: the pre-multiplied weight is
+    // kept as bf16 [hi | lo] row blocks and the two partial queries are added after the product.
+    const int shift = 2 * dm->nh * dm->r - dm->nh * dm->dh;
+    dm->proj_dec.off_qr += shift;
+    dm->proj_dec.off_c += shift;
+    dm->proj_dec.off_kr += shift;
+    if (dm->proj_dec.off_u >= 0) dm->proj_dec.off_u += shift;
+    dm->proj_dec.width += shift;
+    dm->ntot_dec = dm->proj_dec.width;
+  }
   dm->max_slots = ceil_div(c.max_tokens, c.stride);
   dm->max_units = kTargetCtas + c.max_batch;
   dm->n_pages = dm->max_pages = 0;
@@ -128,6 +156,9 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->w_k = take((size_t)dm.r * hd * e);
   p->w_kv_t = take(2 * hd * dm.r * e);
   p->w_o_t = take((size_t)dm.d * hd * e);
+  p->wcat_dec_t = take(dm.fold ? (size_t)dm.ntot_dec * dm.d * e : 0);
+  p->w_vo_t = take(dm.fold ? (size_t)dm.d * 2 * dm.nh * dm.r * e : 0);
+  p->fold_tmp = take(dm.fold ? (size_t)dm.r * dm.d * 4 : 0);
   p->gamma = take(dm.r * 4);
   p->beta = take(dm.r * 4);
   p->hyp_c_w = take((size_t)dm.r * dm.dw * 4);
@@ -147,7 +178,7 @@ void plan_arena(const mtla_config& c, const Dims& dm, ArenaPlan* p) {
   p->seq_tokens = take(paged * 2 * B * sizeof(int));
   p->err_flag = take(16);
   p->scratch_begin = off;
-  p->p1 = take(B * dm.ntot * 4);
+  p->p1 = take(B * (size_t)max(dm.ntot, dm.ntot_dec) * 4);
   p->q16 = take(B * 2 * hd * 2);
   p->qt = take(B * dm.nh * dm.W * 4);
   p->o_part = take((size_t)dm.max_units * dm.nh * dm.r * 4);
@@ -227,6 +258,7 @@ struct mtla_handle {
   // Tensor-core projections (bf16): weight panels as 128-row boxes, serving as the MMA's M side
   // in the decode step and as its N side in the prefill; decode activations as act_bn-row boxes.
   CUtensorMap map_wcat, map_wk, map_wkvt, map_wvt, map_wot;
+  CUtensorMap map_wcat_dec, map_wvo;   // folded decode weights
   CUtensorMap map_q16, map_o16, map_v16;
   int act_bn;               // box rows the three activation maps were encoded with (0: none yet)
   unsigned gemm_attr_mask;  // kernel instances whose shared-memory limit has been raised
@@ -505,6 +537,7 @@ GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, i
   GemmTcArgs g;
   memset(&g, 0, sizeof(g));
   g.c = c; g.c_sm = c_sm; g.c_sn = c_sn; g.m = m; g.n = n; g.k = k; g.alpha = alpha;
+  g.b_k_wrap = 1 << 30;
   return g;
 }
 
@@ -615,6 +648,46 @@ int create_impl(mtla_handle* h, const mtla_weights* w, cudaStream_t st) {
     MTLA_TRY(make_map_2d(&h->map_wkvt, h->at<void>(p.w_kv_t), 2 * hd, dm.r, dm.r, gtc::kBM));
     MTLA_TRY(make_map_2d(&h->map_wvt, h->at<T>(p.w_kv_t) + (size_t)hd * dm.r, hd, dm.r, dm.r, gtc::kBM));
     MTLA_TRY(make_map_2d(&h->map_wot, h->at<void>(p.w_o_t), dm.d, hd, hd, gtc::kBM));
+    if (dm.fold) {
+      // Eq. 12's products, per head, from the weights as given, accumulated in fp32 and kept as
+      // bf16 [hi | lo] halves (about 16 mantissa bits, as the activations of the unfolded path):
+      //   rows h r + j of the decode projection = scale * W_{K,h}[j] . W_{Q,h}^T      [r][d], hi block
+      //   rows n_h r + h r + j                  = its rounding remainder                      lo block
+      //   columns h r + j of W_VO^T             = W_{O,h}^T . W_{V,h}[j]              [d][r], hi half
+      //   columns n_h r + h r + j               = its rounding remainder                      lo half
+      bf16* wdec = h->at<bf16>(p.wcat_dec_t);
+      bf16* wvo = h->at<bf16>(p.w_vo_t);
+      float* tmp = h->at<float>(p.fold_tmp);
+      const T* wk_in = static_cast<const T*>(w->w_k);
+      const T* wq_in = static_cast<const T*>(w->w_q);
+      const T* wv_in = static_cast<const T*>(w->w_v);
+      const long long onr = (long long)dm.nh * dm.r;
+      const float q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+      const unsigned pack_blocks = (unsigned)(((long long)dm.r * dm.d + 255) / 256);
+      for (int hh = 0; hh < dm.nh; ++hh) {
+        MTLA_TRY((gemm<T, T, float>(h, wk_in + (size_t)hh * dm.dh, wq_in + (size_t)hh * dm.dh, tmp, dm.r,
+                                    dm.d, dm.dh, hd, hd, dm.d, q_scale, 1, 0, 0, 0, st)));
+        split_hi_lo_kernel<<<pack_blocks, 256, 0, st>>>(tmp, wdec + (size_t)hh * dm.r * dm.d,
+                                                        wdec + (size_t)(onr + hh * dm.r) * dm.d, dm.r,
+                                                        dm.d, dm.d, dm.d);
+        h->launches++;
+        MTLA_CUDA(cudaGetLastError());
+        MTLA_TRY((gemm<T, T, float>(h, h->at<T>(p.w_o_t) + (size_t)hh * dm.dh, wv_in + (size_t)hh * dm.dh,
+                                    tmp, dm.d, dm.r, dm.dh, hd, hd, dm.r, 1.f, 1, 0, 0, 0, st)));
+        split_hi_lo_kernel<<<pack_blocks, 256, 0, st>>>(tmp, wvo + (size_t)hh * dm.r,
+                                                        wvo + (size_t)(onr + hh * dm.r), dm.d, dm.r,
+                                                        dm.r, 2 * onr);
+        h->launches++;
+        MTLA_CUDA(cudaGetLastError());
+      }
+      // Everything behind the query block is the same in both projections.
+      MTLA_CUDA(cudaMemcpyAsync(wdec + (size_t)2 * onr * dm.d,
+                                h->at<bf16>(p.wcat_t) + (size_t)dm.proj.off_qr * dm.d,
+                                (size_t)(dm.ntot - dm.proj.off_qr) * dm.d * sizeof(bf16),
+                                cudaMemcpyDeviceToDevice, st));
+      MTLA_TRY(make_map_2d(&h->map_wcat_dec, wdec, dm.ntot_dec, dm.d, dm.d, gtc::kBM));
+      MTLA_TRY(make_map_2d(&h->map_wvo, h->at<void>(p.w_vo_t), dm.d, 2 * onr, 2 * onr, gtc::kBM));
+    }
   }
   return MTLA_OK;
 }
@@ -712,9 +785,10 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     MTLA_TRY(ensure_activation_maps(h, B));
     CUtensorMap map_x;
     MTLA_TRY(make_map_2d(&map_x, x, B, dm.d, dm.d, bn));
-    MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x,
-                            gemm_tc_args(h->at<float>(p.p1), 1, dm.ntot, dm.ntot, B, dm.d, 1.f), bn, 1,
-                            true, st));
+    // With pre-multiplied weights the projection's query block is the absorbed query itself.
+    const int n_out = dm.fold ? dm.ntot_dec : dm.ntot;
+    MTLA_TRY(gemm_tc<float>(h, dm.fold ? h->map_wcat_dec : h->map_wcat, map_x,
+                            gemm_tc_args(h->at<float>(p.p1), 1, n_out, n_out, B, dm.d, 1.f), bn, 1, true, st));
   } else {
     MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d,
                                 dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
@@ -723,7 +797,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   MTLA_TRY(prof_mark(h, prof, 1, st));
   PostArgs pa;
   pa.p1 = h->at<float>(p.p1);
-  pa.proj = dm.proj;
+  pa.proj = dm.fold ? dm.proj_dec : dm.proj;
+  pa.absorbed = dm.fold ? 1 : 0;
   pa.gamma = h->at<float>(p.gamma);
   pa.beta = h->at<float>(p.beta);
   pa.hyp_c_w = h->at<float>(p.hyp_c_w);
@@ -763,7 +838,9 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   MTLA_TRY(prof_mark(h, prof, 2, st));
   // a6: q~_h = scale * q_h W_{K,h}^T, one z-slice per head, straight from the fp32 projection
   // (bf16 output where the tensor-core attention consumes it).
-  if (h->use_tc) {
+  if (dm.fold) {
+    // nothing to do: the post kernel has written the absorbed query
+  } else if (h->use_tc) {
     GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.qt), 1, (long long)dm.nh * dm.W, dm.r, B, dm.dh, pa.q_scale);
     g.c_sz = dm.W; g.a_col_z = dm.dh; g.b_col_z = dm.dh; g.b_lo_col = hd;
     MTLA_TRY(gemm_tc<bf16>(h, h->map_wk, h->map_q16, g, bn, dm.nh, true, st, pdl));
@@ -836,7 +913,15 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
 
   // a8: v_h = o_h W_{V,h} per head, then y = concat_h(v_h) W_O.
   MTLA_TRY(prof_mark(h, prof, 5, st));
-  if (h->use_tc) {
+  if (dm.fold) {
+    // y = o (W_V W_O) over K = 2 n_h r: the weight's [hi | lo] halves along K meet the same
+    // columns of o, itself [hi | lo] halves stacked in the B tile.
+    MTLA_TRY(prof_mark(h, prof, 6, st));
+    GemmTcArgs g = gemm_tc_args(y, 1, dm.d, dm.d, B, 2 * dm.nh * dm.r, 1.f);
+    g.b_lo_col = dm.nh * dm.r;
+    g.b_k_wrap = dm.nh * dm.r / gtc::kBK;
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wvo, h->map_o16, g, bn, 1, true, st, pdl && !prof));
+  } else if (h->use_tc) {
     GemmTcArgs g = gemm_tc_args(h->at<bf16>(p.v), 1, 2 * hd, dm.dh, B, dm.r, 1.f);
     g.c_sz = dm.dh; g.a_row_z = dm.dh; g.b_col_z = dm.r; g.b_lo_col = dm.nh * dm.r; g.c_lo_off = hd;
     MTLA_TRY(gemm_tc<bf16>(h, h->map_wvt, h->map_o16, g, bn, dm.nh, true, st, pdl && !prof));

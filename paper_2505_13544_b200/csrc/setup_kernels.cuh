@@ -51,6 +51,19 @@ __global__ void gate_fold_pack_kernel(const float* wg, bf16* dst, int dw, long l
   dst[dw * d + idx] = __float2bfloat16_rn(wg[idx] - __bfloat162float(hi));
 }
 
+// Splits a rows x cols fp32 matrix (row pitch ld_src) into bf16 halves: `hi` receives the rounded
+// values, `lo` the rounding remainders, both with row pitch ld_dst.
+__global__ void split_hi_lo_kernel(const float* src, bf16* hi, bf16* lo, int rows, int cols,
+                                   long long ld_src, long long ld_dst) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)rows * cols) return;
+  const long long i = idx / cols, j = idx % cols;
+  const float v = src[i * ld_src + j];
+  const bf16 h = __float2bfloat16_rn(v);
+  hi[i * ld_dst + j] = h;
+  lo[i * ld_dst + j] = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+
 // gate_s[n] = sum_i gamma[i] A[i][n];  gate_t[n] = sum_i beta[i] A[i][n] + a[n].
 __global__ void gate_fold_vectors_kernel(const float* a /*[r][d_w]*/, const float* bias,
                                          const float* gamma, const float* beta, float* gate_s,
