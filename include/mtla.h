@@ -389,6 +389,15 @@ int mtla_profile_begin_attention(mtla_handle* h, int32_t max_steps);
 int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps);
 int mtla_profile_end_stages(mtla_handle* h, double* stage_ms, int32_t* steps);
 
+/* Beam search on paged handles: when the batch consists of blocks of consecutive sequences of
+ * equal length that share their first page (the beams of one utterance after mtla_beam_reorder),
+ * the tensor-core decode attention walks each block with a gang of CTAs side by side, one
+ * sequence each over the same tiles at the same time, so that a shared page is read from DRAM
+ * once.  Returns the gang size of the handle's latest decode step: 1 = every CTA on its own
+ * share (lock-step batches, unrelated sequences), 0 = no tensor-core decode step has run yet
+ * (or h is NULL).  Host query only; never fails. */
+int32_t mtla_attention_gang(const mtla_handle* h);
+
 /* Name of the decode-attention kernel variant the handle dispatches to ("fma" or "tcgen05"). */
 const char* mtla_attention_variant(const mtla_handle* h);
 

@@ -10,6 +10,7 @@ from __future__ import annotations
 import ctypes
 from dataclasses import dataclass
 
+import numpy as np
 import torch
 
 from .build import LIB_PATH, build_library
@@ -27,7 +28,7 @@ EXPORTED_SYMBOLS = (
     "mtla_arena_bytes", "mtla_create", "mtla_prefill", "mtla_decode_step",
     "mtla_decode_step_host", "mtla_cache_bytes", "mtla_destroy", "mtla_reset", "mtla_position",
     "mtla_cache_export", "mtla_cache_import", "mtla_check", "mtla_launch_count",
-    "mtla_attention_variant", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
+    "mtla_attention_variant", "mtla_attention_gang", "mtla_error_string", "mtla_profile_begin", "mtla_profile_end",
     "mtla_profile_end_stages", "mtla_decode_step_static", "mtla_profile_begin_attention",
     "mtla_arena_bytes_paged", "mtla_create_paged", "mtla_prefill_seqs", "mtla_beam_reorder",
     "mtla_seq_positions", "mtla_pages_in_use", "mtla_cache_export_seq", "mtla_cache_import_seqs",
@@ -141,6 +142,7 @@ def load_library() -> ctypes.CDLL:
         "mtla_check": (ctypes.c_int, [vp, vp]),
         "mtla_launch_count": (ctypes.c_int64, [vp]),
         "mtla_attention_variant": (ctypes.c_char_p, [vp]),
+        "mtla_attention_gang": (ctypes.c_int32, [vp]),
         "mtla_profile_begin": (ctypes.c_int, [vp, i32]),
         "mtla_profile_begin_attention": (ctypes.c_int, [vp, i32]),
         "mtla_profile_end": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double),
@@ -342,6 +344,10 @@ def mtla_cache_import_seqs(h: Handle, seq0: int, cache: torch.Tensor, tokens: in
 
 
 def _i32_array(values):
+    """int32 C array of a sequence; a contiguous numpy int32 array is passed as it is (no copy),
+    which is what a decoding loop that calls once per step should hand over."""
+    if isinstance(values, np.ndarray) and values.dtype == np.int32 and values.flags.c_contiguous:
+        return values.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
     return (ctypes.c_int32 * len(values))(*[int(v) for v in values])
 
 
@@ -512,6 +518,11 @@ def mtla_clear_error(h: Handle, stream=None) -> None:
 
 def mtla_launch_count(h: Handle) -> int:
     return load_library().mtla_launch_count(h.ptr)
+
+
+def mtla_attention_gang(h: Handle) -> int:
+    """Gang size of the latest decode step's attention launch (see include/mtla.h)."""
+    return int(load_library().mtla_attention_gang(h.ptr))
 
 
 def mtla_attention_variant(h: Handle) -> str:

@@ -53,7 +53,10 @@
 // tile, so only the tile's TMA coordinate changes; the tile list is then B variable-length runs,
 // whose prefix sums every CTA forms in shared memory before it locates its share, and the page
 // numbers of the share's first tiles are staged in shared memory so that no load waits for a
-// table lookup.
+// table lookup.  With a gang size (gridDim.x) above 1 the list is that of the gangs' first
+// sequences, CTA (j, v) is member j of virtual CTA v and walks v's share on sequence
+// entry * gang + j; partials and tickets are indexed so that each member's parts keep the
+// order of the virtual CTAs.
 //
 // Every wait is a bounded mbarrier wait (see sm100_ptx.cuh), the rendezvous of the softmax
 // threads included; on a timeout the CTA raises its abort word, all roles unwind, and the host
@@ -79,6 +82,13 @@ struct AttnTcArgs {
   const int* seq_tokens;   // [B] tokens per sequence, this step's included
   const int* page_table;   // [B][max_pages] page of tile t of sequence b
   int max_pages, stride;
+  // Ragged batches: `gang` consecutive sequences with equal tile counts (the beams of one
+  // utterance, which share all pages but their newest) are walked by `gang` CTAs side by side,
+  // one sequence each over the same tile range at the same time, so that a shared page is read
+  // from DRAM once and served to the other CTAs by L2.  The ragged kernel is launched on a
+  // grid (gang, virtual CTAs): blockIdx.x is the member, blockIdx.y the virtual CTA whose share
+  // of the list of gangs it walks; gang 1 gives every CTA its own share of the whole list.
+  int n_list;              // entries of the tile list: batch / gang
   // 0: the partials are combined by decode_combine_parts_kernel afterwards (lock-step batches
   // whose sequences are spread over many CTAs), 1: by the last CTA of each sequence.
   int fused_combine;
@@ -271,15 +281,20 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   // This CTA's share of the tile list.
   const uint32_t prefix_s = base + kOffPrefix, staged_s = base + kOffStaged;   // ragged only
   long long total = (long long)a.batch * a.tiles_per_seq;
+  // Lock-step batches: a 1-D grid.  Ragged ones: (gang member, virtual CTA), all of them special
+  // registers, so that no thread carries them through its loop.
+  const int gang = RAGGED ? gridDim.x : 1;
+  const int vcta = RAGGED ? blockIdx.y : blockIdx.x, member = RAGGED ? blockIdx.x : 0;
+  const int n_list = RAGGED ? a.n_list : a.batch;   // entries of the tile list (sequences or gangs)
   if constexpr (RAGGED) {
     // prefix[b] = tiles of the sequences before b; prefix[batch + 1] repeats the total.
     int* prefix = reinterpret_cast<int*>(sm + kOffPrefix);
-    for (int i = threadIdx.x; i < a.batch; i += kThreads)
-      prefix[i + 1] = ceil_div(ceil_div(a.seq_tokens[i], a.stride), kTile);
+    for (int i = threadIdx.x; i < n_list; i += kThreads)
+      prefix[i + 1] = ceil_div(ceil_div(a.seq_tokens[i * gang], a.stride), kTile);
     __syncthreads();
     if (warp == 0) {
-      const int per = ceil_div(a.batch, 32);
-      const int lo = min(a.batch, lane * per), hi = min(a.batch, lo + per);
+      const int per = ceil_div(n_list, 32);
+      const int lo = min(n_list, lane * per), hi = min(n_list, lo + per);
       int sum = 0;
       for (int i = lo; i < hi; ++i) sum += prefix[i + 1];
       int incl = sum;
@@ -296,22 +311,22 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (lane == 0) prefix[0] = 0;
     }
     __syncthreads();
-    total = prefix[a.batch];
+    total = prefix[n_list];
     if (threadIdx.x == 0) {
-      prefix[a.batch + 1] = (int)total;
+      prefix[n_list + 1] = (int)total;
       misc->total_tiles = total;
     }
   }
-  const long long G = gridDim.x;
-  const long long g0 = share_begin(blockIdx.x, total, G), g1 = share_begin(blockIdx.x + 1, total, G);
+  const long long G = RAGGED ? gridDim.y : gridDim.x;     // (virtual) CTAs that share the list
+  const long long g0 = share_begin(vcta, total, G), g1 = share_begin(vcta + 1, total, G);
   const int n_tiles = (int)(g1 - g0);
   const int tps_u = a.tiles_per_seq;
   if constexpr (RAGGED) {
     int* staged = reinterpret_cast<int*>(sm + kOffStaged);
     for (int n = threadIdx.x; n < min(n_tiles, kStagedPages); n += kThreads) {
       TileCursor<true> c;
-      c.locate(g0 + n, 0, prefix_s, a.batch);
-      staged[n] = a.page_table[(long long)c.b * a.max_pages + c.t];
+      c.locate(g0 + n, 0, prefix_s, n_list);
+      staged[n] = a.page_table[(long long)(c.b * gang + member) * a.max_pages + c.t];
     }
     __syncthreads();
   }
@@ -327,14 +342,14 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     bool ok = true;
     int pc = 0, seg = 0;
     TileCursor<RAGGED> cur, ahead;
-    cur.locate(g0, tps_u, prefix_s, a.batch);
+    cur.locate(g0, tps_u, prefix_s, n_list);
     ahead = cur;
     // TMA coordinates (slot, plane) of a tile: its place in the sequence's row range, or its page.
     auto tile_coords = [&](const TileCursor<RAGGED>& c, int n, int& c_slot, int& c_plane) {
       if constexpr (RAGGED) {
         c_slot = 0;
         c_plane = n < kStagedPages ? lds_i32(staged_s + 4 * n)
-                                   : __ldg(a.page_table + (long long)c.b * a.max_pages + c.t);
+                                   : __ldg(a.page_table + (long long)(c.b * gang + member) * a.max_pages + c.t);
       } else {
         c_slot = c.t * kTile;
         c_plane = c.b;
@@ -353,9 +368,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     };
     for (int n = 0; n < kPrefetchAhead; ++n) prefetch_tile(n);
     for (int n = 0; n < n_tiles && ok; ++n, cur.next(prefix_s)) {
-      const int b = cur.b;
       prefetch_tile(n + kPrefetchAhead);
       if (n == 0 || cur.seq_first()) {
+        const int b = cur.b * gang + member;
         // A segment starts: q~ of sequence b, once the previous segment's score MMAs are done.
         ok = mbar_wait(bar(&misc->q_empty), (seg & 1) ^ 1, abort_word, a.error_word, 1);
         if (!ok) break;
@@ -500,7 +515,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     };
     float l_acc[NQ];
     TileCursor<false> cur;             // lock-step batches: every thread walks the list
-    if constexpr (!RAGGED) cur.locate(g0, tps_u, prefix_s, a.batch);
+    if constexpr (!RAGGED) cur.locate(g0, tps_u, prefix_s, n_list);
     int seg_left = 0;                  // ragged batches: tiles left in the running segment
     for (int n = 0; n < n_tiles; ++n) {
       bool seg_first, seg_last;
@@ -509,9 +524,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         if (seg_first && sidx == 0) {
           // One thread finds the segment that starts at tile n and describes it in shared memory.
           TileCursor<true> c;
-          c.locate(g0 + n, 0, prefix_s, a.batch);
+          c.locate(g0 + n, 0, prefix_s, n_list);
           const int tiles = min(n_tiles - n, c.tps - c.t);
-          const int seq_slots = ceil_div(__ldg(a.seq_tokens + c.b), a.stride);
+          const int seq_slots = ceil_div(__ldg(a.seq_tokens + c.b * gang + member), a.stride);
           misc->seg_b = c.b;
           misc->seg_tiles = tiles;
           misc->seg_tps = c.tps;
@@ -661,7 +676,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (!seg_last) continue;
       // ---------------------------------------------------------------- end of a segment
       // Partial of sequence b: wait for the last value MMAs, read O^T from TMEM.
-      int b, seq_tiles;
+      int b, seq_tiles;                // b: list entry (the sequence, or its gang)
       long long seq_start;
       if constexpr (RAGGED) {          // read before the first rendezvous below
         b = misc->seg_b;
@@ -672,7 +687,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         seq_tiles = tps_u;
         seq_start = (long long)b * tps_u;
       }
-      const long long part = blockIdx.x + b;      // unique per (CTA, sequence), increasing
+      const int seq = b * gang + member;
+      // Unique per (CTA, sequence); a sequence's parts follow one another `gang` entries apart.
+      const long long part = ((long long)vcta + b) * gang + member;
       if (ok) ok = mbar_wait(bar(&misc->p_empty[n & 1]), (n >> 1) & 1, abort_word, a.error_word, 8);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
@@ -705,16 +722,16 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       if (sidx == 0) {
         int last = 0;
         if (ok) {
-          const int old = atomicAdd(a.tickets + b, 1);
+          const int old = atomicAdd(a.tickets + seq, 1);
           last = old == n_parts - 1;
-          if (last) a.tickets[b] = 0;
+          if (last) a.tickets[seq] = 0;
         }
         misc->last_flag = last;
       }
       group_sync();
       if (ok && misc->last_flag) {
         __threadfence();
-        const long long part0 = c_first + b;
+        const long long part0 = (c_first + b) * gang + member;
         // Per head: global reference, each part's weight 2^(m_p - m) and the denominator.  All
         // loops over the parts keep kU loads in flight: a sequence spread over many CTAs (a small
         // batch with a long context) has tens of parts, and one load at a time would make this
@@ -722,7 +739,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         constexpr int kU = 8;
         if (sidx < a.n_heads) {
           const float* ml0 = a.ml_part + (part0 * a.n_heads + sidx) * 2;
-          const long long ml_step = 2ll * a.n_heads;
+          const long long ml_step = 2ll * a.n_heads * gang;
           float m = -INFINITY;
           for (int p0 = 0; p0 < n_parts; p0 += kU) {
             float mv[kU];
@@ -756,9 +773,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         const int col_groups = a.r >> 2, lanes = kSoftmaxThreads / col_groups;
         const int cg = sidx % col_groups, hh = sidx / col_groups;
         if (ok && hh < lanes) {
-          bf16* o_hi = a.o16 + (long long)b * 2 * a.n_heads * a.r + 4 * cg;
+          bf16* o_hi = a.o16 + (long long)seq * 2 * a.n_heads * a.r + 4 * cg;
           bf16* o_lo = o_hi + (long long)a.n_heads * a.r;
-          const long long o_step = (long long)a.n_heads * a.r, ml_step = 2ll * a.n_heads;
+          const long long o_step = (long long)a.n_heads * a.r * gang, ml_step = 2ll * a.n_heads * gang;
           for (int h = hh; h < a.n_heads; h += lanes) {
             const float* o0 = a.o_part + (part0 * a.n_heads + h) * a.r + 4 * cg;
             const float* ml0 = a.ml_part + (part0 * a.n_heads + h) * 2;

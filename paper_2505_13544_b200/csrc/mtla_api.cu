@@ -242,6 +242,7 @@ struct mtla_handle {
   // changes (prefill, import, reset) mark it stale and the next call re-sends them.
   PagePool* pool;
   std::vector<int> seq_tokens;
+  int last_gang = 0;      // gang size of the latest tensor-core decode attention launch (0: none yet)
   bool tokens_stale;
   // Comparison layers (mtla_baseline_create): multi-head / grouped-query / multi-query attention
   // over a key-value cache; g key/value heads per sequence, each a plane of the cache.
@@ -542,7 +543,7 @@ GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, i
 }
 
 template <int NHP, bool RAGGED>
-int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_t st, bool dependent) {
+int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, dim3 grid, cudaStream_t st, bool dependent) {
   constexpr int kSmem = RAGGED ? tc::kSmemBytesRagged : tc::kSmemBytes;
 #define MTLA_TC_CASE(RP)                                                                       \
   case RP:                                                                                     \
@@ -557,7 +558,7 @@ int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, int grid, cudaStream_
       MTLA_CUDA(cudaFuncSetAttribute(decode_attn_tc_kernel<NHP, RP, RAGGED>,                           \
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem)); \
     }                                                                                          \
-    MTLA_CUDA(launch_kernel(decode_attn_tc_kernel<NHP, RP, RAGGED>, dim3(grid), dim3(tc::kThreads),    \
+    MTLA_CUDA(launch_kernel(decode_attn_tc_kernel<NHP, RP, RAGGED>, grid, dim3(tc::kThreads),          \
                             kSmem, st, dependent, h->cache_map, h->q_map, a));                 \
     break;
   switch (a.r / 128) {
@@ -737,6 +738,40 @@ int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
   return launch_attn_fma_rpt<T, TQ, 32>(h, a, B, st);
 }
 
+// Gang size for the paged attention launch (beam search).  The kernel needs the batch to be
+// blocks of g consecutive sequences with equal token counts; gangs pay when the sequences of a
+// block share their pages, which is taken from the first page: g is the length of the first run
+// of sequences that have the same first page and length, and at least half of the blocks must
+// share theirs (an utterance shorter than a page does not: its only page is the one each beam
+// writes).  The gang is the largest divisor of g that leaves at most a tenth of the SMs without
+// a whole gang.  1: no gangs.
+int beam_gang(const mtla_handle* h, int B) {
+  auto same_len = [&](int a, int b) { return h->seq_tokens[a] == h->seq_tokens[b]; };
+  auto same_page = [&](int a, int b) {
+    return h->pool->pages_held(a) > 0 && h->pool->pages_held(b) > 0 &&
+           h->pool->row(a)[0] == h->pool->row(b)[0];
+  };
+  int b0 = 0;
+  while (b0 + 1 < B && !(same_len(b0, b0 + 1) && same_page(b0, b0 + 1))) ++b0;
+  if (b0 + 1 >= B) return 1;
+  int g = 1;
+  while (b0 + g < B && same_len(b0, b0 + g) && same_page(b0, b0 + g)) ++g;
+  if (B % g || b0 % g) return 1;
+  int sharing = 0;
+  for (int k = 0; k < B; k += g) {
+    bool shares = true;
+    for (int j = 1; j < g; ++j) {
+      if (!same_len(k, k + j)) return 1;
+      shares = shares && same_page(k, k + j);
+    }
+    sharing += shares ? 1 : 0;
+  }
+  if (2 * sharing < B / g) return 1;
+  for (int gang = g; gang >= 2; --gang)
+    if (g % gang == 0 && gang <= h->sm_count && (h->sm_count % gang) * 10 <= h->sm_count) return gang;
+  return 1;
+}
+
 // Where the attention kernels keep their split partials; nullptr members select the arena.
 struct AttnScratch {
   float* o_part;
@@ -871,8 +906,16 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     ta.seq_tokens = seq_tokens;
     ta.page_table = h->paged() ? h->d_page_table(buf) : nullptr;
     ta.max_pages = dm.max_pages; ta.stride = dm.s;
-    const long long total = h->paged() ? ragged_tiles : (long long)B * ta.tiles_per_seq;
-    const int grid = (int)(total < h->sm_count ? total : h->sm_count);
+    long long total = h->paged() ? ragged_tiles : (long long)B * ta.tiles_per_seq;
+    // Beam search: consecutive sequences of equal length that start on the same page (the beams
+    // of one utterance) are walked by a gang of CTAs side by side (AttnTcArgs::gang).
+    const int gang = h->paged() ? beam_gang(h, B) : 1;
+    ta.n_list = B / gang;
+    h->last_gang = gang;
+    if (gang > 1) total = ragged_tiles / gang;              // tiles of the gangs' first sequences
+    const int grid_slots = h->sm_count / gang;              // whole gangs that fit the SMs
+    const int vctas = (int)(total < grid_slots ? total : grid_slots);
+    const int grid = vctas * gang;
     aa.n_split = 0;
     // A lock-step batch whose sequences are each spread over many CTAs hands the combine to a
     // launch of its own, one CTA per (head, sequence), instead of one CTA per sequence.
@@ -881,11 +924,12 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     ta.attn_grid = grid;
     const bool attn_pdl = pdl && !prof;     // the attention kernel is bracketed by events when timed
     if (h->paged()) {
-      if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, true>(h, ta, grid, st, attn_pdl)));
-      else MTLA_TRY((launch_attn_tc_rp<32, true>(h, ta, grid, st, attn_pdl)));
+      // (gang member, virtual CTA): members of a gang are neighbours in launch order.
+      if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, true>(h, ta, dim3(gang, vctas), st, attn_pdl)));
+      else MTLA_TRY((launch_attn_tc_rp<32, true>(h, ta, dim3(gang, vctas), st, attn_pdl)));
     } else {
-      if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, false>(h, ta, grid, st, attn_pdl)));
-      else MTLA_TRY((launch_attn_tc_rp<32, false>(h, ta, grid, st, attn_pdl)));
+      if (dm.nh <= 16) MTLA_TRY((launch_attn_tc_rp<16, false>(h, ta, dim3(grid), st, attn_pdl)));
+      else MTLA_TRY((launch_attn_tc_rp<32, false>(h, ta, dim3(grid), st, attn_pdl)));
     }
     MTLA_TRY(prof_mark(h, prof, 4, st));
     if (split_combine) {
@@ -1956,6 +2000,8 @@ int mtla_profile_end(mtla_handle* h, double* attention_ms, int32_t* steps) {
   if (rc == MTLA_OK) *attention_ms = stage_ms[MTLA_STAGE_ATTENTION];
   return rc;
 }
+
+int32_t mtla_attention_gang(const mtla_handle* h) { return h ? h->last_gang : 0; }
 
 const char* mtla_attention_variant(const mtla_handle* h) {
   return (h && h->use_tc) ? "tcgen05" : "fma";

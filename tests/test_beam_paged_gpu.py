@@ -25,9 +25,10 @@ def slots_of(tokens, s):
     return -(-tokens // s)
 
 
-def beam_search_against_oracle(w, n_utt, beam, lengths, steps, reorder_every=1):
+def beam_search_against_oracle(w, n_utt, beam, lengths, steps, reorder_every=1, want_gang=None):
     """Ragged prompts (one per utterance, copied to its `beam` hypotheses by a re-parenting),
-    then decode steps with a re-parenting in between; every output is compared."""
+    then decode steps with a re-parenting in between; every output is compared.  want_gang:
+    the gang size every decode step's attention launch must report."""
     weights = synth.make_weights(w)
     p = H.oracle_params(w, weights)
     n_seq = n_utt * beam
@@ -54,6 +55,8 @@ def beam_search_against_oracle(w, n_utt, beam, lengths, steps, reorder_every=1):
             want = np.stack([O.decode_step(p, states[b], x[b].double().numpy()) for b in range(n_seq)])
             H.assert_close(y, want, w.dtype, f"decode step {i}")
             assert M.mtla_seq_positions(h) == [st.tokens for st in states]
+            if want_gang is not None:
+                assert M.mtla_attention_gang(h) == want_gang, f"decode step {i}"
             if (i + 1) % reorder_every == 0:
                 parents = synth.beam_parents(w.seed, i, n_utt, beam)
                 M.mtla_beam_reorder(h, parents)
@@ -82,6 +85,30 @@ def test_beam_search_bf16_tensor_cores(s, heads):
     w = synth.WORKLOADS["paper"].scaled(stride=s, n_heads=heads, seed=30 + s)
     lengths = [PAGE * s * 2 + 3, 17, PAGE * s, 3 * PAGE * s - 1]
     beam_search_against_oracle(w, n_utt=4, beam=4, lengths=lengths, steps=40)
+
+
+@pytest.mark.parametrize("beam,gang,heads,s", [(4, 4, 8, 2), (8, 8, 32, 2), (5, 5, 8, 3), (50, 10, 8, 2),
+                                               (3, 3, 16, 1)])
+def test_beams_walk_shared_pages_as_a_gang(beam, gang, heads, s):
+    """Every utterance is longer than a page, so its beams share their first page and the
+    attention launch co-schedules them (gang = the largest divisor of the beam that leaves at
+    most a tenth of the SMs idle: 50 -> 10).  Utterances of different lengths: the gangs' shares
+    end inside and at the ends of sequences; the step count crosses a page boundary, where every
+    beam opens a page of its own."""
+    w = synth.WORKLOADS["paper"].scaled(stride=s, n_heads=heads, seed=40 + beam)
+    n_utt = 3 if beam < 50 else 2
+    lengths = [PAGE * s * 3 + 5, PAGE * s + 1, PAGE * s * 6 - 2 * s][:n_utt]
+    beam_search_against_oracle(w, n_utt=n_utt, beam=beam, lengths=lengths, steps=3 * s + 6,
+                               want_gang=gang)
+
+
+def test_gang_needs_most_blocks_to_share_their_first_page():
+    """One utterance shorter than a page (each beam copies and writes that page: nothing
+    shared) among longer ones keeps the gangs; a batch of mostly short utterances does not."""
+    w = synth.WORKLOADS["paper"].scaled(stride=2, seed=47)
+    beam_search_against_oracle(w, n_utt=3, beam=4, lengths=[PAGE * 2 * 2 + 3, 17, PAGE * 2 * 3],
+                               steps=5, want_gang=4)
+    beam_search_against_oracle(w, n_utt=3, beam=4, lengths=[9, 17, PAGE * 2 * 3], steps=5, want_gang=1)
 
 
 @pytest.mark.parametrize("name,kw", [("tiny", {}), ("paper", {"prefill_tokens": 300, "decode_steps": 140})])
