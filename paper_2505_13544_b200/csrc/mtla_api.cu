@@ -35,7 +35,9 @@ constexpr int kPlanSms = 148;
 constexpr int kTargetCtas = 2 * kPlanSms;   // CUDA-core attention: two CTAs per SM
 constexpr int kMinSlotsPerSplit = 64;
 constexpr int kFusedCombineMaxParts = 8;   // more parts per sequence: the combine gets its own launch
-constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill projections
+constexpr int kPrefillBn = 128;             // prompt rows per CTA in the prefill's output projection
+                                            // (its hi / lo halves are stacked: N = 256)
+constexpr int kPrefillBnWide = 256;         // and in its input and key / value projections
 // Layers whose pre-multiplied matrices W_Q W_K^T and W_V W_O (Eq. 12, taken literally) stay below
 // this size each keep them for the decode step: two launches fewer per step, which is what counts
 // where the whole layer lives in L2.  Larger layers keep the two-step form (the pre-multiplied
@@ -262,7 +264,7 @@ struct mtla_handle {
   CUtensorMap map_wcat_dec, map_wvo;   // folded decode weights
   CUtensorMap map_q16, map_o16, map_v16;
   int act_bn;               // box rows the three activation maps were encoded with (0: none yet)
-  unsigned gemm_attr_mask;  // kernel instances whose shared-memory limit has been raised
+  unsigned long long gemm_attr_mask;  // kernel instances whose shared-memory limit has been raised
   // Optional timing of the decode step's kernels: MTLA_DECODE_STAGES + 1 events per profiled step.
   std::vector<cudaEvent_t> prof_events;
   int prof_used;
@@ -438,10 +440,10 @@ template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false>
 int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
                         const GemmTcArgs& g, dim3 grid, cudaStream_t st, bool dependent) {
   constexpr int smem = gtc::smem_bytes(HILO ? 2 * BN : BN, STAGES);
-  if (!(h->gemm_attr_mask & (1u << inst))) {
+  if (!(h->gemm_attr_mask & (1ull << inst))) {
     MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    h->gemm_attr_mask |= 1u << inst;
+    h->gemm_attr_mask |= 1ull << inst;
   }
   MTLA_CUDA(launch_kernel(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS>, grid, dim3(192), smem, st,
                           dependent, ma, mb, g));
@@ -529,7 +531,12 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
     case 32: return launch_gemm_tc_inst<32, 4, OutT, false>(h, 2 + o, ma, mb, g, grid, st, dependent);
     case 64: return launch_gemm_tc_inst<64, 4, OutT, false>(h, 4 + o, ma, mb, g, grid, st, dependent);
     case 128: return launch_gemm_tc_inst<128, 3, OutT, false>(h, 6 + o, ma, mb, g, grid, st, dependent);
-    case 256: return launch_gemm_tc_inst<256, 4, OutT, false>(h, 8 + o, ma, mb, g, grid, st, dependent);
+    case 256:
+      // Prefill (many tiles, no split): two stages leave room for two CTAs per SM, whose epilogues
+      // and main loops overlap; the weight-streaming decode products want the deeper ring.
+      if (!allow_split)
+        return launch_gemm_tc_inst<256, 2, OutT, false>(h, 31 + o, ma, mb, g, grid, st, dependent);
+      return launch_gemm_tc_inst<256, 4, OutT, false>(h, 8 + o, ma, mb, g, grid, st, dependent);
     default: return MTLA_ERR_UNSUPPORTED_SHAPE;
   }
 }
@@ -998,10 +1005,10 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
     // Weights on the MMA's M side, 128 prompt rows per CTA on its N side: neighbouring CTAs
     // share an activation panel while the (small) weight matrix stays in L2.
     CUtensorMap map_x;
-    MTLA_TRY(make_map_2d(&map_x, x, rows, dm.d, dm.d, kPrefillBn));
+    MTLA_TRY(make_map_2d(&map_x, x, rows, dm.d, dm.d, kPrefillBnWide));
     MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x,
                             gemm_tc_args(h->at<float>(p.pf_p1), 1, dm.ntot, dm.ntot, rows, dm.d, 1.f),
-                            kPrefillBn, 1, false, st));
+                            kPrefillBnWide, 1, false, st));
   } else {
     MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot,
                                 dm.d, dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
@@ -1045,11 +1052,11 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
   // Eq. 9-10 on the running-state sequence: keys and values of every column.
   if (h->use_tc) {
     CUtensorMap map_c;
-    MTLA_TRY(make_map_2d(&map_c, h->at<void>(p.pf_cprime), rows, dm.r, dm.r, kPrefillBn));
+    MTLA_TRY(make_map_2d(&map_c, h->at<void>(p.pf_cprime), rows, dm.r, dm.r, kPrefillBnWide));
     // Keys and values as bf16, followed by their rounding remainders: rows of 4 n_h d_h.
     GemmTcArgs gkv = gemm_tc_args(h->at<bf16>(p.pf_kv), 1, 4 * hd, 2 * hd, rows, dm.r, 1.f);
     gkv.c_lo_off = 2 * hd;
-    MTLA_TRY(gemm_tc<bf16>(h, h->map_wkvt, map_c, gkv, kPrefillBn, 1, false, st));
+    MTLA_TRY(gemm_tc<bf16>(h, h->map_wkvt, map_c, gkv, kPrefillBnWide, 1, false, st));
     // Attention on the tensor cores; the closed slots are a strided view of the token rows.
     // d_h = 64: two query tiles per CTA over 64-slot key tiles (prefill_attn_tc2.cuh).
     const bool two_tiles = dm.dh == 64;

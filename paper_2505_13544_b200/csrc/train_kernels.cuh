@@ -231,14 +231,38 @@ __global__ void __launch_bounds__(256) gate_ln_backward_kernel(GateLnBackwardArg
 }
 
 // out[j] = sum_i a[i][j] * (b ? b[i][j] : 1) over `rows` rows of width n: LayerNorm gain / bias
-// and Linear bias gradients.  One thread per column, rows in order (deterministic).
-__global__ void __launch_bounds__(128) column_sum_kernel(const float* a, const float* b, float* out,
-                                                         long long rows, int n, long long ld) {
-  const int j = blockIdx.x * 128 + threadIdx.x;
-  if (j >= n) return;
+// and Linear bias gradients.  A CTA of 32 x 32 threads owns 32 columns: thread (x, y) adds rows
+// y, y + 32, ... of column x in order, then thread (x, 0) adds the 32 partial sums in order, so
+// the result does not depend on the launch.
+__global__ void __launch_bounds__(1024) column_sum_kernel(const float* a, const float* b, float* out,
+                                                          long long rows, int n, long long ld) {
+  __shared__ float part[32][33];
+  const int x = threadIdx.x, y = threadIdx.y;
+  const int j = blockIdx.x * 32 + x;
   float s = 0.f;
-  for (long long i = 0; i < rows; ++i) s += a[i * ld + j] * (b ? b[i * ld + j] : 1.f);
-  out[j] = s;
+  if (j < n)
+    for (long long i = y; i < rows; i += 32) s += a[i * ld + j] * (b ? b[i * ld + j] : 1.f);
+  part[y][x] = s;
+  __syncthreads();
+  if (y == 0 && j < n) {
+    float total = 0.f;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) total += part[k][x];
+    out[j] = total;
+  }
+}
+
+// out(i, j) = alpha * sum_s part[s][i * n + j] + beta * out(i, j), the partial products of a
+// reduction that was split over `splits` launches' worth of CTAs, added in split order.
+__global__ void __launch_bounds__(256) sum_splits_kernel(const float* part, int splits, long long count,
+                                                         int n, float* out, long long c_sm, long long c_sn,
+                                                         float alpha, float beta) {
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= count) return;
+  float s = 0.f;
+  for (int k = 0; k < splits; ++k) s += part[k * count + idx];
+  float* p = out + (idx / n) * c_sm + (idx % n) * c_sn;
+  *p = alpha * s + (beta != 0.f ? beta * *p : 0.f);
 }
 
 // Sinusoidal positional embedding rows pe_{j+1} (dimension r) for chunk j of every sequence:
