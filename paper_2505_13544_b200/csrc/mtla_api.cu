@@ -822,6 +822,11 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   const bool prof = h->prof_used + MTLA_DECODE_STAGES + 1 <= (int)h->prof_events.size();
   MTLA_TRY(prof_mark(h, prof, 0, st));
   const int bn = act_box_rows(B);
+  // On the tensor-core path every kernel is a programmatic dependent launch: its prologue
+  // overlaps the tail of its predecessor in the stream (the previous step's or layer's last
+  // kernel for the first one), and it waits before it touches any data.  Not while events sit
+  // between the kernels.
+  const bool pdl = h->use_tc && !(prof && !h->prof_attention_only);
   if (h->use_tc) {
     // a1 on the tensor cores: weights stream through the MMA's M side, the batch sits in N.
     MTLA_TRY(ensure_activation_maps(h, B));
@@ -830,7 +835,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     // With pre-multiplied weights the projection's query block is the absorbed query itself.
     const int n_out = dm.fold ? dm.ntot_dec : dm.ntot;
     MTLA_TRY(gemm_tc<float>(h, dm.fold ? h->map_wcat_dec : h->map_wcat, map_x,
-                            gemm_tc_args(h->at<float>(p.p1), 1, n_out, n_out, B, dm.d, 1.f), bn, 1, true, st));
+                            gemm_tc_args(h->at<float>(p.p1), 1, n_out, n_out, B, dm.d, 1.f), bn, 1, true, st,
+                            pdl));
   } else {
     MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d,
                                 dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
@@ -860,9 +866,6 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
-  // On the tensor-core path every kernel after the first is a programmatic dependent launch:
-  // its prologue overlaps the tail of its predecessor (not while events sit between them).
-  const bool pdl = h->use_tc && !(prof && !h->prof_attention_only);
   // Layers whose gate needs no matrix (folded form, or s = 1) take the latency-oriented kernel.
   const bool post_fast = dm.proj.off_u >= 0 || !pa.use_gate;
   if (h->use_tc) {

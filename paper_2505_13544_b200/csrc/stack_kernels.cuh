@@ -27,6 +27,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) row_norm_kernel(RowNormArgs a) {
   const int lane = threadIdx.x & 31;
   const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();   // the rows are the previous kernel's output
   if (row >= a.rows) return;
   float* res = a.res + row * a.d;
   const T* add = a.add ? static_cast<const T*>(a.add) + row * a.d : nullptr;
