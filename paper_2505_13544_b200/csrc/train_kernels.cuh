@@ -82,6 +82,103 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(GemmF32Args g) {
     }
 }
 
+// The same product on (16 TM) x (16 TN) output tiles, TM x TN outputs per thread (as two groups of
+// TM / 2 rows and TN / 2 columns, 16 TM / 2 and 16 TN / 2 apart, so that shared-memory reads are
+// 16-byte vectors without bank conflicts), the next 16 reduction steps fetched into registers
+// while the current ones are multiplied.  One accumulator per output, reduction in index order:
+// bit-identical to gemm_f32_kernel.  For products with at least 16 TM rows and 16 TN columns.
+template <int TM, int TN>
+__global__ void __launch_bounds__(256) gemm_f32_tiled_kernel(GemmF32Args g) {
+  constexpr int BM = 16 * TM, BN = 16 * TN, BK = 16, HM = TM / 2, HN = TN / 2;
+  static_assert(HM == 2 || HM == 4, "row groups are float2 / float4 reads");
+  static_assert(HN == 2 || HN == 4, "column groups are float2 / float4 reads");
+  __shared__ __align__(16) float as[2][BK][BM + 4];
+  __shared__ __align__(16) float bs[2][BK][BN + 4];
+  const int tid = threadIdx.x;
+  const int z = blockIdx.z, zo = z / g.z_inner, zi = z % g.z_inner;
+  const float* A = g.a + zi * g.a_z + zo * g.a_z2;
+  const float* B = g.b + zi * g.b_z + zo * g.b_z2;
+  float* C = g.c + zi * g.c_z + zo * g.c_z2;
+  const int i0 = blockIdx.y * BM, j0 = blockIdx.x * BN;
+  const int ty = tid / 16, tx = tid % 16;
+  const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
+  float acc[TM][TN];
+#pragma unroll
+  for (int x = 0; x < TM; ++x)
+#pragma unroll
+    for (int y = 0; y < TN; ++y) acc[x][y] = 0.f;
+  float ra[TM], rb[TN];
+  // Tile element e of this thread: (k, i) for A, (k, j) for B, walking the contiguous index.
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int e = 0; e < TM; ++e) {
+      const int idx = tid + e * 256;
+      const int kk = a_k_fast ? idx % BK : idx / BM, ii = a_k_fast ? idx / BK : idx % BM;
+      const int gi = i0 + ii, gk = k0 + kk;
+      ra[e] = (gi < g.m && gk < g.k) ? A[gi * g.a_sm + gk * g.a_sk] : 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < TN; ++e) {
+      const int idx = tid + e * 256;
+      const int jj = b_n_fast ? idx % BN : idx / BK, kk = b_n_fast ? idx / BN : idx % BK;
+      const int gj = j0 + jj, gk = k0 + kk;
+      rb[e] = (gj < g.n && gk < g.k) ? B[gk * g.b_sk + gj * g.b_sn] : 0.f;
+    }
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int e = 0; e < TM; ++e) {
+      const int idx = tid + e * 256;
+      const int kk = a_k_fast ? idx % BK : idx / BM, ii = a_k_fast ? idx / BK : idx % BM;
+      as[buf][kk][ii] = ra[e];
+    }
+#pragma unroll
+    for (int e = 0; e < TN; ++e) {
+      const int idx = tid + e * 256;
+      const int jj = b_n_fast ? idx % BN : idx / BK, kk = b_n_fast ? idx / BN : idx % BK;
+      bs[buf][kk][jj] = rb[e];
+    }
+  };
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < g.k; k0 += BK) {
+    const bool more = k0 + BK < g.k;
+    if (more) fetch(k0 + BK);
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float a8[TM], b8[TN];
+#pragma unroll
+      for (int hlf = 0; hlf < 2; ++hlf) {
+#pragma unroll
+        for (int x = 0; x < HM; ++x) a8[hlf * HM + x] = as[buf][kk][hlf * (BM / 2) + ty * HM + x];
+#pragma unroll
+        for (int y = 0; y < HN; ++y) b8[hlf * HN + y] = bs[buf][kk][hlf * (BN / 2) + tx * HN + y];
+      }
+#pragma unroll
+      for (int x = 0; x < TM; ++x)
+#pragma unroll
+        for (int y = 0; y < TN; ++y) acc[x][y] = fmaf(a8[x], b8[y], acc[x][y]);
+    }
+    if (more) {
+      stash(buf ^ 1);       // the other buffer was last read before the previous barrier
+      __syncthreads();
+      buf ^= 1;
+    }
+  }
+#pragma unroll
+  for (int x = 0; x < TM; ++x)
+#pragma unroll
+    for (int y = 0; y < TN; ++y) {
+      const int gi = i0 + (x / HM) * (BM / 2) + ty * HM + x % HM;
+      const int gj = j0 + (y / HN) * (BN / 2) + tx * HN + y % HN;
+      if (gi >= g.m || gj >= g.n) continue;
+      float* p = C + gi * g.c_sm + gj * g.c_sn;
+      *p = g.alpha * acc[x][y] + (g.beta != 0.f ? g.beta * *p : 0.f);
+    }
+}
+
 // Row m of a score matrix S [T][T] (log2 units, one matrix per blockIdx.y): softmax under the
 // stride-aware causal mask of Section 4.2 (column n allowed iff n == m, or n < m and
 // (n + 1) mod s == 0 for 0-based m, n), in place.  One warp per row, 8 rows per CTA.

@@ -36,6 +36,9 @@ def layer(d, nh, dh, r, dr, dw, stride, batch, t_len, seed=81):
     (96, 2, 64, 128, 32, 24, 3, 3, 70),      # several 64-wide tiles of every product, ragged
     (128, 2, 128, 64, 64, 8, 4, 1, 130),     # d_h 128, d_R 64
     (64, 4, 64, 64, 32, 16, 1, 2, 33),       # s = 1: no gate, zero hyper-network gradients
+    (128, 8, 64, 128, 32, 16, 2, 10, 250),   # enough tiles for the 128 x 128 and 128 x 64 kernels, ragged
+                                             # edges in both; weight gradients summed in 4 pieces
+    (64, 2, 64, 64, 32, 16, 2, 2, 256),      # 512 rows: weight gradients in 8 pieces of 64 rows
 ])
 def test_forward_and_backward_match_the_training_oracle(d, nh, dh, r, dr, dw, stride, batch, t_len):
     w = layer(d, nh, dh, r, dr, dw, stride, batch, t_len)
