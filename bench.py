@@ -817,7 +817,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--workload", default="large",
                     choices=sorted(synth.WORKLOADS) + sorted(synth.BEAM_WORKLOADS)
-                    + sorted(synth.STACK_WORKLOADS))
+                    + sorted(synth.STACK_WORKLOADS) + ["train_paper_fp32"])
     ap.add_argument("--compare", action="store_true",
                     help="time MHA / GQA / MQA / MLA / MTLA at the workload's width, batch and one context")
     ap.add_argument("--paged", action="store_true",
@@ -834,7 +834,8 @@ def main() -> None:
                     help="override the workload's imported context length")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.workload in synth.BEAM_WORKLOADS or args.workload in synth.STACK_WORKLOADS:
+        if (args.workload in synth.BEAM_WORKLOADS or args.workload in synth.STACK_WORKLOADS
+                or args.workload == "train_paper_fp32"):
             raise SystemExit("--impl reference covers the decode workloads")
         run_reference(args)
         return
@@ -864,6 +865,22 @@ def main() -> None:
         if world > 1:
             raise SystemExit("the beam workloads run on one GPU")
         run_beam(args, synth.BEAM_WORKLOADS[args.workload], device, local)
+        return
+    if args.workload == "train_paper_fp32":
+        # The training path alone (the `training` block of the default run): forward + backward.
+        if world > 1:
+            raise SystemExit("the training workload runs on one GPU")
+        with ClockSampler(local) as clocks:
+            res = time_training(device, runs=max(args.steps, 3) if args.steps < 16 else 3,
+                                cpu_baseline=not args.no_cpu_baseline)
+        ms = res["forward_ms"] + res["backward_ms"]
+        print(json.dumps({"metric": "mtla_train_tokens_per_s", "value": res["tokens_per_s"], "unit": UNIT,
+                          "n_gpus": 1, "steps": 3, "warmup": 1, "ms_per_step": ms, "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                          "config": {"workload": res["workload"], "batch": res["batch"],
+                                     "tokens": res["tokens"], "step": "forward + backward"},
+                          "roofline": res["roofline"], "training": res,
+                          "gpu_launches": res["gpu_launches"], "clocks": clocks.summary()}))
         return
     if args.workload in synth.STACK_WORKLOADS:
         if world > 1:

@@ -466,8 +466,10 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   const bool hilo = g.b_lo_col > 0 && bn <= 128 && sizeof(OutT) == 2;
   const int slots = (hilo && bn == 128) || bn == 256 ? h->sm_count : 2 * h->sm_count;
   int n_split = 1;
-  // The partials are summed by the last CTA of a tile alone: at most four splits keep that short.
-  if (allow_split && tiles < slots) n_split = max(1, min(min(kb_total / 4, (int)(slots / tiles)), 4));
+  // The partials are summed by the last CTA of a tile alone: at most four splits keep that short
+  // (eight where a product has so few tiles that four splits would still leave it on <= 32 CTAs).
+  if (allow_split && tiles < slots)
+    n_split = max(1, min(min(kb_total / 4, (int)(slots / tiles)), tiles <= 8 ? 8 : 4));
   // Short reductions with few activation rows (the paper's layer: K = 512, B <= 64): one CTA per
   // tile with the whole K range in flight at once beats splitting it, which costs a trip of the
   // partials through global memory on top of two load round trips.
