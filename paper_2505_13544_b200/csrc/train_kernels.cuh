@@ -277,12 +277,33 @@ __global__ void __launch_bounds__(256) gate_ln_backward_kernel(GateLnBackwardArg
     __syncthreads();
     float w = 1.f, dz = 0.f;
     if (a.use_gate) {
+      // Linear(c): the r rows of A are cut into 256 / d_w ranges so that every thread works;
+      // the ranges' sums are added in range order (part_s aliases dc_s, written only later).
       float prod = 0.f;
-      for (int n = tid; n < a.dw; n += 256) {
-        float hn = a.hyp_c_b[n];
-        for (int i = 0; i < a.r; ++i) hn = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], hn);
-        h_s[n] = hn;
-        prod += hn * g[n];
+      const int parts = a.dw <= 128 ? 256 / a.dw : 1;
+      if (parts > 1) {
+        float* part_s = dc_s;                      // parts * d_w <= 256 floats
+        const int n = tid % a.dw, pt = tid / a.dw;
+        if (pt < parts) {
+          const int per = (a.r + parts - 1) / parts, lo = pt * per, hi = min(a.r, lo + per);
+          float hn = 0.f;
+          for (int i = lo; i < hi; ++i) hn = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], hn);
+          part_s[pt * a.dw + n] = hn;
+        }
+        __syncthreads();
+        if (tid < a.dw) {
+          float hn = a.hyp_c_b[tid];
+          for (int pt2 = 0; pt2 < parts; ++pt2) hn += part_s[pt2 * a.dw + tid];
+          h_s[tid] = hn;
+          prod = hn * g[tid];
+        }
+      } else {
+        for (int n = tid; n < a.dw; n += 256) {
+          float hn = a.hyp_c_b[n];
+          for (int i = 0; i < a.r; ++i) hn = fmaf(c_s[i], a.hyp_c_w[(long long)i * a.dw + n], hn);
+          h_s[n] = hn;
+          prod += hn * g[n];
+        }
       }
       const float logit = block_sum(prod, red_s);
       w = 1.f / (1.f + expf(-logit));
