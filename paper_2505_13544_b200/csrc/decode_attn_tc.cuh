@@ -113,8 +113,6 @@ static_assert(kFirstSoftmaxWarp % 4 == 0 && kThreads == kFirstSoftmaxWarp * 32 +
               "softmax warps must start at a warpgroup boundary");
 constexpr int kSubBytes = kTile * 128;     // one 64-column sub-tile
 constexpr int kPairBytes = 2 * kSubBytes;
-constexpr int kPairs = 9;
-constexpr int kKrBufs = 3;
 constexpr int kPrefetchAhead = 1;          // tiles asked into L2 ahead of the tile being loaded
 constexpr int kTmemCols = 512;
 constexpr int kSParts = 4;                 // independent partial score accumulators per buffer
@@ -123,28 +121,40 @@ constexpr int kColO = 2 * kSParts * 32;    // output blocks at 256 + 32 * block
 constexpr float kRescaleThreshold = 8.f;
 constexpr int kSmCountMax = 256;           // upper bound on the attention grid (one CTA per SM)
 
-constexpr int kOffPairs = 0;
-constexpr int kOffKr = kPairs * kPairBytes;
-constexpr int kOffQ = kOffKr + kKrBufs * kSubBytes;
 constexpr int kMaxQBytes = 9 * 32 * 128;   // (2 * 4 + 1) chunks x 32 heads x 128 B
-constexpr int kOffP = kOffQ + kMaxQBytes;
 constexpr int kPBytes = 32 * kTile * 2;    // one probability buffer
-constexpr int kOffMisc = kOffP + 2 * kPBytes;
 constexpr int kMiscBytes = 4096;
-constexpr int kSmemBytes = kOffMisc + kMiscBytes + 1024;  // + slack for 1024-byte alignment
-static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 // Ragged batches add the tile prefix sums of up to kMaxRaggedBatch sequences and the page
 // numbers of the first kStagedPages tiles of the CTA's share.
 constexpr int kMaxRaggedBatch = 1022;
 constexpr int kStagedPages = 1024;
-constexpr int kOffPrefix = kOffMisc + kMiscBytes;
-constexpr int kOffStaged = kOffPrefix + (kMaxRaggedBatch + 2) * 4;
-constexpr int kSmemBytesRagged = kOffStaged + kStagedPages * 4 + 1024;
-static_assert(kSmemBytesRagged <= 227 * 1024, "shared memory budget (ragged)");
+constexpr int kMaxPairs = 10, kMaxKrBufs = 3;
+
+// Shared-memory layout.  The ring of latent pairs is what bounds the tiles in flight, and the time
+// of a tile follows the ring's depth (measured at the largest workload: 8 / 9 / 10 pairs = 428 /
+// 417 / 410 us), so lock-step batches spend the 8 KB that ragged ones need for their lists, and
+// one of the three RoPE-key buffers (a RoPE-key buffer is free again as soon as its tile's first
+// score MMA has been issued), on a tenth pair.
+template <bool RAGGED>
+struct Layout {
+  static constexpr int kPairs = RAGGED ? 9 : 10;
+  static constexpr int kKrBufs = RAGGED ? 3 : 2;
+  static constexpr int kOffPairs = 0;
+  static constexpr int kOffKr = kPairs * kPairBytes;
+  static constexpr int kOffQ = kOffKr + kKrBufs * kSubBytes;
+  static constexpr int kOffP = kOffQ + kMaxQBytes;
+  static constexpr int kOffMisc = kOffP + 2 * kPBytes;
+  static constexpr int kOffPrefix = kOffMisc + kMiscBytes;
+  static constexpr int kOffStaged = kOffPrefix + (kMaxRaggedBatch + 2) * 4;
+  // + slack for 1024-byte alignment
+  static constexpr int kSmemBytes = (RAGGED ? kOffStaged + kStagedPages * 4 : kOffPrefix) + 1024;
+  static_assert(kPairs <= kMaxPairs && kKrBufs <= kMaxKrBufs, "barrier arrays too small");
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+};
 
 struct Misc {
-  unsigned long long full_pair[kPairs], empty_pair[kPairs];
-  unsigned long long full_kr[kKrBufs], empty_kr[kKrBufs];
+  unsigned long long full_pair[kMaxPairs], empty_pair[kMaxPairs];
+  unsigned long long full_kr[kMaxKrBufs], empty_kr[kMaxKrBufs];
   unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], q_full, q_empty;
   unsigned long long flag_bar[2], group_sync;
   uint32_t tmem_base;
@@ -223,6 +233,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
 decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
                       const __grid_constant__ CUtensorMap q_map, AttnTcArgs a) {
   using namespace tc;
+  using L = Layout<RAGGED>;
   using namespace ptx;
   constexpr int NCH = 2 * RP + 1;                // 64-column chunks of q~ (latent + RoPE)
   constexpr uint32_t QCHUNK = NHP * 128;         // bytes of one q~ chunk
@@ -234,18 +245,18 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
-  Misc* misc = reinterpret_cast<Misc*>(sm + kOffMisc);
+  Misc* misc = reinterpret_cast<Misc*>(sm + L::kOffMisc);
   volatile int* abort_word = &misc->abort_word;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   auto bar = [&](unsigned long long* p) { return smem_u32(p); };
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kPairs; ++i) {
+    for (int i = 0; i < L::kPairs; ++i) {
       mbar_init(bar(&misc->full_pair[i]), 1);
       mbar_init(bar(&misc->empty_pair[i]), 1);
     }
-    for (int i = 0; i < kKrBufs; ++i) {
+    for (int i = 0; i < L::kKrBufs; ++i) {
       mbar_init(bar(&misc->full_kr[i]), 1);
       mbar_init(bar(&misc->empty_kr[i]), kQkIssuers);
     }
@@ -279,7 +290,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   grid_dependency_wait();        // nothing before this line touches the previous kernel's data
 
   // This CTA's share of the tile list.
-  const uint32_t prefix_s = base + kOffPrefix, staged_s = base + kOffStaged;   // ragged only
+  const uint32_t prefix_s = base + L::kOffPrefix, staged_s = base + L::kOffStaged;   // ragged only
   long long total = (long long)a.batch * a.tiles_per_seq;
   // Lock-step batches: a 1-D grid.  Ragged ones: (gang member, virtual CTA), all of them special
   // registers, so that no thread carries them through its loop.
@@ -288,7 +299,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   const int n_list = RAGGED ? a.n_list : a.batch;   // entries of the tile list (sequences or gangs)
   if constexpr (RAGGED) {
     // prefix[b] = tiles of the sequences before b; prefix[batch + 1] repeats the total.
-    int* prefix = reinterpret_cast<int*>(sm + kOffPrefix);
+    int* prefix = reinterpret_cast<int*>(sm + L::kOffPrefix);
     for (int i = threadIdx.x; i < n_list; i += kThreads)
       prefix[i + 1] = ceil_div(ceil_div(a.seq_tokens[i * gang], a.stride), kTile);
     __syncthreads();
@@ -322,7 +333,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
   const int n_tiles = (int)(g1 - g0);
   const int tps_u = a.tiles_per_seq;
   if constexpr (RAGGED) {
-    int* staged = reinterpret_cast<int*>(sm + kOffStaged);
+    int* staged = reinterpret_cast<int*>(sm + L::kOffStaged);
     for (int n = threadIdx.x; n < min(n_tiles, kStagedPages); n += kThreads) {
       TileCursor<true> c;
       c.locate(g0 + n, 0, prefix_s, n_list);
@@ -331,8 +342,8 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
     __syncthreads();
   }
 
-  const uint32_t pairs_u32 = base + kOffPairs, kr_u32 = base + kOffKr;
-  const uint32_t q_u32 = base + kOffQ, p_u32 = base + kOffP;
+  const uint32_t pairs_u32 = base + L::kOffPairs, kr_u32 = base + L::kOffKr;
+  const uint32_t q_u32 = base + L::kOffQ, p_u32 = base + L::kOffP;
 
   if (warp < kFirstSoftmaxWarp) {
   // Register budget: the producer / issuer warpgroups keep 40 registers, the softmax ones get 176.
@@ -381,16 +392,16 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       }
       int slot, plane;
       tile_coords(cur, n, slot, plane);
-      const int kb = n % kKrBufs;
-      ok = mbar_wait(bar(&misc->empty_kr[kb]), ((n / kKrBufs) & 1) ^ 1, abort_word, a.error_word, 2);
+      const int kb = n % L::kKrBufs;
+      ok = mbar_wait(bar(&misc->empty_kr[kb]), ((n / L::kKrBufs) & 1) ^ 1, abort_word, a.error_word, 2);
       if (!ok) break;
       misc->tile_flags[n & 15] = ((n == 0 || cur.seq_first()) ? 1 : 0) |
                                  ((n + 1 == n_tiles || cur.seq_last()) ? 2 : 0);
       mbar_arrive_expect_tx(bar(&misc->full_kr[kb]), kSubBytes);
       tma_load_3d(kr_u32 + kb * kSubBytes, &cache_map, bar(&misc->full_kr[kb]), a.r, slot, plane);
       for (int c = 0; c < RP && ok; ++c, ++pc) {
-        const int buf = pc % kPairs;
-        ok = mbar_wait(bar(&misc->empty_pair[buf]), ((pc / kPairs) & 1) ^ 1, abort_word,
+        const int buf = pc % L::kPairs;
+        ok = mbar_wait(bar(&misc->empty_pair[buf]), ((pc / L::kPairs) & 1) ^ 1, abort_word,
                        a.error_word, 3);
         if (!ok) break;
         const uint32_t dst = pairs_u32 + buf * kPairBytes;
@@ -412,9 +423,9 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
         const uint64_t bd = make_smem_desc(q_u32 + chunk * QCHUNK + k * 32, 16, 1024, kSwizzle128B);
         mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, accumulate);
       };
-      const int kb = n % kKrBufs;
+      const int kb = n % L::kKrBufs;
       ok = mbar_wait(bar(&misc->s_empty[n & 1]), ((n >> 1) & 1) ^ 1, abort_word, a.error_word, 9) &&
-           mbar_wait(bar(&misc->full_kr[kb]), (n / kKrBufs) & 1, abort_word, a.error_word, 10);
+           mbar_wait(bar(&misc->full_kr[kb]), (n / L::kKrBufs) & 1, abort_word, a.error_word, 10);
       if (!ok) break;
       const int flags = *reinterpret_cast<volatile int*>(&misc->tile_flags[n & 15]);
       const bool seg_last = flags & 2;
@@ -427,8 +438,8 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       qk(kr_u32 + kb * kSubBytes, 2 * RP, 0u);
       mma_commit(bar(&misc->empty_kr[kb]));
       for (int c = 0; c < RP && ok; ++c) {
-        const int pcn = n * RP + c, buf = pcn % kPairs;
-        ok = mbar_wait(bar(&misc->full_pair[buf]), (pcn / kPairs) & 1, abort_word, a.error_word, 11);
+        const int pcn = n * RP + c, buf = pcn % L::kPairs;
+        ok = mbar_wait(bar(&misc->full_pair[buf]), (pcn / L::kPairs) & 1, abort_word, a.error_word, 11);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t src = pairs_u32 + buf * kPairBytes;
@@ -451,7 +462,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       tc_fence_after_sync();
       const bool seg_first = *reinterpret_cast<volatile int*>(&misc->pv_first[n & 1]) != 0;
       for (int mb = j; mb < RP; mb += kPvIssuers) {
-        const int buf = (n * RP + mb) % kPairs;
+        const int buf = (n * RP + mb) % L::kPairs;
         const uint32_t src = pairs_u32 + buf * kPairBytes;
 #pragma unroll
         for (int ks = 0; ks < kTile / 16; ++ks) {
@@ -602,7 +613,7 @@ decode_attn_tc_kernel(const __grid_constant__ CUtensorMap cache_map,
       // P^T as the K-major, un-swizzled B operand of the value MMA: element (head h, slot k)
       // at (h/8)*PSBO + (k/8)*128 + (h%8)*16 + (k%8)*2.
       auto store_probabilities = [&]() {
-        uint8_t* prow = sm + kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
+        uint8_t* prow = sm + L::kOffP + (n & 1) * kPBytes + (row >> 3) * 128 + (row & 7) * 2;
 #pragma unroll
         for (int i = 0; i < NQ; ++i) {
           const int h = HQ + i;

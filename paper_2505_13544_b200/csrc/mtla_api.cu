@@ -553,7 +553,7 @@ GemmTcArgs gemm_tc_args(void* c, long long c_sm, long long c_sn, int m, int n, i
 
 template <int NHP, bool RAGGED>
 int launch_attn_tc_rp(mtla_handle* h, const AttnTcArgs& a, dim3 grid, cudaStream_t st, bool dependent) {
-  constexpr int kSmem = RAGGED ? tc::kSmemBytesRagged : tc::kSmemBytes;
+  constexpr int kSmem = tc::Layout<RAGGED>::kSmemBytes;
 #define MTLA_TC_CASE(RP)                                                                       \
   case RP:                                                                                     \
     if (!h->attn_smem_ready) {                                                                 \
