@@ -23,10 +23,11 @@
 // goes to partial ks, each partial has its own issuing thread (see below), and the softmax
 // threads add the four when they read them.
 //
-// Shared memory: a ring of nine 16 KB "pairs" (two adjacent sub-tiles = a 128-row MN-major
-// operand block), three 8 KB sub-tiles for the RoPE-key columns, q~ as a K-major swizzled B
-// operand (TMA-loaded per segment), and two bf16 probability buffers.  The ring holds a little
-// more than two tiles, and a load can only be issued once its slot is free; to keep the DRAM
+// Shared memory: a ring of ten 16 KB "pairs" (two adjacent sub-tiles = a 128-row MN-major
+// operand block) and two 8 KB sub-tiles for the RoPE-key columns (nine and three for ragged
+// batches, see Layout), q~ as a K-major swizzled B operand (TMA-loaded per segment), and two
+// bf16 probability buffers.  The ring holds a little more than two tiles, and a load can only
+// be issued once its slot is free; to keep the DRAM
 // latency off that path the producer also asks the tile after the one it is loading into L2
 // (cp.async.bulk.prefetch), so the load proper is an L2 hit.
 //
