@@ -353,7 +353,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const float sum[4] = {acc[u].x, acc[u].y, acc[u].z, acc[u].w};
               OutT* p = c + (long long)j * g.c_sn + (long long)i0 * g.c_sm;
               if (g.vec4_ok) {
-                const float val[4] = {g.alpha * sum[0], g.alpha * sum[1], g.alpha * sum[2], g.alpha * sum[3]};
+                float val[4] = {g.alpha * sum[0], g.alpha * sum[1], g.alpha * sum[2], g.alpha * sum[3]};
+                if constexpr (EXTRAS) {
+                  // Four consecutive output features: bias and residual as 16-byte vectors too.
+                  if (g.bias) {
+                    const float4 b4 = *reinterpret_cast<const float4*>(g.bias + i0);
+                    val[0] += b4.x; val[1] += b4.y; val[2] += b4.z; val[3] += b4.w;
+                  }
+                  if (g.relu) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) val[e] = fmaxf(val[e], 0.f);
+                  }
+                  if (g.residual) {
+                    const float4 r4 = *reinterpret_cast<const float4*>(g.residual + i0 + (long long)j * g.r_sn);
+                    val[0] += r4.x; val[1] += r4.y; val[2] += r4.z; val[3] += r4.w;
+                  }
+                }
                 store4(p, val, g.c_lo_off);
               } else {
 #pragma unroll

@@ -486,7 +486,14 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
   if ((long long)m_tiles * g.n_tiles * g.n_split > 0x7fffffffll) return MTLA_ERR_UNSUPPORTED_SHAPE;
   g.vec4_ok = g.c_sm == 1 && g.m % 4 == 0 && reinterpret_cast<uintptr_t>(g.c) % 16 == 0 &&
               g.c_sn * osz % 16 == 0 && g.c_sz * osz % 16 == 0 && g.c_lo_off * osz % 8 == 0;
-  if (g.bias || g.residual || g.relu) g.vec_ok = g.vec4_ok = 0;   // the epilogue extras are scalar
+  if (g.bias || g.residual || g.relu) {
+    // The unsplit epilogue applies the extras one element at a time; the split reduction takes
+    // four consecutive output features at once where bias and residual allow 16-byte reads.
+    g.vec_ok = 0;
+    g.vec4_ok = g.vec4_ok && (!g.bias || reinterpret_cast<uintptr_t>(g.bias) % 16 == 0) &&
+                (!g.residual || (g.r_sm == 1 && g.r_sn % 4 == 0 &&
+                                 reinterpret_cast<uintptr_t>(g.residual) % 16 == 0));
+  }
   dim3 grid(m_tiles * g.n_tiles * g.n_split, 1, batches);
   constexpr int o = sizeof(OutT) == 4 ? 0 : 1;
   if (g.bias || g.residual || g.relu) {
