@@ -26,6 +26,8 @@ struct GemmF32Args {
   int z_inner;                  // z = z_outer * z_inner + z_in: a second level of offsets
   long long a_z2, b_z2, c_z2;   //   applied to z_outer (e.g. sequence over head)
   float alpha, beta;
+  int c_vec;                    // 1: c_sn == 1 and every row start, z offset and n keep 16-byte alignment
+                                // (the tiled kernel then stores four adjacent columns at once)
 };
 
 // 64 x 64 output tile per CTA of 256 threads, 16 reduction steps per stage, 4 x 4 outputs per
@@ -86,7 +88,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(GemmF32Args g) {
 // TM / 2 rows and TN / 2 columns, 16 TM / 2 and 16 TN / 2 apart, so that shared-memory reads are
 // 16-byte vectors without bank conflicts), the next 16 reduction steps fetched into registers
 // while the current ones are multiplied.  One accumulator per output, reduction in index order:
-// bit-identical to gemm_f32_kernel.  For products with at least 16 TM rows and 16 TN columns.
+// the same sums as gemm_f32_kernel.  For products with at least 16 TM rows and 16 TN columns.
 template <int TM, int TN>
 __global__ void __launch_bounds__(256) gemm_f32_tiled_kernel(GemmF32Args g) {
   constexpr int BM = 16 * TM, BN = 16 * TN, BK = 16, HM = TM / 2, HN = TN / 2;
@@ -168,15 +170,34 @@ __global__ void __launch_bounds__(256) gemm_f32_tiled_kernel(GemmF32Args g) {
     }
   }
 #pragma unroll
-  for (int x = 0; x < TM; ++x)
+  for (int x = 0; x < TM; ++x) {
+    const int gi = i0 + (x / HM) * (BM / 2) + ty * HM + x % HM;
+    if (gi >= g.m) continue;
+    if (HN == 4 && g.c_vec) {
+      // The thread's columns come in runs of four adjacent ones: one 16-byte access each.
+#pragma unroll
+      for (int yh = 0; yh < 2; ++yh) {
+        const int gj = j0 + yh * (BN / 2) + tx * HN;
+        if (gj >= g.n) continue;                       // n is a multiple of 4: whole runs only
+        float4* p = reinterpret_cast<float4*>(C + gi * g.c_sm + gj);
+        float4 v = make_float4(g.alpha * acc[x][yh * HN], g.alpha * acc[x][yh * HN + 1],
+                               g.alpha * acc[x][yh * HN + 2], g.alpha * acc[x][yh * HN + 3]);
+        if (g.beta != 0.f) {
+          const float4 o = *p;
+          v.x += g.beta * o.x; v.y += g.beta * o.y; v.z += g.beta * o.z; v.w += g.beta * o.w;
+        }
+        *p = v;
+      }
+      continue;
+    }
 #pragma unroll
     for (int y = 0; y < TN; ++y) {
-      const int gi = i0 + (x / HM) * (BM / 2) + ty * HM + x % HM;
       const int gj = j0 + (y / HN) * (BN / 2) + tx * HN + y % HN;
-      if (gi >= g.m || gj >= g.n) continue;
+      if (gj >= g.n) continue;
       float* p = C + gi * g.c_sm + gj * g.c_sn;
       *p = g.alpha * acc[x][y] + (g.beta != 0.f ? g.beta * *p : 0.f);
     }
+  }
 }
 
 // Row m of a score matrix S [T][T] (log2 units, one matrix per blockIdx.y): softmax under the
@@ -224,6 +245,8 @@ struct GateLnBackwardArgs {
   const float* gamma;
   const float* beta;
   const float* hyp_c_w;   // [r][d_w]
+  const float* hyp_c_wt;  // [d_w][r]: the same matrix transposed, so that the reverse product's reads
+                          // (one thread per latent column) coalesce as the forward product's do
   const float* hyp_c_b;   // [d_w]
   const float* gate_pe;   // [max_slots][d_w]: Linear(pe_j) per chunk
   const float* dcprime;   // [rows][r] gradient of the running merge states (Eq. 14's sequence)
@@ -324,7 +347,7 @@ __global__ void __launch_bounds__(256) gate_ln_backward_kernel(GateLnBackwardArg
       float d = w * suf_s[i];
       if (a.use_gate) {
         float t = 0.f;
-        for (int n = 0; n < a.dw; ++n) t = fmaf(dh_s[n], a.hyp_c_w[(long long)i * a.dw + n], t);
+        for (int n = 0; n < a.dw; ++n) t = fmaf(dh_s[n], a.hyp_c_wt[(long long)n * a.r + i], t);
         d += t;
       }
       dc_s[i] = d;
