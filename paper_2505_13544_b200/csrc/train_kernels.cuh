@@ -26,6 +26,11 @@ struct GemmF32Args {
   int z_inner;                  // z = z_outer * z_inner + z_in: a second level of offsets
   long long a_z2, b_z2, c_z2;   //   applied to z_outer (e.g. sequence over head)
   float alpha, beta;
+  int causal;                   // square products of the causal attention (row m sees columns n <= m):
+                                // 1: output tiles wholly above the diagonal are skipped (their
+                                //    consumers never read them); 2: A(i, k) is zero for k < i, the
+                                //    reduction starts at the tile's first row; 3: A(i, k) is zero for
+                                //    k > i, it ends after the tile's last row.  0: a full product.
   int c_vec;                    // 1: c_sn == 1 and every row start, z offset and n keep 16-byte alignment
                                 // (the tiled kernel then stores four adjacent columns at once)
 };
@@ -42,6 +47,9 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(GemmF32Args g) {
   const float* B = g.b + zi * g.b_z + zo * g.b_z2;
   float* C = g.c + zi * g.c_z + zo * g.c_z2;
   const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+  if (g.causal == 1 && j0 > i0 + 63) return;
+  const int k_begin = g.causal == 2 ? i0 / 16 * 16 : 0;
+  const int k_end = g.causal == 3 ? min(g.k, i0 + 64) : g.k;
   const int ti = (tid / 16) * 4, tj = (tid % 16) * 4;
   float acc[4][4];
 #pragma unroll
@@ -49,16 +57,16 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(GemmF32Args g) {
 #pragma unroll
     for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
   const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
-  for (int k0 = 0; k0 < g.k; k0 += 16) {
+  for (int k0 = k_begin; k0 < k_end; k0 += 16) {
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const int idx = tid + t * 256;
       const int kk = a_k_fast ? idx % 16 : idx / 64, ii = a_k_fast ? idx / 16 : idx % 64;
       const int gi = i0 + ii, gk = k0 + kk;
-      as[kk][ii] = (gi < g.m && gk < g.k) ? A[gi * g.a_sm + gk * g.a_sk] : 0.f;
+      as[kk][ii] = (gi < g.m && gk < k_end) ? A[gi * g.a_sm + gk * g.a_sk] : 0.f;
       const int jj = b_n_fast ? idx % 64 : idx / 16, kb = b_n_fast ? idx / 64 : idx % 16;
       const int gj = j0 + jj, gkb = k0 + kb;
-      bs[kb][jj] = (gj < g.n && gkb < g.k) ? B[gkb * g.b_sk + gj * g.b_sn] : 0.f;
+      bs[kb][jj] = (gj < g.n && gkb < k_end) ? B[gkb * g.b_sk + gj * g.b_sn] : 0.f;
     }
     __syncthreads();
 #pragma unroll
@@ -102,6 +110,9 @@ __global__ void __launch_bounds__(256) gemm_f32_tiled_kernel(GemmF32Args g) {
   const float* B = g.b + zi * g.b_z + zo * g.b_z2;
   float* C = g.c + zi * g.c_z + zo * g.c_z2;
   const int i0 = blockIdx.y * BM, j0 = blockIdx.x * BN;
+  if (g.causal == 1 && j0 > i0 + BM - 1) return;
+  const int k_begin = g.causal == 2 ? i0 / BK * BK : 0;
+  const int k_end = g.causal == 3 ? min(g.k, i0 + BM) : g.k;
   const int ty = tid / 16, tx = tid % 16;
   const bool a_k_fast = g.a_sk == 1, b_n_fast = g.b_sn == 1;
   float acc[TM][TN];
@@ -117,14 +128,14 @@ __global__ void __launch_bounds__(256) gemm_f32_tiled_kernel(GemmF32Args g) {
       const int idx = tid + e * 256;
       const int kk = a_k_fast ? idx % BK : idx / BM, ii = a_k_fast ? idx / BK : idx % BM;
       const int gi = i0 + ii, gk = k0 + kk;
-      ra[e] = (gi < g.m && gk < g.k) ? A[gi * g.a_sm + gk * g.a_sk] : 0.f;
+      ra[e] = (gi < g.m && gk < k_end) ? A[gi * g.a_sm + gk * g.a_sk] : 0.f;
     }
 #pragma unroll
     for (int e = 0; e < TN; ++e) {
       const int idx = tid + e * 256;
       const int jj = b_n_fast ? idx % BN : idx / BK, kk = b_n_fast ? idx / BN : idx % BK;
       const int gj = j0 + jj, gk = k0 + kk;
-      rb[e] = (gj < g.n && gk < g.k) ? B[gk * g.b_sk + gj * g.b_sn] : 0.f;
+      rb[e] = (gj < g.n && gk < k_end) ? B[gk * g.b_sk + gj * g.b_sn] : 0.f;
     }
   };
   auto stash = [&](int buf) {
@@ -141,12 +152,12 @@ __global__ void __launch_bounds__(256) gemm_f32_tiled_kernel(GemmF32Args g) {
       bs[buf][kk][jj] = rb[e];
     }
   };
-  fetch(0);
+  fetch(k_begin);
   stash(0);
   __syncthreads();
   int buf = 0;
-  for (int k0 = 0; k0 < g.k; k0 += BK) {
-    const bool more = k0 + BK < g.k;
+  for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+    const bool more = k0 + BK < k_end;
     if (more) fetch(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
