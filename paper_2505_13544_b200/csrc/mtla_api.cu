@@ -1048,13 +1048,16 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
   pa.use_gate = dm.s > 1;
   pa.ln_eps = h->cfg.ln_eps;
   pa.q_scale = q_scale;
+  pa.batch = B;
   const dim3 post_grid(ceil_div(T_len, dm.s), B);
+  // The fast kernel takes one warp per (chunk, sequence), eight to a CTA.
+  const dim3 fast_grid((unsigned)(((long long)ceil_div(T_len, dm.s) * B + 7) / 8));
   const bool post_fast = (dm.proj.off_u >= 0 || !pa.use_gate) && dm.s <= kPostFastMaxStride;
   if (h->use_tc) {
-    if (post_fast) prefill_post_fast_kernel<T, bf16><<<post_grid, 256, 0, st>>>(pa);
+    if (post_fast) prefill_post_fast_kernel<T, bf16><<<fast_grid, 256, 0, st>>>(pa);
     else prefill_post_kernel<T, bf16><<<post_grid, 256, 0, st>>>(pa);
   } else {
-    if (post_fast) prefill_post_fast_kernel<T, float><<<post_grid, 256, 0, st>>>(pa);
+    if (post_fast) prefill_post_fast_kernel<T, float><<<fast_grid, 256, 0, st>>>(pa);
     else prefill_post_kernel<T, float><<<post_grid, 256, 0, st>>>(pa);
   }
   h->launches++;

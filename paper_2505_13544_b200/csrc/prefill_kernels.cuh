@@ -28,6 +28,7 @@ struct PrefillPostArgs {
   void* cprime;           // [B*T][r]: running merge state after each token (Eq. 14's sequence)
   void* kr;               // [B*T][d_R]: rotated RoPE key of each token (query element type)
   int n_heads, head_dim, r, dr, dw, stride, T, max_slots;
+  int batch;              // sequences of the call (prefill_post_fast_kernel's grid is flat)
   int use_gate;
   float ln_eps, q_scale;
 };
@@ -121,45 +122,70 @@ __global__ void __launch_bounds__(256) prefill_post_kernel(PrefillPostArgs a) {
     for (int i = tid; i < a.r; i += 256) a.open_acc[(long long)(a.seq0 + b) * a.r + i] = acc_s[i];
 }
 
+// Stores four / two consecutive values in the element type of the destination (16 / 8 bytes of
+// fp32, 8 / 4 bytes of bf16; the address is aligned to the access).
+__device__ __forceinline__ void put4(float* p, float v0, float v1, float v2, float v3) {
+  *reinterpret_cast<float4*>(p) = make_float4(v0, v1, v2, v3);
+}
+__device__ __forceinline__ void put4(bf16* p, float v0, float v1, float v2, float v3) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v0, v1), b = __floats2bfloat162_rn(v2, v3);
+  *reinterpret_cast<uint2*>(p) =
+      make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+}
+__device__ __forceinline__ void put2(float* p, float v0, float v1) {
+  *reinterpret_cast<float2*>(p) = make_float2(v0, v1);
+}
+__device__ __forceinline__ void put2(bf16* p, float v0, float v1) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(v0, v1);
+}
+
 // The same work for layers whose gate needs no matrix (folded into the projection, or absent at
-// s = 1) and whose stride is at most 8: the tokens of a chunk are normalised and gated in
-// parallel, one warp per token, and only the running sum walks them in order (in the same fp32
-// order as the decode steps).  One CTA of 256 threads per (chunk, sequence).
+// s = 1) and whose stride is at most 8, laid out for bandwidth: ONE WARP per (chunk, sequence),
+// eight chunks per CTA, no shared memory and no block-wide barrier.  The warp walks the chunk's
+// tokens in order; lane l owns latent columns 128 k + 4 l .. + 3 (k < 4), so the projection row is
+// read and the running state written 16 bytes at a time, the LayerNorm statistics are warp
+// shuffles, and the running sum lives in registers and grows in the same fp32 order as the
+// decode steps form it.  Queries and RoPE queries / keys move as 16- and 8-byte vectors too.
 constexpr int kPostFastMaxStride = 8;
 
 template <typename T, typename TQ>
-__global__ void __launch_bounds__(256) prefill_post_fast_kernel(PrefillPostArgs a) {
-  __shared__ float c_s[kPostFastMaxStride][512];   // normalised latents of the chunk's tokens
-  __shared__ float w_s[kPostFastMaxStride];        // their merge weights
-  const int chunk = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-  const int warp = tid >> 5, lane = tid & 31;
+__global__ void __launch_bounds__(256, 3) prefill_post_fast_kernel(PrefillPostArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int chunks = (a.T + a.stride - 1) / a.stride;
+  const long long unit = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);    // (sequence, chunk)
+  if (unit >= (long long)a.batch * chunks) return;
+  const int b = (int)(unit / chunks), chunk = (int)(unit % chunks);
   const int W = a.r + a.dr, DQ = a.head_dim + a.dr, half = a.dr / 2;
   const int tok0 = chunk * a.stride, ntok = min(a.T, tok0 + a.stride) - tok0;
   const long long row0 = (long long)b * a.T + tok0;
+  const int hd = a.n_heads * a.head_dim, dh_shift = a.head_dim == 64 ? 6 : 7;   // d_h is 64 or 128
+  T* slot_row = static_cast<T*>(a.cache.base) + cache_row(a.cache, a.seq0 + b, chunk) * W;
 
-  if (warp < ntok) {
-    const float* row = a.p1 + (row0 + warp) * a.proj.width;
-    float cv[16];                                   // r <= 512: at most 16 values per lane
+  float acc[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+  for (int t = 0; t < ntok; ++t) {
+    const long long rowi = row0 + t;
+    const float* row = a.p1 + rowi * a.proj.width;
+    // Latent: LayerNorm (two-pass variance over the registers), gate, running sum.
+    float cv[16];
     float sum = 0.f;
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const int i = lane + 32 * k;
-      cv[k] = i < a.r ? row[a.proj.off_c + i] : 0.f;
-      sum += cv[k];
+    for (int k = 0; k < 4; ++k) {
+      const int i = 128 * k + 4 * lane;
+      const float4 c4 = i < a.r ? *reinterpret_cast<const float4*>(row + a.proj.off_c + i)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+      cv[4 * k] = c4.x; cv[4 * k + 1] = c4.y; cv[4 * k + 2] = c4.z; cv[4 * k + 3] = c4.w;
+      sum += (c4.x + c4.y) + (c4.z + c4.w);
     }
     const float mean = warp_sum(sum) / a.r;
     float sq = 0.f;
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
-      const float dlt = lane + 32 * k < a.r ? cv[k] - mean : 0.f;
+      const float dlt = 128 * (k / 4) + 4 * lane < a.r ? cv[k] - mean : 0.f;
       sq += dlt * dlt;
     }
     const float rstd = rsqrtf(warp_sum(sq) / a.r + a.ln_eps);
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const int i = lane + 32 * k;
-      if (i < a.r) c_s[warp][i] = (cv[k] - mean) * rstd * a.gamma[i] + a.beta[i];
-    }
     float w = 1.f;
     if (a.use_gate) {
       const float* u = row + a.proj.off_u;
@@ -171,54 +197,81 @@ __global__ void __launch_bounds__(256) prefill_post_fast_kernel(PrefillPostArgs 
       }
       w = 1.f / (1.f + expf(-warp_sum(prod)));
     }
-    if (lane == 0) w_s[warp] = w;
-  }
-  __syncthreads();
-
-  // Running merge state after each token (Eq. 14's sequence), final state into the cache.
-  T* slot_row = static_cast<T*>(a.cache.base) + cache_row(a.cache, a.seq0 + b, chunk) * W;
-  for (int i = tid; i < a.r; i += 256) {
-    float acc = 0.f;
-    for (int t = 0; t < ntok; ++t) {
-      acc += w_s[t] * c_s[t][i];
-      static_cast<T*>(a.cprime)[(row0 + t) * a.r + i] = Elem<T>::from_float(acc);
+    T* cp = static_cast<T*>(a.cprime) + rowi * a.r;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = 128 * k + 4 * lane;
+      if (i >= a.r) continue;
+      const float4 g4 = *reinterpret_cast<const float4*>(a.gamma + i);
+      const float4 b4 = *reinterpret_cast<const float4*>(a.beta + i);
+      const float gam[4] = {g4.x, g4.y, g4.z, g4.w}, bet[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float c = (cv[4 * k + e] - mean) * rstd * gam[e] + bet[e];
+        acc[4 * k + e] += w * c;
+      }
+      put4(cp + i, acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
     }
-    slot_row[i] = Elem<T>::from_float(acc);
-    if (tok0 + ntok == a.T) a.open_acc[(long long)(a.seq0 + b) * a.r + i] = acc;
-  }
-  // RoPE keys (rounded to the cache type, which is what decoding reads back); the slot keeps
-  // the key of the chunk's last token.
-  for (int idx = tid; idx < ntok * half; idx += 256) {
-    const int t = idx / half, k = idx % half;
-    const float* row = a.p1 + (row0 + t) * a.proj.width;
-    const float cs = a.rope_cos[(long long)(tok0 + t) * half + k], sn = a.rope_sin[(long long)(tok0 + t) * half + k];
-    const float x0 = row[a.proj.off_kr + 2 * k], x1 = row[a.proj.off_kr + 2 * k + 1];
-    const T k0 = Elem<T>::from_float(x0 * cs - x1 * sn), k1 = Elem<T>::from_float(x0 * sn + x1 * cs);
-    TQ* kr = static_cast<TQ*>(a.kr) + (row0 + t) * a.dr;
-    kr[2 * k] = Elem<TQ>::from_float(Elem<T>::to_float(k0));
-    kr[2 * k + 1] = Elem<TQ>::from_float(Elem<T>::to_float(k1));
-    if (t == ntok - 1) {
-      slot_row[a.r + 2 * k] = k0;
-      slot_row[a.r + 2 * k + 1] = k1;
+    // RoPE key (rounded to the cache type, which is what decoding reads back); the slot keeps
+    // the key of the chunk's last token.
+    const float* cs_row = a.rope_cos + (long long)(tok0 + t) * half;
+    const float* sn_row = a.rope_sin + (long long)(tok0 + t) * half;
+    if (lane < half) {
+      const float2 x = *reinterpret_cast<const float2*>(row + a.proj.off_kr + 2 * lane);
+      const float cs = cs_row[lane], sn = sn_row[lane];
+      const float k0 = Elem<T>::to_float(Elem<T>::from_float(x.x * cs - x.y * sn));
+      const float k1 = Elem<T>::to_float(Elem<T>::from_float(x.x * sn + x.y * cs));
+      put2(static_cast<TQ*>(a.kr) + rowi * a.dr + 2 * lane, k0, k1);
+      if (t == ntok - 1) put2(slot_row + a.r + 2 * lane, k0, k1);
+    }
+    // Scaled queries, four columns per lane and step (they never straddle a head).
+    TQ* qrow = static_cast<TQ*>(a.qcat) + rowi * a.n_heads * DQ;
+    // (Four loads are issued before the first store: the compiler cannot move a load over a
+    // store to another buffer by itself.)
+    for (int i0 = 4 * lane; i0 < hd; i0 += 512) {
+      float4 q4[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + 128 * j < hd) q4[j] = *reinterpret_cast<const float4*>(row + a.proj.off_q + i0 + 128 * j);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int i = i0 + 128 * j;
+        if (i < hd)
+          put4(qrow + (i >> dh_shift) * DQ + (i & (a.head_dim - 1)), q4[j].x * a.q_scale,
+               q4[j].y * a.q_scale, q4[j].z * a.q_scale, q4[j].w * a.q_scale);
+      }
+    }
+    // Rotated, scaled RoPE queries, one pair per lane and step.
+    // Pair idx of the row = pair idx mod (d_R / 2) of head idx / (d_R / 2); the pairs of a row are
+    // contiguous in the projection, so lane and step index them directly.
+    const int half_shift = half == 16 ? 4 : 5;                      // d_R is 32 or 64
+    for (int i0 = lane; i0 < a.n_heads * half; i0 += 128) {
+      float2 x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i0 + 32 * j < a.n_heads * half)
+          x[j] = *reinterpret_cast<const float2*>(row + a.proj.off_qr + 2 * (i0 + 32 * j));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int idx = i0 + 32 * j;
+        if (idx >= a.n_heads * half) continue;
+        const int h = idx >> half_shift, k = idx & (half - 1);
+        const float cs = cs_row[k], sn = sn_row[k];
+        put2(qrow + h * DQ + a.head_dim + 2 * k, (x[j].x * cs - x[j].y * sn) * a.q_scale,
+             (x[j].x * sn + x[j].y * cs) * a.q_scale);
+      }
     }
   }
-  // Scaled queries and rotated, scaled RoPE queries.
-  const int hd = a.n_heads * a.head_dim;
-  for (int idx = tid; idx < ntok * hd; idx += 256) {
-    const int t = idx / hd, i = idx % hd;
-    const float* row = a.p1 + (row0 + t) * a.proj.width;
-    static_cast<TQ*>(a.qcat)[(row0 + t) * a.n_heads * DQ + (i / a.head_dim) * DQ + i % a.head_dim] =
-        Elem<TQ>::from_float(row[a.proj.off_q + i] * a.q_scale);
-  }
-  const int nqr = a.n_heads * half;
-  for (int idx = tid; idx < ntok * nqr; idx += 256) {
-    const int t = idx / nqr, i = idx % nqr, h = i / half, k = i % half;
-    const float* row = a.p1 + (row0 + t) * a.proj.width;
-    const float cs = a.rope_cos[(long long)(tok0 + t) * half + k], sn = a.rope_sin[(long long)(tok0 + t) * half + k];
-    const float x0 = row[a.proj.off_qr + h * a.dr + 2 * k], x1 = row[a.proj.off_qr + h * a.dr + 2 * k + 1];
-    TQ* qc = static_cast<TQ*>(a.qcat) + (row0 + t) * a.n_heads * DQ + h * DQ + a.head_dim;
-    qc[2 * k] = Elem<TQ>::from_float((x0 * cs - x1 * sn) * a.q_scale);
-    qc[2 * k + 1] = Elem<TQ>::from_float((x0 * sn + x1 * cs) * a.q_scale);
+  // The chunk's final state is what the cache holds; the last, still open chunk also leaves its
+  // fp32 sum for the decode steps that follow.
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int i = 128 * k + 4 * lane;
+    if (i >= a.r) continue;
+    put4(slot_row + i, acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
+    if (tok0 + ntok == a.T)
+      *reinterpret_cast<float4*>(a.open_acc + (long long)(a.seq0 + b) * a.r + i) =
+          make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
   }
 }
 
