@@ -11,7 +11,9 @@
 // blocks plus two output blocks fit TMEM's 512 columns.
 //
 // A key tile beyond what query tile 0 may see (the pair's tile count follows its last row) and
-// the diagonal passes of the other query tile are simply masked out by the predicate.
+// the diagonal passes over the other query tile's tokens hold nothing a query tile may attend
+// to: that tile's issuer, softmax warps and value products skip them (`relevant` below), and
+// each query tile counts its own tiles for the parities of its score and probability buffers.
 //
 // Warp roles: warp 0 = TMA producer, warps 1-2 = score issuers of query tile 0 / 1 (warp 1 owns
 // TMEM), warp 3 = value issuer of both, warps 4-7 / 8-11 = softmax and epilogue of query tile
@@ -120,6 +122,14 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
   constexpr int DIAG = kQTiles * kQTile / KT;              // diagonal passes over the pair's own tokens
   const int n_tiles = n_kv + DIAG;
   const int hd = a.n_heads * DH;
+  // Key tiles over the closed slots that query tile 0's last row can see.
+  const int n_kv0 = ((min(a.T, q0 + kQTile) - 1) / a.stride + KT - 1) / KT;
+  // Does key tile t hold anything query tile u may see?  Closed slots up to its last row's
+  // count; of the diagonal passes, the two over its own 128 tokens.
+  auto relevant = [&](int u, int t) {
+    return t < n_kv ? (u == 1 || t < n_kv0) : (t - n_kv) * KT / kQTile == u;
+  };
+  const int n_rel[2] = {n_kv0 + kQTile / KT, n_kv + kQTile / KT};
 
   const uint32_t q_u32 = base + kOffQ, key_u32 = base + kOffKey, val_u32 = base + kOffVal;
   const uint32_t p_u32 = base + kOffP;
@@ -173,14 +183,22 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
     // ------------------------------------------------------------------ score issuer of query tile u
     const int u = warp - 1;
     bool ok = mbar_wait(bar(&bars->q_full), 0, abort_word, a.error_word, 42);
+    int c = 0;                                     // this query tile's tiles so far
     for (int t = 0; t < n_tiles && ok; ++t) {
       const int st = t % kStages;
-      ok = mbar_wait(bar(&bars->s_empty[u][t & 1]), ((t >> 1) & 1) ^ 1, abort_word, a.error_word, 43) &&
-           mbar_wait(bar(&bars->k_full[st]), (t / kStages) & 1, abort_word, a.error_word, 44);
+      // (Also for a skipped tile: the stage's previous phase must be over before this arrival
+      // may count towards the new one.)
+      ok = mbar_wait(bar(&bars->k_full[st]), (t / kStages) & 1, abort_word, a.error_word, 44);
+      if (!ok) break;
+      if (!relevant(u, t)) {
+        mbar_arrive(bar(&bars->k_empty[st]));
+        continue;
+      }
+      ok = mbar_wait(bar(&bars->s_empty[u][c & 1]), ((c >> 1) & 1) ^ 1, abort_word, a.error_word, 43);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t kbase = key_u32 + st * kKeyBytes;
-      const uint32_t d_tmem = tmem_base + (u * 2 + (t & 1)) * KT;
+      const uint32_t d_tmem = tmem_base + (u * 2 + (c & 1)) * KT;
       // K hi and K lo meet the head's queries, the RoPE keys the RoPE queries.
 #pragma unroll
       for (int kc = 0; kc < 3; ++kc) {
@@ -192,18 +210,22 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
           mma_bf16_ss(d_tmem, ad, bd, IDESC_QK, (kc > 0 || ks > 0) ? 1u : 0u);
         }
       }
-      mma_commit(bar(&bars->s_full[u][t & 1]));
+      mma_commit(bar(&bars->s_full[u][c & 1]));
       mma_commit(bar(&bars->k_empty[st]));
+      ++c;
     }
   } else if (warp == 3 && lane == 0) {
     // ------------------------------------------------------------------ value issuer (both query tiles)
     bool ok = true;
+    int cu[kQTiles] = {0, 0};                      // each query tile's tiles so far
     for (int t = 0; t < n_tiles && ok; ++t) {
       const int st = t % kStages;
       ok = mbar_wait(bar(&bars->v_full[st]), (t / kStages) & 1, abort_word, a.error_word, 45);
       const uint32_t vbase = val_u32 + st * kValBytes;
       for (int u = 0; u < kQTiles && ok; ++u) {
-        ok = mbar_wait(bar(&bars->p_full[u]), t & 1, abort_word, a.error_word, 46);
+        if (!relevant(u, t)) continue;
+        const int c = cu[u]++;
+        ok = mbar_wait(bar(&bars->p_full[u]), c & 1, abort_word, a.error_word, 46);
         if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll
@@ -211,7 +233,7 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
           // A = P [128 rows x 64 keys], K-major; B = V [d_h columns x 64 keys], MN-major.
           const uint64_t ad = make_smem_desc(p_u32 + u * kPBytes + ks * 32, 16, 1024, kSwizzle128B);
           const uint64_t bd = make_smem_desc(vbase + ks * 2048, SUB, 1024, kSwizzle128B);
-          mma_bf16_ss(tmem_base + kColO + u * 2 * DH, ad, bd, IDESC_PV, (t > 0 || ks > 0) ? 1u : 0u);
+          mma_bf16_ss(tmem_base + kColO + u * 2 * DH, ad, bd, IDESC_PV, (c > 0 || ks > 0) ? 1u : 0u);
         }
         mma_commit(bar(&bars->p_empty[u]));
       }
@@ -227,8 +249,11 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
     const uint32_t o_base = lane_base + kColO + u * 2 * DH;
     bool ok = true;
     float m_run = -INFINITY, l_run = 0.f;
+    int cnt = -1;                                  // this query tile's tiles so far
     for (int t = 0; t < n_tiles; ++t) {
-      if (ok) ok = mbar_wait(bar(&bars->s_full[u][t & 1]), (t >> 1) & 1, abort_word, a.error_word, 47);
+      if (!relevant(u, t)) continue;
+      ++cnt;
+      if (ok) ok = mbar_wait(bar(&bars->s_full[u][cnt & 1]), (cnt >> 1) & 1, abort_word, a.error_word, 47);
       ok = __all_sync(0xffffffffu, ok);                    // TMEM accesses are whole-warp operations
       if (!ok) break;
       tc_fence_after_sync();
@@ -242,11 +267,11 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
 #pragma unroll
       for (int c0 = 0; c0 < KT; c0 += 32) {
         uint32_t(&v)[32] = *reinterpret_cast<uint32_t(*)[32]>(&sv[c0]);
-        tmem_ld_x32(lane_base + (u * 2 + (t & 1)) * KT + c0, v);
+        tmem_ld_x32(lane_base + (u * 2 + (cnt & 1)) * KT + c0, v);
       }
       tmem_wait_ld();
       tc_fence_before_sync();
-      mbar_arrive(bar(&bars->s_empty[u][t & 1]));         // the scores are in registers now
+      mbar_arrive(bar(&bars->s_empty[u][cnt & 1]));       // the scores are in registers now
       uint32_t pk[KT / 2];
       // Fully visible tile and every row has a reference: probabilities at once, the tile's sum
       // tells whether a reference was outgrown (see prefill_attn_tc.cuh).
@@ -277,9 +302,9 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
         const bool raise = mt > m_run + kRescaleThreshold;
         const float m_new = raise ? mt : m_run;
         const float fac = (raise && m_run != -INFINITY) ? exp2f(m_run - m_new) : 1.f;
-        if (__any_sync(0xffffffffu, raise && t > 0)) {
+        if (__any_sync(0xffffffffu, raise && cnt > 0)) {
           // O rows are scaled to the old references: wait for the previous tile's value MMAs.
-          ok = mbar_wait(bar(&bars->p_empty[u]), (t & 1) ^ 1, abort_word, a.error_word, 48);
+          ok = mbar_wait(bar(&bars->p_empty[u]), (cnt & 1) ^ 1, abort_word, a.error_word, 48);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after_sync();
@@ -310,7 +335,7 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
         l_run += (lsum[0] + lsum[1]) + (lsum[2] + lsum[3]);
       }
       // This query tile's probability buffer is free once its previous value MMAs have completed.
-      ok = mbar_wait(bar(&bars->p_empty[u]), (t & 1) ^ 1, abort_word, a.error_word, 49);
+      ok = mbar_wait(bar(&bars->p_empty[u]), (cnt & 1) ^ 1, abort_word, a.error_word, 49);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       // P as the K-major, 128-byte-swizzled A operand: row r at r*128, its 16-byte piece c at
@@ -327,7 +352,7 @@ prefill_attn_tc2_kernel(const __grid_constant__ CUtensorMap q_map,
       mbar_arrive(bar(&bars->p_full[u]));
     }
     // Epilogue: wait for the last value MMAs, normalise this row and store hi / lo halves.
-    if (ok) ok = mbar_wait(bar(&bars->p_empty[u]), (n_tiles - 1) & 1, abort_word, a.error_word, 50);
+    if (ok) ok = mbar_wait(bar(&bars->p_empty[u]), (n_rel[u] - 1) & 1, abort_word, a.error_word, 50);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after_sync();
