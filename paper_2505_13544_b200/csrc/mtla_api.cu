@@ -1158,9 +1158,8 @@ int send_scatter(mtla_handle* h, int* dst, const std::vector<int>& idx, const st
       ops.idx[i] = idx[at + i];
       ops.val[i] = val[at + i];
     }
-    int_scatter_kernel<<<ceil_div(ops.n, 128), 128, 0, st>>>(dst, ops);
+    MTLA_CUDA(launch_kernel(int_scatter_kernel, dim3(ceil_div(ops.n, 128)), dim3(128), 0, st, true, dst, ops));
     h->launches++;
-    MTLA_CUDA(cudaGetLastError());
   }
   return MTLA_OK;
 }
@@ -1187,10 +1186,9 @@ int apply_page_ops(mtla_handle* h, const std::vector<PageSet>& sets, const std::
       ops.dst[i] = copies[at + i].dst;
       ops.rows[i] = copies[at + i].rows;
     }
-    page_copy_kernel<<<ops.n, 256, 0, st>>>(h->at<char>(h->plan.cache), page_bytes,
-                                            (int)(h->dm.W * h->dm.elem), ops);
+    MTLA_CUDA(launch_kernel(page_copy_kernel, dim3(ops.n), dim3(256), 0, st, true, h->at<char>(h->plan.cache),
+                            page_bytes, (int)(h->dm.W * h->dm.elem), ops));
     h->launches++;
-    MTLA_CUDA(cudaGetLastError());
   }
   std::vector<int> idx(sets.size()), val(sets.size());
   for (size_t i = 0; i < sets.size(); ++i) {
@@ -1868,9 +1866,8 @@ int mtla_beam_reorder(mtla_handle* h, const int32_t* parents, int32_t n_new, voi
     p.n = min(kBeamChunk, n_new - at);
     p.first = at;
     for (int i = 0; i < p.n; ++i) p.parent[i] = parents[at + i];
-    beam_gather_kernel<<<p.n, 128, 0, st>>>(a, p);
+    MTLA_CUDA(launch_kernel(beam_gather_kernel, dim3(p.n), dim3(128), 0, st, true, a, p));
     h->launches++;
-    MTLA_CUDA(cudaGetLastError());
   }
   h->pool->reorder(parents, n_new, h->batch);
   std::vector<int> moved(h->cfg.max_batch, 0);

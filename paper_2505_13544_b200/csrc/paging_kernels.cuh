@@ -2,10 +2,13 @@
 // the host-side page pool has decided (table entries, page copies, beam reordering) and that
 // move whole sequences between the paged pool and a contiguous [sequence][slot] layout.
 // Their operands travel as kernel parameters, so a call may return before the work has run
-// without any host buffer having to stay alive.
+// without any host buffer having to stay alive.  The three kernels of a beam-search step are
+// programmatic dependent launches (see sm100_ptx.cuh): they start while their predecessor drains
+// and wait before they touch memory.
 #pragma once
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace mtla {
 
@@ -17,6 +20,8 @@ struct IntScatter {          // dst[idx[i]] = val[i]
 };
 __global__ void int_scatter_kernel(int* dst, IntScatter ops) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
   if (i < ops.n) dst[ops.idx[i]] = ops.val[i];
 }
 
@@ -29,6 +34,8 @@ struct PageCopies {          // rows [0, rows[i]) of page src[i] -> page dst[i]
 __global__ void __launch_bounds__(256) page_copy_kernel(char* pool, long long page_bytes, int row_bytes,
                                                          PageCopies ops) {
   const int i = blockIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
   const uint4* s = reinterpret_cast<const uint4*>(pool + ops.src[i] * page_bytes);
   uint4* d = reinterpret_cast<uint4*>(pool + ops.dst[i] * page_bytes);
   const int n = ops.rows[i] * (row_bytes / 16);
@@ -50,6 +57,8 @@ struct BeamArgs {
 // table row (the pages in use) and open-slot accumulator from the old buffers to the new ones.
 __global__ void __launch_bounds__(128) beam_gather_kernel(BeamArgs a, BeamParents p) {
   const int b = p.first + blockIdx.x, src = p.parent[blockIdx.x];
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
   const int tokens = a.tokens_old[src];
   if (threadIdx.x == 0) a.tokens_new[b] = tokens;
   const int pages = ceil_div(ceil_div(tokens, a.stride), 64);
