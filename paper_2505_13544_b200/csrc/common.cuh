@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace mtla {
 
 typedef __nv_bfloat16 bf16;
@@ -95,6 +97,25 @@ __device__ inline float block_sum(float v, float* scratch) {
   }
   __syncthreads();
   return scratch[32];
+}
+
+// Launches `kernel`; with `dependent` it may start its prologue while the previous kernel on
+// the stream is still running (programmatic dependent launch: the kernel itself waits, with
+// griddepcontrol.wait, before it touches that kernel's data).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                          cudaStream_t st, bool dependent, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 }  // namespace mtla

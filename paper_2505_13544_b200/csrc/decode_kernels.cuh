@@ -390,6 +390,8 @@ __global__ void __launch_bounds__(256) decode_attn_fma_kernel(AttnArgs a) {
   float* m_s = ps + TS * NH;
   float* fac_s = m_s + NH;
   const int tid = threadIdx.x, b = blockIdx.y, split = blockIdx.x;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();   // the query and the cache row are the previous kernels' output
   const int slot0 = split * a.slots_per_split;
   // A split beyond a short sequence's end leaves an empty partial (maximum -inf, sum 0).
   const int n_slots = a.seq_tokens ? ceil_div(a.seq_tokens[b], a.stride) : a.n_slots;
@@ -515,6 +517,8 @@ struct CombineArgs {
 template <typename T>
 __global__ void __launch_bounds__(128) decode_combine_kernel(CombineArgs a) {
   const int h = blockIdx.x, b = blockIdx.y;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
   float m = -INFINITY;
   for (int sp = 0; sp < a.n_split; ++sp)
     m = fmaxf(m, a.ml_part[(((long long)b * a.n_split + sp) * a.n_heads + h) * 2]);

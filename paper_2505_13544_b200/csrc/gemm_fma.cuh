@@ -6,6 +6,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace mtla {
 
@@ -33,6 +34,8 @@ __global__ void __launch_bounds__(256) gemm_nt_fma_kernel(GemmArgs g) {
   TOut* c = static_cast<TOut*>(g.c) + (long long)blockIdx.z * g.zc;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();   // a no-op unless this is a programmatic dependent launch
 
   float acc[TM][TN];
 #pragma unroll
@@ -98,19 +101,18 @@ __global__ void __launch_bounds__(256) gemm_nt_fma_kernel(GemmArgs g) {
 // Launches the NT GEMM over `batches` z-slices.  K must be a multiple of the 16-byte
 // vector widths of TA and TB and all row starts 16-byte aligned (guaranteed by the caller).
 template <typename TA, typename TB, typename TOut>
-inline cudaError_t launch_gemm_nt_fma(const GemmArgs& g, int batches, cudaStream_t st) {
+inline cudaError_t launch_gemm_nt_fma(const GemmArgs& g, int batches, cudaStream_t st,
+                                      bool dependent = false) {
   if (g.m <= 0 || g.n <= 0 || batches <= 0) return cudaSuccess;
   if (g.m <= 16) {
     dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 16), batches);
-    gemm_nt_fma_kernel<TA, TB, TOut, 16><<<grid, 256, 0, st>>>(g);
+    return launch_kernel(gemm_nt_fma_kernel<TA, TB, TOut, 16>, grid, dim3(256), 0, st, dependent, g);
   } else if (g.m <= 64) {
     dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 64), batches);
-    gemm_nt_fma_kernel<TA, TB, TOut, 64><<<grid, 256, 0, st>>>(g);
-  } else {
-    dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 128), batches);
-    gemm_nt_fma_kernel<TA, TB, TOut, 128><<<grid, 256, 0, st>>>(g);
+    return launch_kernel(gemm_nt_fma_kernel<TA, TB, TOut, 64>, grid, dim3(256), 0, st, dependent, g);
   }
-  return cudaGetLastError();
+  dim3 grid(ceil_div(g.n, 64), ceil_div(g.m, 128), batches);
+  return launch_kernel(gemm_nt_fma_kernel<TA, TB, TOut, 128>, grid, dim3(256), 0, st, dependent, g);
 }
 
 }  // namespace mtla

@@ -322,12 +322,12 @@ int launch_widen(mtla_handle* h, const void* src, float* dst, long long n, cudaS
 template <typename TA, typename TB, typename TOut>
 int gemm(mtla_handle* h, const void* a, const void* bt, void* c, int m, int n, int k, int lda,
          int ldb, int ldc, float alpha, int batches, long long za, long long zb, long long zc,
-         cudaStream_t st) {
+         cudaStream_t st, bool dependent = false) {
   GemmArgs g;
   g.a = a; g.bt = bt; g.c = c; g.m = m; g.n = n; g.k = k;
   g.lda = lda; g.ldb = ldb; g.ldc = ldc; g.za = za; g.zb = zb; g.zc = zc; g.alpha = alpha;
   h->launches++;
-  return launch_gemm_nt_fma<TA, TB, TOut>(g, batches, st) == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
+  return launch_gemm_nt_fma<TA, TB, TOut>(g, batches, st, dependent) == cudaSuccess ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
 #define MTLA_TRY(expr)            \
@@ -415,25 +415,6 @@ int make_map_3d(CUtensorMap* map, const void* ptr, long long cols, long long n1,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
-}
-
-// Launches `kernel`; with `dependent` it may start its prologue while the previous kernel on
-// the stream is still running (programmatic dependent launch: the kernel itself waits, with
-// griddepcontrol.wait, before it touches that kernel's data).
-template <typename... KArgs, typename... Args>
-cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                          cudaStream_t st, bool dependent, Args&&... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = dependent ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false>
@@ -726,19 +707,19 @@ int ensure_activation_maps(mtla_handle* h, int B) {
 }
 
 template <typename T, typename TQ, int NH>
-int launch_attn_fma_rpt(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
+int launch_attn_fma_rpt(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st, bool dependent) {
   const size_t smem = attn_fma_smem_bytes(NH, a.r, a.dr);
   dim3 grid(a.n_split, B);
   if (a.r <= 256) {
     if (!h->attn_smem_ready)
       MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, TQ, NH, 1>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_attn_fma_kernel<T, TQ, NH, 1><<<grid, 256, smem, st>>>(a);
+    MTLA_CUDA(launch_kernel(decode_attn_fma_kernel<T, TQ, NH, 1>, grid, dim3(256), smem, st, dependent, a));
   } else {
     if (!h->attn_smem_ready)
       MTLA_CUDA(cudaFuncSetAttribute(decode_attn_fma_kernel<T, TQ, NH, 2>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    decode_attn_fma_kernel<T, TQ, NH, 2><<<grid, 256, smem, st>>>(a);
+    MTLA_CUDA(launch_kernel(decode_attn_fma_kernel<T, TQ, NH, 2>, grid, dim3(256), smem, st, dependent, a));
   }
   h->attn_smem_ready = true;
   h->launches++;
@@ -747,11 +728,11 @@ int launch_attn_fma_rpt(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t s
 }
 
 template <typename T, typename TQ>
-int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st) {
-  if (a.n_heads <= 4) return launch_attn_fma_rpt<T, TQ, 4>(h, a, B, st);
-  if (a.n_heads <= 8) return launch_attn_fma_rpt<T, TQ, 8>(h, a, B, st);
-  if (a.n_heads <= 16) return launch_attn_fma_rpt<T, TQ, 16>(h, a, B, st);
-  return launch_attn_fma_rpt<T, TQ, 32>(h, a, B, st);
+int launch_attn_fma(mtla_handle* h, const AttnArgs& a, int B, cudaStream_t st, bool dependent) {
+  if (a.n_heads <= 4) return launch_attn_fma_rpt<T, TQ, 4>(h, a, B, st, dependent);
+  if (a.n_heads <= 8) return launch_attn_fma_rpt<T, TQ, 8>(h, a, B, st, dependent);
+  if (a.n_heads <= 16) return launch_attn_fma_rpt<T, TQ, 16>(h, a, B, st, dependent);
+  return launch_attn_fma_rpt<T, TQ, 32>(h, a, B, st, dependent);
 }
 
 // Gang size for the paged attention launch (beam search).  The kernel needs the batch to be
@@ -836,6 +817,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   // kernel for the first one), and it waits before it touches any data.  Not while events sit
   // between the kernels.
   const bool pdl = h->use_tc && !(prof && !h->prof_attention_only);
+  const bool pdl_cc = !h->use_tc && !(prof && !h->prof_attention_only);   // the same on the CUDA-core path
   if (h->use_tc) {
     // a1 on the tensor cores: weights stream through the MMA's M side, the batch sits in N.
     MTLA_TRY(ensure_activation_maps(h, B));
@@ -848,7 +830,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
                             pdl));
   } else {
     MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.p1), B, dm.ntot, dm.d,
-                                dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
+                                dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st, pdl_cc)));
   }
 
   MTLA_TRY(prof_mark(h, prof, 1, st));
@@ -883,8 +865,8 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     else
       MTLA_CUDA(launch_kernel(decode_post_kernel<T, bf16>, dim3(B), dim3(256), 0, st, pdl, pa));
   } else {
-    if (post_fast) decode_post_fast_kernel<T, float><<<B, 256, 0, st>>>(pa);
-    else decode_post_kernel<T, float><<<B, 256, 0, st>>>(pa);
+    if (post_fast) MTLA_CUDA(launch_kernel(decode_post_fast_kernel<T, float>, dim3(B), dim3(256), 0, st, pdl_cc, pa));
+    else MTLA_CUDA(launch_kernel(decode_post_kernel<T, float>, dim3(B), dim3(256), 0, st, pdl_cc, pa));
     MTLA_CUDA(cudaGetLastError());
   }
   h->launches++;
@@ -901,7 +883,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   } else
     MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.p1) + dm.proj.off_q, h->at<T>(p.w_k),
                                     h->at<float>(p.qt), B, dm.r, dm.dh, dm.ntot, hd, dm.nh * dm.W,
-                                    pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st)));
+                                    pa.q_scale, dm.nh, dm.dh, dm.dh, dm.W, st, pdl_cc)));
 
   MTLA_TRY(prof_mark(h, prof, 3, st));
   AttnArgs aa;
@@ -961,7 +943,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
     if (n_split < 1) n_split = 1;
     aa.slots_per_split = ceil_div(ceil_div(n_slots, n_split), kAttnFmaTile) * kAttnFmaTile;
     aa.n_split = ceil_div(n_slots, aa.slots_per_split);
-    MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st)));
+    MTLA_TRY((launch_attn_fma<T, float>(h, aa, B, st, pdl_cc && !prof)));
     MTLA_TRY(prof_mark(h, prof, 4, st));
   }
 
@@ -969,7 +951,7 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   ca.o_part = aa.o_part; ca.ml_part = aa.ml_part; ca.o = h->at<void>(p.o);
   ca.n_heads = dm.nh; ca.r = dm.r; ca.n_split = aa.n_split;
   if (!h->use_tc) {
-    decode_combine_kernel<float><<<dim3(dm.nh, B), 128, 0, st>>>(ca);
+    MTLA_CUDA(launch_kernel(decode_combine_kernel<float>, dim3(dm.nh, B), dim3(128), 0, st, pdl_cc && !prof, ca));
     h->launches++;
     MTLA_CUDA(cudaGetLastError());
   }
@@ -995,10 +977,10 @@ int decode_impl(mtla_handle* h, const void* x, int B, void* y, cudaStream_t st,
   } else {
     MTLA_TRY((gemm<float, T, float>(h, h->at<float>(p.o), h->at<T>(p.w_kv_t) + (size_t)hd * dm.r,
                                     h->at<float>(p.v), B, dm.dh, dm.r, dm.nh * dm.r, dm.r, hd, 1.f,
-                                    dm.nh, dm.r, (long long)dm.dh * dm.r, dm.dh, st)));
+                                    dm.nh, dm.r, (long long)dm.dh * dm.r, dm.dh, st, pdl_cc && !prof)));
     MTLA_TRY(prof_mark(h, prof, 6, st));
     MTLA_TRY((gemm<float, T, T>(h, h->at<float>(p.v), h->at<T>(p.w_o_t), y, B, dm.d, hd, hd, hd,
-                                dm.d, 1.f, 1, 0, 0, 0, st)));
+                                dm.d, 1.f, 1, 0, 0, 0, st, pdl_cc)));
   }
   MTLA_TRY(prof_mark(h, prof, 7, st));
   if (prof) h->prof_used += MTLA_DECODE_STAGES + 1;
