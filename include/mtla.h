@@ -12,7 +12,11 @@
  *   - "device" pointers are CUDA device addresses, 16-byte aligned; "host" pointers are
  *     ordinary host addresses.  `stream` is a cudaStream_t passed as void* (NULL = the
  *     legacy default stream).  Calls enqueue work on `stream` and return; the caller
- *     synchronises.  Calls on one handle must be issued in order on one stream.
+ *     synchronises.  Calls on one handle must be issued in order on one stream.  The
+ *     kernels of a decode step are programmatic dependent launches: one may begin (its
+ *     set-up only) while earlier work on the stream is still finishing, but none reads or
+ *     writes memory before all earlier work on the stream, the caller's included, is complete,
+ *     so stream order holds for every buffer.
  *   - Ownership: the caller owns x, y, the weight buffers (may be freed once mtla_create
  *     has completed on its stream) and the arena (must outlive the handle and must not be
  *     touched while the handle lives).  The library owns only the host-side handle.
