@@ -59,6 +59,13 @@ struct GemmTcArgs {
   const float* residual;
   long long r_sm, r_sn;
   int relu;
+  // Optional second destination (the QSPLIT instantiations; the prefill's fused projection):
+  // output features below q_rows are the queries; they go, scaled and rounded to bf16, straight
+  // into the attention's query rows [token][head][q_dq] instead of the fp32 output.
+  bf16* q_out;
+  int q_rows, q_dh_shift, q_dq;   // d_h = 1 << q_dh_shift; q_dq = d_h + d_R
+  long long q_sn;                 // elements between the query rows of consecutive tokens
+  float q_scale;
   float* partial;             // [tiles][n_split][BN][128] fp32 (split-K only)
   int* tickets;               // [tiles][4], zero between launches (split-K only)
   int* error_word;
@@ -145,7 +152,7 @@ __device__ __forceinline__ float finish(const GemmTcArgs& g, float acc, int i, i
 
 }  // namespace gtc
 
-template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false>
+template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false, bool QSPLIT = false>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                GemmTcArgs g) {
@@ -256,6 +263,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       auto emit = [&](const uint32_t (&v)[32], int c0) {
         const int j0 = nt * BN + c0;
         if (!row_ok) return;
+        if constexpr (QSPLIT) {
+          if (i_row < g.q_rows) {        // uniform over the CTA: q_rows is a multiple of 128
+            bf16* p = g.q_out + (i_row >> g.q_dh_shift) * g.q_dq + (i_row & ((1 << g.q_dh_shift) - 1));
+#pragma unroll
+            for (int j = 0; j < CH; ++j)
+              if (j0 + j < g.n)
+                p[(long long)(j0 + j) * g.q_sn] = __float2bfloat16_rn(g.alpha * __uint_as_float(v[j]) * g.q_scale);
+            return;
+          }
+        }
         if (g.c_sn == 1) {
           OutT* p = c + (long long)i_row * g.c_sm + j0;
           if (g.vec_ok && g.c_lo_off == 0 && j0 + CH <= g.n) {

@@ -417,16 +417,16 @@ int make_map_3d(CUtensorMap* map, const void* ptr, long long cols, long long n1,
   return rc == CUDA_SUCCESS ? MTLA_OK : MTLA_ERR_CUDA;
 }
 
-template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false>
+template <int BN, int STAGES, typename OutT, bool HILO, bool EXTRAS = false, bool QSPLIT = false>
 int launch_gemm_tc_inst(mtla_handle* h, int inst, const CUtensorMap& ma, const CUtensorMap& mb,
                         const GemmTcArgs& g, dim3 grid, cudaStream_t st, bool dependent) {
   constexpr int smem = gtc::smem_bytes(HILO ? 2 * BN : BN, STAGES);
   if (!(h->gemm_attr_mask & (1ull << inst))) {
-    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS>,
+    MTLA_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS, QSPLIT>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     h->gemm_attr_mask |= 1ull << inst;
   }
-  MTLA_CUDA(launch_kernel(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS>, grid, dim3(192), smem, st,
+  MTLA_CUDA(launch_kernel(gemm_tc_kernel<BN, STAGES, OutT, HILO, EXTRAS, QSPLIT>, grid, dim3(192), smem, st,
                           dependent, ma, mb, g));
   h->launches++;
   return MTLA_OK;
@@ -524,6 +524,11 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
     case 256:
       // Prefill (many tiles, no split): two stages leave room for two CTAs per SM, whose epilogues
       // and main loops overlap; the weight-streaming decode products want the deeper ring.
+      if constexpr (sizeof(OutT) == 4) {
+        if (!allow_split && g.q_out)
+          return launch_gemm_tc_inst<256, 2, OutT, false, false, true>(h, 33, ma, mb, g, grid, st, dependent);
+      }
+      if (g.q_out) return MTLA_ERR_UNSUPPORTED_SHAPE;
       if (!allow_split)
         return launch_gemm_tc_inst<256, 2, OutT, false>(h, 31 + o, ma, mb, g, grid, st, dependent);
       return launch_gemm_tc_inst<256, 4, OutT, false>(h, 8 + o, ma, mb, g, grid, st, dependent);
@@ -994,15 +999,26 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
   const int hd = dm.nh * dm.dh;
   const int rows = B * T_len;
   const float q_scale = (float)(1.4426950408889634 / sqrt((double)dm.dh));
+  const bool post_fast = (dm.proj.off_u >= 0 || dm.s == 1) && dm.s <= kPostFastMaxStride;
+  const bool q_split = h->use_tc && post_fast && hd % gtc::kBM == 0;
 
   if (h->use_tc) {
     // Weights on the MMA's M side, 128 prompt rows per CTA on its N side: neighbouring CTAs
     // share an activation panel while the (small) weight matrix stays in L2.
     CUtensorMap map_x;
     MTLA_TRY(make_map_2d(&map_x, x, rows, dm.d, dm.d, kPrefillBnWide));
-    MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x,
-                            gemm_tc_args(h->at<float>(p.pf_p1), 1, dm.ntot, dm.ntot, rows, dm.d, 1.f),
-                            kPrefillBnWide, 1, false, st));
+    GemmTcArgs g1 = gemm_tc_args(h->at<float>(p.pf_p1), 1, dm.ntot, dm.ntot, rows, dm.d, 1.f);
+    if (q_split) {
+      // The query block leaves the projection kernel scaled and rounded, in the attention's
+      // layout; the post kernel then has only the latent, the gate and the RoPE vectors to do.
+      g1.q_out = h->at<bf16>(p.pf_qcat);
+      g1.q_rows = hd;
+      g1.q_dh_shift = dm.dh == 64 ? 6 : 7;
+      g1.q_dq = dm.dh + dm.dr;
+      g1.q_sn = (long long)dm.nh * (dm.dh + dm.dr);
+      g1.q_scale = q_scale;
+    }
+    MTLA_TRY(gemm_tc<float>(h, h->map_wcat, map_x, g1, kPrefillBnWide, 1, false, st));
   } else {
     MTLA_TRY((gemm<T, T, float>(h, x, h->at<T>(p.wcat_t), h->at<float>(p.pf_p1), rows, dm.ntot,
                                 dm.d, dm.d, dm.d, dm.ntot, 1.f, 1, 0, 0, 0, st)));
@@ -1034,7 +1050,7 @@ int prefill_impl(mtla_handle* h, const void* x, int seq0, int B, int T_len, void
   const dim3 post_grid(ceil_div(T_len, dm.s), B);
   // The fast kernel takes one warp per (chunk, sequence), eight to a CTA.
   const dim3 fast_grid((unsigned)(((long long)ceil_div(T_len, dm.s) * B + 7) / 8));
-  const bool post_fast = (dm.proj.off_u >= 0 || !pa.use_gate) && dm.s <= kPostFastMaxStride;
+  pa.q_done = q_split ? 1 : 0;
   if (h->use_tc) {
     if (post_fast) prefill_post_fast_kernel<T, bf16><<<fast_grid, 256, 0, st>>>(pa);
     else prefill_post_kernel<T, bf16><<<post_grid, 256, 0, st>>>(pa);

@@ -29,6 +29,7 @@ struct PrefillPostArgs {
   void* kr;               // [B*T][d_R]: rotated RoPE key of each token (query element type)
   int n_heads, head_dim, r, dr, dw, stride, T, max_slots;
   int batch;              // sequences of the call (prefill_post_fast_kernel's grid is flat)
+  int q_done;             // 1: the projection kernel has already written the scaled queries to qcat
   int use_gate;
   float ln_eps, q_scale;
 };
@@ -228,7 +229,7 @@ __global__ void __launch_bounds__(256, 3) prefill_post_fast_kernel(PrefillPostAr
     TQ* qrow = static_cast<TQ*>(a.qcat) + rowi * a.n_heads * DQ;
     // (Four loads are issued before the first store: the compiler cannot move a load over a
     // store to another buffer by itself.)
-    for (int i0 = 4 * lane; i0 < hd; i0 += 512) {
+    for (int i0 = 4 * lane; i0 < hd && !a.q_done; i0 += 512) {
       float4 q4[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j)
