@@ -511,7 +511,11 @@ int gemm_tc(mtla_handle* h, const CUtensorMap& ma, const CUtensorMap& mb, GemmTc
         case 16: return launch_gemm_tc_inst<16, 4, OutT, true>(h, 10, ma, mb, g, grid, st, dependent);
         case 32: return launch_gemm_tc_inst<32, 4, OutT, true>(h, 11, ma, mb, g, grid, st, dependent);
         case 64: return launch_gemm_tc_inst<64, 3, OutT, true>(h, 12, ma, mb, g, grid, st, dependent);
-        case 128: return launch_gemm_tc_inst<128, 4, OutT, true>(h, 13, ma, mb, g, grid, st, dependent);
+        case 128:
+          // Prefill (many tiles, no split): two stages, so that two CTAs share an SM.
+          if (!allow_split)
+            return launch_gemm_tc_inst<128, 2, OutT, true>(h, 34, ma, mb, g, grid, st, dependent);
+          return launch_gemm_tc_inst<128, 4, OutT, true>(h, 13, ma, mb, g, grid, st, dependent);
         default: return MTLA_ERR_UNSUPPORTED_SHAPE;
       }
     }
